@@ -1,0 +1,99 @@
+/*
+ * gproj_attn.h -- C ABI of the fused BF16 attention forward / backward with the GProj
+ * (gauge projection) correction, for NVIDIA B200 (sm_100a).
+ *
+ * Conventions shared by every entry point
+ *   - Tensors Q, K, V, O, dO, dQ, dK, dV are DEVICE pointers to BF16 (16-bit patterns),
+ *     layout [B][H][N][d] contiguous with d fastest; base addresses 16-byte aligned.
+ *   - LSE is a DEVICE pointer to FP32 [B][H][N]: the natural-log sum-exp of the scaled scores
+ *     s_ij = softmax_scale * q_i . k_j over the row's support.
+ *   - Supported shapes: d in {64, 128}; N a positive multiple of 128; B, H >= 1; one H for
+ *     queries and keys (no grouped heads); N_q = N_k = N; causal != 0 means row i attends to j <= i.
+ *   - The caller owns all memory.  The library never allocates, frees or synchronises; work is
+ *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).
+ *   - Return value: GPROJ_OK (0) or a negative gproj_status.  Nothing throws, aborts or traps.
+ *     Inputs are never modified; outputs are fully overwritten; non-finite inputs are undefined
+ *     behaviour (the paper's error decomposition assumes finite quantities).
+ *   - Every in-kernel wait is bounded.  A wait that gives up makes the launch finish early with
+ *     undefined outputs and records a code readable through gproj_last_device_status().
+ */
+#ifndef GPROJ_ATTN_H
+#define GPROJ_ATTN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gproj_status {
+  GPROJ_OK = 0,
+  GPROJ_ERR_NULL = -1,      /* a required pointer is NULL */
+  GPROJ_ERR_SHAPE = -2,     /* unsupported d, N not a multiple of 128, non-positive dimension, size overflow */
+  GPROJ_ERR_ALIGN = -3,     /* a tensor base address is not 16-byte aligned */
+  GPROJ_ERR_WORKSPACE = -4, /* workspace NULL, misaligned or smaller than gproj_attn_bwd_workspace_bytes() */
+  GPROJ_ERR_SCALE = -5,     /* softmax_scale not finite or not > 0 */
+  GPROJ_ERR_ARCH = -6,      /* current device is not compute capability 10.x */
+  GPROJ_ERR_CUDA = -7,      /* a CUDA runtime / driver call failed (descriptor encode, launch) */
+  GPROJ_ERR_TIMEOUT = -8,   /* reported by gproj_last_device_status(): a bounded in-kernel wait gave up */
+  GPROJ_ERR_FLAGS = -9      /* unknown bit set in flags */
+} gproj_status;
+
+/* flags of gproj_attn_bwd (ablations of Section 5.2: "FA3-SBS" = both bits, "GProj-Q" = bit 1 only) */
+#define GPROJ_FLAG_NO_Q_CORRECTION 1u /* dQ = BF16(alpha * tK): Algorithm 1 line 14 without the lambda term */
+#define GPROJ_FLAG_NO_K_CORRECTION 2u /* dK = BF16(alpha * t^T Q): Algorithm 1 without Pass 2 (lines 15-18) */
+
+/*
+ * Forward: O = softmax(softmax_scale * Q K^T [causal]) V and the row log-sum-exp.
+ * Follows Eq. "row-attention" (Section 3.1) with the subtract-before-scale softmax of
+ * Eq. "gproj-forward" (Appendix "Implemented Arithmetic and Rounding", "Forward and saved state"):
+ * the unscaled row maximum is subtracted with its own FP32 rounding before the scale and the
+ * base-two exponential; the value product uses BF16 probabilities, the normaliser their FP32 values.
+ *   in : Q, K, V  (device, BF16)        out: O (device, BF16), LSE (device, FP32)
+ */
+int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE,
+                   int B, int H, int N, int d, float softmax_scale, int causal, void *stream);
+
+/*
+ * Bytes of device scratch gproj_attn_bwd needs for this shape (0 if the shape is unsupported).
+ * The paper's resource statement (Appendix "Implemented Arithmetic", "Cost") allows a query-shaped
+ * workspace and two row-statistic arrays; this implementation uses one BF16 query-shaped array
+ * (the operand BF16(lambda_i q_i) of Algorithm 1 line 17) and two FP32 row arrays (LSE in base two, D).
+ */
+size_t gproj_attn_bwd_workspace_bytes(int B, int H, int N, int d);
+
+/*
+ * Backward with the GProj correction: Algorithm 1 (Section 4), rounding points of
+ * Eq. "gproj-row-mass", "gproj-query-implemented" and "gproj-key-implemented".
+ *   D = rowsum(dO * O) from the saved BF16 O; P = exp(S - LSE); r = BF16(P); t = BF16(P (dP - D));
+ *   rho = rowsum(t), m = rowsum(r), lambda = rho / m (0 where m = 0);
+ *   dQ = BF16(alpha (tK - lambda rK));  dK = BF16(alpha (t^T Q - r^T BF16(lambda Q)));  dV = BF16(r^T dO).
+ *   in : Q, K, V, O, dO (device, BF16), LSE (device, FP32, as written by gproj_attn_fwd)
+ *   out: dQ, dK, dV (device, BF16)
+ *   workspace: device scratch, 256-byte aligned, at least gproj_attn_bwd_workspace_bytes(); contents
+ *              undefined on entry and on exit; must not be shared by calls that overlap on the GPU.
+ *   flags: 0 = full GProj; see GPROJ_FLAG_*.
+ */
+int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                   void *dQ, void *dK, void *dV,
+                   int B, int H, int N, int d, float softmax_scale, int causal,
+                   void *workspace, size_t workspace_bytes, unsigned flags, void *stream);
+
+/*
+ * Synchronises `stream`, then returns GPROJ_OK, GPROJ_ERR_TIMEOUT if any kernel launched by this
+ * library on the current device since the last call recorded an abandoned wait, or GPROJ_ERR_CUDA.
+ * If `detail` is non-NULL it receives the raw device code (0 when fine) and the code is cleared.
+ * (No counterpart in the paper: diagnostics only.)
+ */
+int gproj_last_device_status(void *stream, int *detail);
+
+/* Static, human-readable name of a status code. */
+const char *gproj_status_string(int status);
+
+/* Number of kernels the most recent successful gproj_attn_fwd / gproj_attn_bwd call on this thread launched. */
+int gproj_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPROJ_ATTN_H */

@@ -1,0 +1,16 @@
+"""B200-native fused BF16 attention forward / backward with the GProj correction.
+
+Public calls mirror the C ABI of ``include/gproj_attn.h``; they raise if the CUDA
+library has not been built or the device is not sm_100a (there is no CPU path).
+"""
+from .binding import (  # noqa: F401
+    FLAG_NO_K_CORRECTION,
+    FLAG_NO_Q_CORRECTION,
+    GprojError,
+    gproj_attn_bwd,
+    gproj_attn_bwd_workspace_bytes,
+    gproj_attn_fwd,
+    gproj_last_device_status,
+    gproj_last_launch_count,
+    status_string,
+)

@@ -1,0 +1,127 @@
+"""ctypes binding of the C ABI in ``include/gproj_attn.h`` (argument marshalling only).
+
+Every step of the attention path runs in the CUDA library; PyTorch supplies device
+memory and the stream.  There is no CPU fallback: if the library is missing or the
+device is not sm_100a the calls raise.
+"""
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libgproj_attn.so")
+
+GPROJ_OK = 0
+FLAG_NO_Q_CORRECTION = 1
+FLAG_NO_K_CORRECTION = 2
+
+EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_last_device_status",
+           "gproj_status_string", "gproj_last_launch_count")
+
+_lib = None
+
+
+class GprojError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def load():
+    """Load the shared library (no CUDA call is made by loading)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -c 'import __graft_entry__ as g; g.build()'` "
+                               "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i, f, u, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_uint, ctypes.c_size_t
+        lib.gproj_attn_fwd.restype = i
+        lib.gproj_attn_fwd.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp]
+        lib.gproj_attn_bwd_workspace_bytes.restype = sz
+        lib.gproj_attn_bwd_workspace_bytes.argtypes = [i, i, i, i]
+        lib.gproj_attn_bwd.restype = i
+        lib.gproj_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, sz, u, vp]
+        lib.gproj_last_device_status.restype = i
+        lib.gproj_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+        lib.gproj_status_string.restype = ctypes.c_char_p
+        lib.gproj_status_string.argtypes = [i]
+        lib.gproj_last_launch_count.restype = i
+        lib.gproj_last_launch_count.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load().gproj_status_string(int(status)).decode()
+
+
+def _check_bf16(name, t, shape=None):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA bfloat16 tensor")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+
+
+def _stream(device):
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def gproj_attn_bwd_workspace_bytes(B, H, N, d) -> int:
+    return int(load().gproj_attn_bwd_workspace_bytes(B, H, N, d))
+
+
+def gproj_attn_fwd(Q, K, V, softmax_scale, causal, O=None, LSE=None):
+    """O, LSE = attention forward.  Q, K, V: CUDA bfloat16 [B, H, N, d]."""
+    _check_bf16("Q", Q)
+    B, H, N, d = Q.shape
+    _check_bf16("K", K, Q.shape); _check_bf16("V", V, Q.shape)
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None:
+        LSE = torch.empty((B, H, N), dtype=torch.float32, device=Q.device)
+    _check_bf16("O", O, Q.shape)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
+                                   B, H, N, d, float(softmax_scale), int(bool(causal)), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_fwd")
+    return O, LSE
+
+
+def gproj_attn_bwd(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, workspace=None, dQ=None, dK=None, dV=None):
+    """dQ, dK, dV = attention backward with the GProj correction (flags: FLAG_NO_*_CORRECTION)."""
+    _check_bf16("Q", Q)
+    B, H, N, d = Q.shape
+    for name, t in (("K", K), ("V", V), ("O", O), ("dO", dO)):
+        _check_bf16(name, t, Q.shape)
+    if not (LSE.is_cuda and LSE.dtype == torch.float32 and LSE.is_contiguous() and tuple(LSE.shape) == (B, H, N)):
+        raise TypeError("LSE must be a contiguous CUDA float32 tensor [B, H, N]")
+    need = gproj_attn_bwd_workspace_bytes(B, H, N, d)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device)
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(Q) if dK is None else dK
+    dV = torch.empty_like(Q) if dV is None else dV
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_bwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
+                                   dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, N, d, float(softmax_scale),
+                                   int(bool(causal)), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                   int(flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_bwd")
+    return dQ, dK, dV
+
+
+def gproj_last_device_status(device=None):
+    """Synchronise the current stream and return (status, raw device code)."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    detail = ctypes.c_int(0)
+    with torch.cuda.device(device):
+        rc = load().gproj_last_device_status(_stream(device), ctypes.byref(detail))
+    return rc, detail.value
+
+
+def gproj_last_launch_count() -> int:
+    return int(load().gproj_last_launch_count())

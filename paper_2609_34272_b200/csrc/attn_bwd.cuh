@@ -1,0 +1,506 @@
+// Fused attention backward with the GProj correction for sm_100a (Algorithm 1).
+//
+// The work of Algorithm 1 is organised as two stationary kernels so that every accumulator lives
+// in TMEM from its first to its last contribution (no atomics, no BF16 round trip, deterministic):
+//
+//   bwd_dq_kernel   query tile stationary; streams 64-key steps.  Per step: S = Q K^T, dP = dO V^T
+//                   (tensor core -> TMEM), then per row (thread <-> TMEM lane): P = exp(S - LSE),
+//                   r = BF16(P), t = BF16(P (dP - D)), rho += sum t, m += sum r (sums of the ROUNDED
+//                   operands, Eq. "gproj-row-mass"), and two more contractions A += t K, B += r K with
+//                   t, r read from TMEM.  Epilogue: lambda = rho / m (0 if m = 0),
+//                   dQ = BF16(alpha (A - lambda B)) (Eq. "gproj-query-implemented"), and the scaled-query
+//                   operand of the key correction, stored negated: Z = -BF16(lambda q).
+//                   Also produces D = rowsum(dO * O) (Algorithm 1 line 1) and keeps it, with LSE in base
+//                   two, for the second kernel.
+//   bwd_dkv_kernel  key tile stationary; streams 64-query steps.  Per step: S^T = K Q^T, dP^T = V dO^T,
+//                   r^T, t^T as above (thread <-> key row; LSE, D are per-column values from shared
+//                   memory), dV += r^T dO, dK += t^T Q + r^T Z  -- the correction lands in the FP32
+//                   accumulator before the final cast (Eq. "gproj-key-implemented").
+//                   Epilogue: dK = BF16(alpha acc), dV = BF16(acc).
+//
+// Both kernels double-buffer the score tiles in TMEM: two compute warpgroups alternate steps, so the
+// tensor core works on step n+1 (and on the second-stage products of step n-1) while step n is in the ALUs.
+#pragma once
+#include "sm100_primitives.cuh"
+
+namespace gproj {
+
+constexpr unsigned kFlagNoQCorrection = 1u;
+constexpr unsigned kFlagNoKCorrection = 2u;
+
+template <int D>
+struct BwdCfg {
+  static constexpr int kSlabs = D / 64;
+  static constexpr int kBigSlabBytes = 128 * 128;                 // 128-row slab (stationary tile)
+  static constexpr int kBigTileBytes = kSlabs * kBigSlabBytes;
+  static constexpr int kStepRows = 64;                            // rows of a streamed tile
+  static constexpr int kStepSlabBytes = kStepRows * 128;
+  static constexpr int kStepTileBytes = kSlabs * kStepSlabBytes;
+  static constexpr int kThreads = 320;                            // producer warp, MMA warp, 2 compute warpgroups
+  // TMEM columns: score buffers S[2] at 0 / 64, dP[2] at 128 / 192, accumulators at 256 and 256 + D
+  static constexpr int kTmemCols = 512;
+  static constexpr uint32_t kColS = 0, kColDP = 128, kColAcc0 = 256, kColAcc1 = 256 + D;
+  // dQ-side kernel: Q, dO resident; ring of (K, V) step tiles
+  static constexpr int kDqStages = 4;
+  static constexpr int kDqStageBytes = 2 * kStepTileBytes;
+  static constexpr int kDqSmemBytes = 2 * kBigTileBytes + kDqStages * kDqStageBytes + 1024;
+  // dK/dV-side kernel: K, V resident; ring of (Q, dO, Z, stats) step tiles
+  static constexpr int kDkvStages = (D == 64) ? 4 : 3;
+  static constexpr int kDkvStageBytes = 3 * kStepTileBytes + 1024;   // + 64 x float2 row statistics (512 B used)
+  static constexpr int kDkvSmemBytes = 2 * kBigTileBytes + kDkvStages * kDkvStageBytes + 1024;
+};
+
+enum BwdWaitCode {
+  kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26,
+  kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36
+};
+
+// ============================================================================================
+// dQ side
+// ============================================================================================
+template <int D, bool CAUSAL>
+__global__ void __launch_bounds__(320, 1)
+bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
+              const __grid_constant__ CUtensorMap tmdO,   // box 64 x 128 rows
+              const __grid_constant__ CUtensorMap tmK,    // box 64 x 64 rows
+              const __grid_constant__ CUtensorMap tmV,    // box 64 x 64 rows
+              const __nv_bfloat16 *__restrict__ Qg, const __nv_bfloat16 *__restrict__ Og,
+              const __nv_bfloat16 *__restrict__ dOg, const float *__restrict__ LSE,
+              __nv_bfloat16 *__restrict__ dQ, __nv_bfloat16 *__restrict__ Zneg, float2 *__restrict__ stats,
+              int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
+  using C = BwdCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t *sQ = smem;
+  uint8_t *sdO = sQ + C::kBigTileBytes;
+  uint8_t *sKV = sdO + C::kBigTileBytes;    // stage s: K step tile, then V step tile
+
+  __shared__ uint64_t bar_q, bar_kv_full[C::kDqStages], bar_kv_empty[C::kDqStages];
+  __shared__ uint64_t bar_sdp_full[2], bar_tr_ready[2], bar_acc_done;
+  __shared__ uint32_t tmem_base_smem;
+  __shared__ int cta_abort, cta_skip;
+  __shared__ float s_rho[128], s_m[128], s_lam[128];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
+  __syncthreads();
+  if (cta_skip != 0) return;
+
+  const int n_qt = N / 128;
+  const int lin = blockIdx.x;
+  const int qt = CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH);
+  const int bh = lin % BH;
+  const int T = CAUSAL ? 2 * (qt + 1) : N / C::kStepRows;       // 64-key steps
+  const int row0 = bh * N + qt * 128;
+
+  AbortState ab{status, &cta_abort};
+  if (threadIdx.x == 0) {
+    cta_abort = 0;
+    mbar_init(&bar_q, 1);
+    for (int s = 0; s < C::kDqStages; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
+    mbar_init(&bar_acc_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmdO); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_smem;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(&bar_q, 2 * C::kBigTileBytes);
+      for (int s = 0; s < C::kSlabs; ++s) {
+        tma_load_2d(sQ + s * C::kBigSlabBytes, &tmQ, &bar_q, s * 64, row0);
+        tma_load_2d(sdO + s * C::kBigSlabBytes, &tmdO, &bar_q, s * 64, row0);
+      }
+      for (int n = 0; n < T; ++n) {
+        const int st = n % C::kDqStages;
+        if (n >= C::kDqStages) mbar_wait(&bar_kv_empty[st], ((n / C::kDqStages) - 1) & 1, ab, kDqWaitKVEmpty);
+        mbar_expect_tx(&bar_kv_full[st], C::kDqStageBytes);
+        uint8_t *dst = sKV + st * C::kDqStageBytes;
+        const int krow = bh * N + n * C::kStepRows;
+        for (int s = 0; s < C::kSlabs; ++s) {
+          tma_load_2d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow);
+          tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow);
+        }
+      }
+      if (cta_abort) {
+        for (int n = (T > C::kDqStages ? T - C::kDqStages : 0); n < T; ++n)
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_kv_full[n % C::kDqStages], (n / C::kDqStages) & 1); ++spin) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- tensor-core issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 queries] x [64 keys], contraction over d
+      constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 queries] x [d], contraction over 64 keys
+      const uint32_t aQ = smem_u32(sQ), adO = smem_u32(sdO);
+      mbar_wait(&bar_q, 0, ab, kDqWaitQ);
+      for (int n = 0; n <= T; ++n) {
+        if (n < T) {
+          const int st = n % C::kDqStages, b = n & 1;
+          mbar_wait(&bar_kv_full[st], (n / C::kDqStages) & 1, ab, kDqWaitKV);
+          tc_fence_after();
+          const uint32_t aK = smem_u32(sKV + st * C::kDqStageBytes), aV = aK + C::kStepTileBytes;
+          const uint32_t tS = tmem_base + C::kColS + 64 * b, tdP = tmem_base + C::kColDP + 64 * b;
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tS, smem_desc_sw128(aQ + oa, 16, 1024), smem_desc_sw128(aK + ob, 16, 1024), idesc_s, k > 0);
+          }
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tdP, smem_desc_sw128(adO + oa, 16, 1024), smem_desc_sw128(aV + ob, 16, 1024), idesc_s, k > 0);
+          }
+          umma_commit(&bar_sdp_full[b]);
+        }
+        if (n >= 1) {
+          const int p = n - 1, st = p % C::kDqStages, b = p & 1;
+          mbar_wait(&bar_tr_ready[b], (p >> 1) & 1, ab, kDqWaitTR);
+          tc_fence_after();
+          const uint32_t aK = smem_u32(sKV + st * C::kDqStageBytes);
+          const uint32_t tR = tmem_base + C::kColS + 64 * b, tT = tmem_base + C::kColDP + 64 * b;   // packed BF16 over S / dP
+#pragma unroll
+          for (int k = 0; k < C::kStepRows / 16; ++k)
+            umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, smem_desc_sw128(aK + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
+                    (p > 0) || (k > 0));
+#pragma unroll
+          for (int k = 0; k < C::kStepRows / 16; ++k)
+            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, smem_desc_sw128(aK + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
+                    (p > 0) || (k > 0));
+          umma_commit(&bar_kv_empty[st]);
+        }
+      }
+      umma_commit(&bar_acc_done);
+    }
+  } else {
+    // ---------------------------------------------------------------- compute: thread <-> query row
+    const int wg = (warp - 2) >> 2;
+    const int row = 32 * (warp & 3) + lane;
+    const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
+    const size_t grow = static_cast<size_t>(row0 + row);
+
+    // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1)
+    float Dv = 0.f;
+    {
+      const uint4 *o4 = reinterpret_cast<const uint4 *>(Og + grow * D);
+      const uint4 *g4 = reinterpret_cast<const uint4 *>(dOg + grow * D);
+#pragma unroll 4
+      for (int v = 0; v < D / 8; ++v) {
+        const uint4 a = __ldg(o4 + v), b = __ldg(g4 + v);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          Dv = fmaf(bf16_lo_to_f32(aw[w]), bf16_lo_to_f32(bw[w]), Dv);
+          Dv = fmaf(bf16_hi_to_f32(aw[w]), bf16_hi_to_f32(bw[w]), Dv);
+        }
+      }
+    }
+    const float neg_lse2 = -LSE[grow] * 1.4426950408889634f;
+    if (wg == 0) stats[grow] = make_float2(neg_lse2, Dv);
+
+    float rho = 0.f, msum = 0.f;
+    for (int n = wg; n < T; n += 2) {
+      mbar_wait(&bar_sdp_full[wg], (n >> 1) & 1, ab, kDqWaitSdP);
+      tc_fence_after();
+      const uint32_t tS = tmem_base + C::kColS + 64 * wg + lane_addr, tdP = tmem_base + C::kColDP + 64 * wg + lane_addr;
+      const bool diag = CAUSAL && (n >= T - 2);
+      const int kcol0 = n * C::kStepRows - qt * 128;      // key index of column 0 relative to this tile's first query
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t xs[32], xp[32];
+        tmem_ld32(tS + 32 * c, xs);
+        tmem_ld32(tdP + 32 * c, xp);
+        tmem_wait_ld();
+        uint32_t pr[16], pt[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, neg_lse2));
+          float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, neg_lse2));
+          if (diag) {
+            if (kcol0 + 32 * c + 2 * i > row) p0 = 0.f;
+            if (kcol0 + 32 * c + 2 * i + 1 > row) p1 = 0.f;
+          }
+          const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), Dv));
+          const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), Dv));
+          const uint32_t rp = pack_bf16x2(p0, p1), tp = pack_bf16x2(t0, t1);
+          msum += bf16_lo_to_f32(rp); msum += bf16_hi_to_f32(rp);
+          rho += bf16_lo_to_f32(tp); rho += bf16_hi_to_f32(tp);
+          pr[i] = rp; pt[i] = tp;
+        }
+        tmem_st16(tS + 16 * c, pr);      // r over the consumed S columns
+        tmem_st16(tdP + 16 * c, pt);     // t over the consumed dP columns
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bar_tr_ready[wg]);
+    }
+
+    // ---- row statistics of both warpgroups, lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
+    if (wg == 1) { s_rho[row] = rho; s_m[row] = msum; }
+    named_bar_sync(1, 256);
+    if (wg == 0) {
+      rho += s_rho[row]; msum += s_m[row];
+      s_lam[row] = (msum != 0.f) ? __fdiv_rn(rho, msum) : 0.f;
+    }
+    named_bar_sync(1, 256);
+    const float lam = s_lam[row];
+    const float lam_q = (flags & kFlagNoQCorrection) ? 0.f : lam;
+    const float lam_k = (flags & kFlagNoKCorrection) ? 0.f : lam;
+
+    mbar_wait(&bar_acc_done, 0, ab, kDqWaitAcc);
+    tc_fence_after();
+    // each warpgroup finishes half of the d columns
+#pragma unroll
+    for (int cc = 0; cc < D / 64; ++cc) {
+      const int col = wg * (D / 2) + 32 * cc;
+      uint32_t a[32], b[32];
+      tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
+      tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);
+      tmem_wait_ld();
+      const uint4 *q4 = reinterpret_cast<const uint4 *>(Qg + grow * D + col);
+      uint4 *dq4 = reinterpret_cast<uint4 *>(dQ + grow * D + col);
+      uint4 *z4 = reinterpret_cast<uint4 *>(Zneg + grow * D + col);
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const uint4 qv = __ldg(q4 + v);
+        const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
+        uint32_t dqw[4], zw[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const int i = 8 * v + 2 * w;
+          const float g0 = __fmul_rn(alpha, __fsub_rn(__uint_as_float(a[i]), __fmul_rn(lam_q, __uint_as_float(b[i]))));
+          const float g1 = __fmul_rn(alpha, __fsub_rn(__uint_as_float(a[i + 1]), __fmul_rn(lam_q, __uint_as_float(b[i + 1]))));
+          dqw[w] = pack_bf16x2(g0, g1);
+          // z = BF16(fl32[lambda q]); the sign flip is exact
+          zw[w] = pack_bf16x2(__fmul_rn(lam_k, bf16_lo_to_f32(qw[w])), __fmul_rn(lam_k, bf16_hi_to_f32(qw[w]))) ^ 0x80008000u;
+        }
+        dq4[v] = make_uint4(dqw[0], dqw[1], dqw[2], dqw[3]);
+        z4[v] = make_uint4(zw[0], zw[1], zw[2], zw[3]);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
+}
+
+// ============================================================================================
+// dK / dV side
+// ============================================================================================
+template <int D, bool CAUSAL>
+__global__ void __launch_bounds__(320, 1)
+bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
+               const __grid_constant__ CUtensorMap tmV,    // box 64 x 128 rows
+               const __grid_constant__ CUtensorMap tmQ,    // box 64 x 64 rows
+               const __grid_constant__ CUtensorMap tmdO,   // box 64 x 64 rows
+               const __grid_constant__ CUtensorMap tmZ,    // box 64 x 64 rows
+               const float2 *__restrict__ stats, __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV,
+               int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
+  using C = BwdCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t *sK = smem;
+  uint8_t *sV = sK + C::kBigTileBytes;
+  uint8_t *sStage = sV + C::kBigTileBytes;   // stage s: Q, dO, Z step tiles, then 64 x float2 {-LSE log2 e, D}
+
+  __shared__ uint64_t bar_kv, bar_q_full[C::kDkvStages], bar_q_empty[C::kDkvStages];
+  __shared__ uint64_t bar_sdp_full[2], bar_tr_ready[2], bar_acc_done;
+  __shared__ uint32_t tmem_base_smem;
+  __shared__ int cta_abort, cta_skip;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
+  __syncthreads();
+  if (cta_skip != 0) return;
+
+  const int n_kt = N / 128;
+  const int lin = blockIdx.x;
+  const int kt = lin / BH;                                   // causal: key tile 0 has the most query steps -> first
+  const int bh = lin % BH;
+  const int q_start = CAUSAL ? kt * 128 : 0;
+  const int T = (N - q_start) / C::kStepRows;                 // 64-query steps
+  const int krow0 = bh * N + kt * 128;
+  const bool use_z = (flags & kFlagNoKCorrection) == 0;
+  const uint32_t stage_tx = (use_z ? 3 : 2) * C::kStepTileBytes + 512;
+  (void)n_kt;
+
+  AbortState ab{status, &cta_abort};
+  if (threadIdx.x == 0) {
+    cta_abort = 0;
+    mbar_init(&bar_kv, 1);
+    for (int s = 0; s < C::kDkvStages; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
+    mbar_init(&bar_acc_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmdO); tma_prefetch_desc(&tmZ);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_smem;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(&bar_kv, 2 * C::kBigTileBytes);
+      for (int s = 0; s < C::kSlabs; ++s) {
+        tma_load_2d(sK + s * C::kBigSlabBytes, &tmK, &bar_kv, s * 64, krow0);
+        tma_load_2d(sV + s * C::kBigSlabBytes, &tmV, &bar_kv, s * 64, krow0);
+      }
+      for (int n = 0; n < T; ++n) {
+        const int st = n % C::kDkvStages;
+        if (n >= C::kDkvStages) mbar_wait(&bar_q_empty[st], ((n / C::kDkvStages) - 1) & 1, ab, kDkvWaitQEmpty);
+        mbar_expect_tx(&bar_q_full[st], stage_tx);
+        uint8_t *dst = sStage + st * C::kDkvStageBytes;
+        const int qrow = bh * N + q_start + n * C::kStepRows;
+        for (int s = 0; s < C::kSlabs; ++s) {
+          tma_load_2d(dst + s * C::kStepSlabBytes, &tmQ, &bar_q_full[st], s * 64, qrow);
+          tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow);
+          if (use_z) tma_load_2d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow);
+        }
+        bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + qrow, 512, &bar_q_full[st]);
+      }
+      if (cta_abort) {
+        for (int n = (T > C::kDkvStages ? T - C::kDkvStages : 0); n < T; ++n)
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full[n % C::kDkvStages], (n / C::kDkvStages) & 1); ++spin) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- tensor-core issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 keys] x [64 queries], contraction over d
+      constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 keys] x [d], contraction over 64 queries
+      const uint32_t aK = smem_u32(sK), aV = smem_u32(sV);
+      mbar_wait(&bar_kv, 0, ab, kDkvWaitKV);
+      for (int n = 0; n <= T; ++n) {
+        if (n < T) {
+          const int st = n % C::kDkvStages, b = n & 1;
+          mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);
+          tc_fence_after();
+          const uint32_t aQ = smem_u32(sStage + st * C::kDkvStageBytes), adO = aQ + C::kStepTileBytes;
+          const uint32_t tS = tmem_base + C::kColS + 64 * b, tdP = tmem_base + C::kColDP + 64 * b;
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tS, smem_desc_sw128(aK + oa, 16, 1024), smem_desc_sw128(aQ + ob, 16, 1024), idesc_s, k > 0);
+          }
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tdP, smem_desc_sw128(aV + oa, 16, 1024), smem_desc_sw128(adO + ob, 16, 1024), idesc_s, k > 0);
+          }
+          umma_commit(&bar_sdp_full[b]);
+        }
+        if (n >= 1) {
+          const int p = n - 1, st = p % C::kDkvStages, b = p & 1;
+          mbar_wait(&bar_tr_ready[b], (p >> 1) & 1, ab, kDkvWaitTR);
+          tc_fence_after();
+          const uint32_t aQ = smem_u32(sStage + st * C::kDkvStageBytes), adO = aQ + C::kStepTileBytes, aZ = adO + C::kStepTileBytes;
+          const uint32_t tR = tmem_base + C::kColS + 64 * b, tT = tmem_base + C::kColDP + 64 * b;
+#pragma unroll
+          for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
+            umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, smem_desc_sw128(adO + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
+                    (p > 0) || (k > 0));
+#pragma unroll
+          for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
+            umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, smem_desc_sw128(aQ + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
+                    (p > 0) || (k > 0));
+          if (use_z) {
+#pragma unroll
+            for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
+              umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, smem_desc_sw128(aZ + k * 2048, C::kStepSlabBytes, 1024), idesc_a, 1);
+          }
+          umma_commit(&bar_q_empty[st]);
+        }
+      }
+      umma_commit(&bar_acc_done);
+    }
+  } else {
+    // ---------------------------------------------------------------- compute: thread <-> key row
+    const int wg = (warp - 2) >> 2;
+    const int row = 32 * (warp & 3) + lane;                  // key row within the tile
+    const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
+
+    for (int n = wg; n < T; n += 2) {
+      const int st = n % C::kDkvStages;
+      mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);      // row statistics of this step landed
+      mbar_wait(&bar_sdp_full[wg], (n >> 1) & 1, ab, kDkvWaitSdP);
+      tc_fence_after();
+      const float4 *st4 = reinterpret_cast<const float4 *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
+      const uint32_t tS = tmem_base + C::kColS + 64 * wg + lane_addr, tdP = tmem_base + C::kColDP + 64 * wg + lane_addr;
+      const bool diag = CAUSAL && (n < 2);
+      const int qcol0 = n * C::kStepRows;                     // query index of column 0 relative to this tile's first key
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t xs[32], xp[32];
+        tmem_ld32(tS + 32 * c, xs);
+        tmem_ld32(tdP + 32 * c, xp);
+        tmem_wait_ld();
+        uint32_t pr[16], pt[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float4 sd = st4[16 * c + i];                  // {-lse2, D} of columns 32c+2i and 32c+2i+1
+          float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, sd.x));
+          float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, sd.z));
+          if (diag) {
+            if (row > qcol0 + 32 * c + 2 * i) p0 = 0.f;
+            if (row > qcol0 + 32 * c + 2 * i + 1) p1 = 0.f;
+          }
+          const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), sd.y));
+          const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), sd.w));
+          pr[i] = pack_bf16x2(p0, p1);
+          pt[i] = pack_bf16x2(t0, t1);
+        }
+        tmem_st16(tS + 16 * c, pr);
+        tmem_st16(tdP + 16 * c, pt);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bar_tr_ready[wg]);
+    }
+
+    mbar_wait(&bar_acc_done, 0, ab, kDkvWaitAcc);
+    tc_fence_after();
+    const size_t grow = static_cast<size_t>(krow0 + row);
+#pragma unroll
+    for (int cc = 0; cc < D / 64; ++cc) {
+      const int col = wg * (D / 2) + 32 * cc;
+      uint32_t a[32], b[32];
+      tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
+      tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);
+      tmem_wait_ld();
+      uint4 *dv4 = reinterpret_cast<uint4 *>(dV + grow * D + col);
+      uint4 *dk4 = reinterpret_cast<uint4 *>(dK + grow * D + col);
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        uint32_t vw[4], kw[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const int i = 8 * v + 2 * w;
+          vw[w] = pack_bf16x2(__uint_as_float(a[i]), __uint_as_float(a[i + 1]));
+          kw[w] = pack_bf16x2(__fmul_rn(alpha, __uint_as_float(b[i])), __fmul_rn(alpha, __uint_as_float(b[i + 1])));
+        }
+        dv4[v] = make_uint4(vw[0], vw[1], vw[2], vw[3]);
+        dk4[v] = make_uint4(kw[0], kw[1], kw[2], kw[3]);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
+}
+
+}  // namespace gproj

@@ -1,0 +1,229 @@
+// Host side of the C ABI declared in include/gproj_attn.h: argument checks, TMA descriptors,
+// kernel launches.  No allocation, no synchronisation (except gproj_last_device_status).
+#include "gproj_attn.h"
+
+#include <cmath>
+#include <cstdint>
+#include <mutex>
+
+#include "attn_bwd.cuh"
+#include "attn_fwd.cuh"
+
+namespace {
+
+using namespace gproj;
+
+// Launch-status word: written by a kernel whose bounded wait gave up, read back on request.
+__device__ int g_device_status;
+
+constexpr int kMaxDevices = 64;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceState {
+  bool ready = false;
+  bool arch_ok = false;
+  int *status_ptr = nullptr;
+};
+
+std::mutex g_mutex;
+DeviceState g_dev[kMaxDevices];
+EncodeTiledFn g_encode = nullptr;
+thread_local int tl_launch_count = 0;
+
+template <typename Kernel>
+cudaError_t allow_smem(Kernel kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+// One-time, per-device set-up: capability check, status word address, shared-memory opt-in.
+int device_state(DeviceState **out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GPROJ_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState &st = g_dev[dev];
+  if (!st.ready) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return GPROJ_ERR_CUDA;
+    st.arch_ok = (major == 10);
+    if (st.arch_ok) {
+      if (!g_encode) {
+        cudaDriverEntryPointQueryResult q;
+        void *fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn)
+          return GPROJ_ERR_CUDA;
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+      }
+      if (cudaGetSymbolAddress(reinterpret_cast<void **>(&st.status_ptr), g_device_status) != cudaSuccess)
+        return GPROJ_ERR_CUDA;
+      bool ok = true;
+      ok &= allow_smem(attn_fwd_kernel<64, true>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dq_kernel<64, true>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dq_kernel<64, false>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dq_kernel<128, true>, BwdCfg<128>::kDqSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dq_kernel<128, false>, BwdCfg<128>::kDqSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dkv_kernel<64, true>, BwdCfg<64>::kDkvSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dkv_kernel<64, false>, BwdCfg<64>::kDkvSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dkv_kernel<128, true>, BwdCfg<128>::kDkvSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dkv_kernel<128, false>, BwdCfg<128>::kDkvSmemBytes) == cudaSuccess;
+      if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+    }
+    st.ready = true;
+  }
+  *out = &st;
+  return st.arch_ok ? GPROJ_OK : GPROJ_ERR_ARCH;
+}
+
+// [rows x d] BF16 row-major view, box = 64 columns (128 B, one swizzle atom) x box_rows.
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, int d, int box_rows) {
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(d), rows};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(d) * 2};
+  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t elem[2] = {1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(int B, int H, int N, int d) {
+  if (B <= 0 || H <= 0 || N <= 0) return GPROJ_ERR_SHAPE;
+  if (d != 64 && d != 128) return GPROJ_ERR_SHAPE;
+  if (N % 128 != 0) return GPROJ_ERR_SHAPE;
+  const long long rows = static_cast<long long>(B) * H * N;
+  if (rows >= (1LL << 31) || static_cast<long long>(B) * H >= (1LL << 20)) return GPROJ_ERR_SHAPE;
+  if (rows / 128 >= (1LL << 31)) return GPROJ_ERR_SHAPE;
+  return GPROJ_OK;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+
+extern "C" {
+
+int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int N, int d,
+                   float softmax_scale, int causal, void *stream) {
+  if (!Q || !K || !V || !O || !LSE) return GPROJ_ERR_NULL;
+  if (int rc = check_shape(B, H, N, d)) return rc;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || (reinterpret_cast<uintptr_t>(LSE) & 3u))
+    return GPROJ_ERR_ALIGN;
+  if (!std::isfinite(softmax_scale) || !(softmax_scale > 0.f)) return GPROJ_ERR_SCALE;
+  DeviceState *st = nullptr;
+  if (int rc = device_state(&st)) return rc;
+
+  const int BH = B * H;
+  const uint64_t rows = static_cast<uint64_t>(BH) * N;
+  CUtensorMap mQ, mK, mV;
+  if (!make_map(&mQ, Q, rows, d, 128) || !make_map(&mK, K, rows, d, 128) || !make_map(&mV, V, rows, d, 128))
+    return GPROJ_ERR_CUDA;
+  const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
+  const dim3 grid(static_cast<unsigned>(BH * (N / 128)));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  __nv_bfloat16 *Ob = static_cast<__nv_bfloat16 *>(O);
+#define GPROJ_LAUNCH_FWD(DD, CC)                                                                              \
+  attn_fwd_kernel<DD, CC><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(mQ, mK, mV, Ob, LSE, N, BH, \
+                                                                                      scale_log2, softmax_scale, st->status_ptr)
+  if (d == 64) { if (causal) GPROJ_LAUNCH_FWD(64, true); else GPROJ_LAUNCH_FWD(64, false); }
+  else         { if (causal) GPROJ_LAUNCH_FWD(128, true); else GPROJ_LAUNCH_FWD(128, false); }
+#undef GPROJ_LAUNCH_FWD
+  if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
+  tl_launch_count = 1;
+  return GPROJ_OK;
+}
+
+size_t gproj_attn_bwd_workspace_bytes(int B, int H, int N, int d) {
+  if (check_shape(B, H, N, d) != GPROJ_OK) return 0;
+  const size_t rows = static_cast<size_t>(B) * H * N;
+  return align256(rows * sizeof(float2)) + align256(rows * static_cast<size_t>(d) * 2);
+}
+
+int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                   void *dQ, void *dK, void *dV, int B, int H, int N, int d, float softmax_scale, int causal,
+                   void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
+  if (!Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return GPROJ_ERR_NULL;
+  if (int rc = check_shape(B, H, N, d)) return rc;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
+      !aligned16(dK) || !aligned16(dV) || (reinterpret_cast<uintptr_t>(LSE) & 3u))
+    return GPROJ_ERR_ALIGN;
+  if (!std::isfinite(softmax_scale) || !(softmax_scale > 0.f)) return GPROJ_ERR_SCALE;
+  if (flags & ~(GPROJ_FLAG_NO_Q_CORRECTION | GPROJ_FLAG_NO_K_CORRECTION)) return GPROJ_ERR_FLAGS;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+      workspace_bytes < gproj_attn_bwd_workspace_bytes(B, H, N, d))
+    return GPROJ_ERR_WORKSPACE;
+  DeviceState *st = nullptr;
+  if (int rc = device_state(&st)) return rc;
+
+  const int BH = B * H;
+  const uint64_t rows = static_cast<uint64_t>(BH) * N;
+  float2 *stats = static_cast<float2 *>(workspace);
+  __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + align256(rows * sizeof(float2)));
+
+  CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64;
+  bool ok = make_map(&mQ128, Q, rows, d, 128) && make_map(&mdO128, dO, rows, d, 128) && make_map(&mK64, K, rows, d, 64) &&
+            make_map(&mV64, V, rows, d, 64) && make_map(&mK128, K, rows, d, 128) && make_map(&mV128, V, rows, d, 128) &&
+            make_map(&mQ64, Q, rows, d, 64) && make_map(&mdO64, dO, rows, d, 64) && make_map(&mZ64, Zneg, rows, d, 64);
+  if (!ok) return GPROJ_ERR_CUDA;
+
+  const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
+  const dim3 grid(static_cast<unsigned>(BH * (N / 128)));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __nv_bfloat16 *Qb = static_cast<const __nv_bfloat16 *>(Q), *Ob = static_cast<const __nv_bfloat16 *>(O),
+                      *dOb = static_cast<const __nv_bfloat16 *>(dO);
+  __nv_bfloat16 *dQb = static_cast<__nv_bfloat16 *>(dQ), *dKb = static_cast<__nv_bfloat16 *>(dK),
+                *dVb = static_cast<__nv_bfloat16 *>(dV);
+#define GPROJ_LAUNCH_BWD(DD, CC)                                                                                        \
+  do {                                                                                                                  \
+    bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                                 \
+        mQ128, mdO128, mK64, mV64, Qb, Ob, dOb, LSE, dQb, Zneg, stats, N, BH, scale_log2, softmax_scale, flags,         \
+        st->status_ptr);                                                                                                \
+    bwd_dkv_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                               \
+        mK128, mV128, mQ64, mdO64, mZ64, stats, dKb, dVb, N, BH, scale_log2, softmax_scale, flags, st->status_ptr);     \
+  } while (0)
+  if (d == 64) { if (causal) GPROJ_LAUNCH_BWD(64, true); else GPROJ_LAUNCH_BWD(64, false); }
+  else         { if (causal) GPROJ_LAUNCH_BWD(128, true); else GPROJ_LAUNCH_BWD(128, false); }
+#undef GPROJ_LAUNCH_BWD
+  if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
+  tl_launch_count = 2;
+  return GPROJ_OK;
+}
+
+int gproj_last_device_status(void *stream, int *detail) {
+  if (detail) *detail = 0;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return GPROJ_ERR_CUDA;
+  int code = 0;
+  if (cudaMemcpyFromSymbol(&code, g_device_status, sizeof(int)) != cudaSuccess) return GPROJ_ERR_CUDA;
+  if (code != 0) {
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return GPROJ_ERR_CUDA;
+    if (detail) *detail = code;
+    return GPROJ_ERR_TIMEOUT;
+  }
+  return GPROJ_OK;
+}
+
+const char *gproj_status_string(int status) {
+  switch (status) {
+    case GPROJ_OK: return "ok";
+    case GPROJ_ERR_NULL: return "null pointer argument";
+    case GPROJ_ERR_SHAPE: return "unsupported shape (need d in {64,128}, N a positive multiple of 128)";
+    case GPROJ_ERR_ALIGN: return "tensor base address not 16-byte aligned";
+    case GPROJ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case GPROJ_ERR_SCALE: return "softmax_scale must be finite and positive";
+    case GPROJ_ERR_ARCH: return "device is not compute capability 10.x (sm_100a)";
+    case GPROJ_ERR_CUDA: return "CUDA runtime or driver call failed";
+    case GPROJ_ERR_TIMEOUT: return "a bounded in-kernel wait gave up; outputs of that launch are undefined";
+    case GPROJ_ERR_FLAGS: return "unknown flag bit";
+    default: return "unknown status";
+  }
+}
+
+int gproj_last_launch_count(void) { return tl_launch_count; }
+
+}  // extern "C"

@@ -1,0 +1,69 @@
+"""CPU-only checks of the C-ABI library: it loads, exports what the header declares, and rejects
+bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from paper_2609_34272_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    entry.build()
+    return binding.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "gproj_attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gproj_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_and_exports_agree(lib):
+    names = declared_functions()
+    assert set(names) == set(binding.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_status_strings(lib):
+    assert binding.status_string(0) == "ok"
+    for code in range(-9, 0):
+        assert binding.status_string(code) not in ("ok", "unknown status")
+    assert binding.status_string(-99) == "unknown status"
+
+
+def test_workspace_bytes(lib):
+    # one BF16 query-shaped array + two FP32 row arrays (the paper's "Cost" paragraph allows more)
+    B, H, N, d = 2, 3, 256, 64
+    rows = B * H * N
+    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, d) == rows * 8 + rows * d * 2
+    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 0
+    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 128, 96) == 0
+
+
+def test_argument_validation_without_gpu(lib):
+    p = ctypes.c_void_p(0x1000)        # never dereferenced: validation fails first
+    bad = ctypes.c_void_p(0x1008)
+    fwd = lambda Q=p, LSE=p, B=1, H=1, N=128, d=64, scale=0.125: lib.gproj_attn_fwd(Q, p, p, p, LSE, B, H, N, d, scale, 1, None)
+    assert fwd(Q=None) == -1
+    assert fwd(N=100) == -2 and fwd(d=96) == -2 and fwd(B=0) == -2 and fwd(N=0) == -2
+    assert fwd(Q=bad) == -3
+    assert fwd(scale=0.0) == -5 and fwd(scale=float("nan")) == -5 and fwd(scale=-1.0) == -5
+    bwd = lambda ws=ctypes.c_void_p(0x1000), nbytes=1 << 30, flags=0, dQ=p: lib.gproj_attn_bwd(
+        p, p, p, p, p, p, dQ, p, p, 1, 1, 128, 64, 0.125, 1, ws, nbytes, flags, None)
+    assert bwd(dQ=None) == -1
+    assert bwd(flags=4) == -9
+    assert bwd(ws=None) == -4 and bwd(nbytes=16) == -4 and bwd(ws=ctypes.c_void_p(0x1010)) == -4
+
+
+def test_python_binding_refuses_cpu_tensors():
+    import torch
+    x = torch.zeros(1, 1, 128, 64, dtype=torch.bfloat16)
+    with pytest.raises(TypeError):
+        binding.gproj_attn_fwd(x, x, x, 0.125, True)

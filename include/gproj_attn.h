@@ -36,12 +36,17 @@ typedef enum gproj_status {
   GPROJ_ERR_ARCH = -6,      /* current device is not compute capability 10.x */
   GPROJ_ERR_CUDA = -7,      /* a CUDA runtime / driver call failed (descriptor encode, launch) */
   GPROJ_ERR_TIMEOUT = -8,   /* reported by gproj_last_device_status(): a bounded in-kernel wait gave up */
-  GPROJ_ERR_FLAGS = -9      /* unknown bit set in flags */
+  GPROJ_ERR_FLAGS = -9      /* unknown bit set in flags, or both ONLY_* bits */
 } gproj_status;
 
 /* flags of gproj_attn_bwd (ablations of Section 5.2: "FA3-SBS" = both bits, "GProj-Q" = bit 1 only) */
 #define GPROJ_FLAG_NO_Q_CORRECTION 1u /* dQ = BF16(alpha * tK): Algorithm 1 line 14 without the lambda term */
 #define GPROJ_FLAG_NO_K_CORRECTION 2u /* dK = BF16(alpha * t^T Q): Algorithm 1 without Pass 2 (lines 15-18) */
+/* Profiling aids (no counterpart in the paper): launch one of the two backward kernels only, so that it can be
+ * timed by itself.  ONLY_DKV reads the row statistics and the scaled-query operand that an earlier full or
+ * ONLY_DQ call with the same inputs left in the same workspace.  The two bits are mutually exclusive. */
+#define GPROJ_FLAG_ONLY_DQ_PASS 4u  /* writes dQ (and the workspace); dK, dV untouched */
+#define GPROJ_FLAG_ONLY_DKV_PASS 8u /* writes dK, dV; dQ untouched */
 
 /*
  * Forward: O = softmax(softmax_scale * Q K^T [causal]) V and the row log-sum-exp.

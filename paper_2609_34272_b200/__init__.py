@@ -6,6 +6,8 @@ library has not been built or the device is not sm_100a (there is no CPU path).
 from .binding import (  # noqa: F401
     FLAG_NO_K_CORRECTION,
     FLAG_NO_Q_CORRECTION,
+    FLAG_ONLY_DKV_PASS,
+    FLAG_ONLY_DQ_PASS,
     GprojError,
     gproj_attn_bwd,
     gproj_attn_bwd_workspace_bytes,

@@ -15,6 +15,8 @@ LIB_PATH = os.path.join(_PKG, "libgproj_attn.so")
 GPROJ_OK = 0
 FLAG_NO_Q_CORRECTION = 1
 FLAG_NO_K_CORRECTION = 2
+FLAG_ONLY_DQ_PASS = 4
+FLAG_ONLY_DKV_PASS = 8
 
 EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_last_device_status",
            "gproj_status_string", "gproj_last_launch_count")

@@ -153,7 +153,10 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
       !aligned16(dK) || !aligned16(dV) || (reinterpret_cast<uintptr_t>(LSE) & 3u))
     return GPROJ_ERR_ALIGN;
   if (!std::isfinite(softmax_scale) || !(softmax_scale > 0.f)) return GPROJ_ERR_SCALE;
-  if (flags & ~(GPROJ_FLAG_NO_Q_CORRECTION | GPROJ_FLAG_NO_K_CORRECTION)) return GPROJ_ERR_FLAGS;
+  if (flags & ~(GPROJ_FLAG_NO_Q_CORRECTION | GPROJ_FLAG_NO_K_CORRECTION | GPROJ_FLAG_ONLY_DQ_PASS | GPROJ_FLAG_ONLY_DKV_PASS))
+    return GPROJ_ERR_FLAGS;
+  const bool run_dq = !(flags & GPROJ_FLAG_ONLY_DKV_PASS), run_dkv = !(flags & GPROJ_FLAG_ONLY_DQ_PASS);
+  if (!run_dq && !run_dkv) return GPROJ_ERR_FLAGS;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
       workspace_bytes < gproj_attn_bwd_workspace_bytes(B, H, N, d))
     return GPROJ_ERR_WORKSPACE;
@@ -180,17 +183,19 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
                 *dVb = static_cast<__nv_bfloat16 *>(dV);
 #define GPROJ_LAUNCH_BWD(DD, CC)                                                                                        \
   do {                                                                                                                  \
-    bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                                 \
-        mQ128, mdO128, mK64, mV64, Qb, Ob, dOb, LSE, dQb, Zneg, stats, N, BH, scale_log2, softmax_scale, flags,         \
-        st->status_ptr);                                                                                                \
-    bwd_dkv_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                               \
-        mK128, mV128, mQ64, mdO64, mZ64, stats, dKb, dVb, N, BH, scale_log2, softmax_scale, flags, st->status_ptr);     \
+    if (run_dq)                                                                                                         \
+      bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                               \
+          mQ128, mdO128, mK64, mV64, Qb, Ob, dOb, LSE, dQb, Zneg, stats, N, BH, scale_log2, softmax_scale, flags,       \
+          st->status_ptr);                                                                                              \
+    if (run_dkv)                                                                                                        \
+      bwd_dkv_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
+          mK128, mV128, mQ64, mdO64, mZ64, stats, dKb, dVb, N, BH, scale_log2, softmax_scale, flags, st->status_ptr);   \
   } while (0)
   if (d == 64) { if (causal) GPROJ_LAUNCH_BWD(64, true); else GPROJ_LAUNCH_BWD(64, false); }
   else         { if (causal) GPROJ_LAUNCH_BWD(128, true); else GPROJ_LAUNCH_BWD(128, false); }
 #undef GPROJ_LAUNCH_BWD
   if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
-  tl_launch_count = 2;
+  tl_launch_count = (run_dq ? 1 : 0) + (run_dkv ? 1 : 0);
   return GPROJ_OK;
 }
 

@@ -58,7 +58,7 @@ def test_argument_validation_without_gpu(lib):
     bwd = lambda ws=ctypes.c_void_p(0x1000), nbytes=1 << 30, flags=0, dQ=p: lib.gproj_attn_bwd(
         p, p, p, p, p, p, dQ, p, p, 1, 1, 128, 64, 0.125, 1, ws, nbytes, flags, None)
     assert bwd(dQ=None) == -1
-    assert bwd(flags=4) == -9
+    assert bwd(flags=16) == -9 and bwd(flags=12) == -9
     assert bwd(ws=None) == -4 and bwd(nbytes=16) == -4 and bwd(ws=ctypes.c_void_p(0x1010)) == -4
 
 

@@ -18,8 +18,11 @@
 //                   accumulator before the final cast (Eq. "gproj-key-implemented").
 //                   Epilogue: dK = BF16(alpha acc), dV = BF16(acc).
 //
-// Both kernels double-buffer the score tiles in TMEM: two compute warpgroups alternate steps, so the
-// tensor core works on step n+1 (and on the second-stage products of step n-1) while step n is in the ALUs.
+// Pipeline.  TMEM holds kNB score buffers (S and dP of one 64-wide step each) next to the two FP32
+// accumulators: 3 buffers at d = 64, 2 at d = 128 (512 columns either way).  Compute warpgroup w owns
+// buffer w and the steps n = w (mod kNB); it overwrites the consumed S / dP columns with the packed BF16
+// operands r / t.  One warp issues every MMA: scores of step n first, then the second-stage products of
+// step n - (kNB - 1), so up to kNB steps are in flight and the tensor core works while the ALUs do.
 #pragma once
 #include "sm100_primitives.cuh"
 
@@ -36,18 +39,22 @@ struct BwdCfg {
   static constexpr int kStepRows = 64;                            // rows of a streamed tile
   static constexpr int kStepSlabBytes = kStepRows * 128;
   static constexpr int kStepTileBytes = kSlabs * kStepSlabBytes;
-  static constexpr int kThreads = 320;                            // producer warp, MMA warp, 2 compute warpgroups
-  // TMEM columns: score buffers S[2] at 0 / 64, dP[2] at 128 / 192, accumulators at 256 and 256 + D
+  static constexpr int kNB = (D == 64) ? 3 : 2;                   // score buffers = compute warpgroups
+  static constexpr int kLag = kNB - 1;                            // second-stage MMAs trail the scores by this many steps
+  static constexpr int kThreads = 64 + 128 * kNB;                 // producer warp, MMA warp, kNB compute warpgroups
+  // TMEM columns: buffer b holds S at 128 b and dP at 128 b + 64; accumulators follow
   static constexpr int kTmemCols = 512;
-  static constexpr uint32_t kColS = 0, kColDP = 128, kColAcc0 = 256, kColAcc1 = 256 + D;
+  static constexpr uint32_t kColAcc0 = 128 * kNB, kColAcc1 = 128 * kNB + D;
+  static_assert(kColAcc1 + D <= 512, "TMEM budget");
   // dQ-side kernel: Q, dO resident; ring of (K, V) step tiles
-  static constexpr int kDqStages = 4;
+  static constexpr int kDqStages = (D == 64) ? 6 : 4;
   static constexpr int kDqStageBytes = 2 * kStepTileBytes;
   static constexpr int kDqSmemBytes = 2 * kBigTileBytes + kDqStages * kDqStageBytes + 1024;
   // dK/dV-side kernel: K, V resident; ring of (Q, dO, Z, stats) step tiles
-  static constexpr int kDkvStages = (D == 64) ? 4 : 3;
+  static constexpr int kDkvStages = (D == 64) ? 5 : 3;
   static constexpr int kDkvStageBytes = 3 * kStepTileBytes + 1024;   // + 64 x float2 row statistics (512 B used)
   static constexpr int kDkvSmemBytes = 2 * kBigTileBytes + kDkvStages * kDkvStageBytes + 1024;
+  static_assert(kDqStages >= kNB + 1 && kDkvStages >= kNB + 1, "a stage stays busy until its second-stage MMAs finish");
 };
 
 enum BwdWaitCode {
@@ -55,11 +62,74 @@ enum BwdWaitCode {
   kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36
 };
 
+// One 64-column step of the dQ side for one query row.  `lim` = (row index) - (key index of column 0):
+// with MASKED, column c is beyond the causal diagonal when c > lim.
+template <bool MASKED>
+__device__ __forceinline__ void dq_step(uint32_t tS, uint32_t tdP, float scale_log2, float neg_lse2, float Dv, int lim,
+                                        float (&rho)[2], float (&msum)[2]) {
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    uint32_t xs[32], xp[32];
+    tmem_ld32(tS + 32 * c, xs);
+    tmem_ld32(tdP + 32 * c, xp);
+    tmem_wait_ld();
+    uint32_t pr[16], pt[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, neg_lse2));
+      float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, neg_lse2));
+      if (MASKED) {
+        if (32 * c + 2 * i > lim) p0 = 0.f;
+        if (32 * c + 2 * i + 1 > lim) p1 = 0.f;
+      }
+      const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), Dv));
+      const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), Dv));
+      const uint32_t rp = pack_bf16x2(p0, p1), tp = pack_bf16x2(t0, t1);
+      // row masses of the operands as rounded (two chains each, to keep the adds off one dependency chain)
+      msum[0] += bf16_lo_to_f32(rp); msum[1] += bf16_hi_to_f32(rp);
+      rho[0] += bf16_lo_to_f32(tp); rho[1] += bf16_hi_to_f32(tp);
+      pr[i] = rp; pt[i] = tp;
+    }
+    tmem_st16(tS + 16 * c, pr);      // r over the consumed S columns
+    tmem_st16(tdP + 16 * c, pt);     // t over the consumed dP columns
+  }
+}
+
+// One 64-column step of the dK/dV side for one key row.  `lim` = (key row) - (query index of column 0):
+// with MASKED, column c is a query before this key when c < lim.
+template <bool MASKED>
+__device__ __forceinline__ void dkv_step(uint32_t tS, uint32_t tdP, const float4 *st4, float scale_log2, int lim) {
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    uint32_t xs[32], xp[32];
+    tmem_ld32(tS + 32 * c, xs);
+    tmem_ld32(tdP + 32 * c, xp);
+    tmem_wait_ld();
+    uint32_t pr[16], pt[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float4 sd = st4[16 * c + i];                  // {-LSE log2 e, D} of columns 32c+2i and 32c+2i+1
+      float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, sd.x));
+      float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, sd.z));
+      if (MASKED) {
+        if (32 * c + 2 * i < lim) p0 = 0.f;
+        if (32 * c + 2 * i + 1 < lim) p1 = 0.f;
+      }
+      const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), sd.y));
+      const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), sd.w));
+      pr[i] = pack_bf16x2(p0, p1);
+      pt[i] = pack_bf16x2(t0, t1);
+    }
+    tmem_st16(tS + 16 * c, pr);
+    tmem_st16(tdP + 16 * c, pt);
+  }
+}
+
 // ============================================================================================
 // dQ side
 // ============================================================================================
 template <int D, bool CAUSAL>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(BwdCfg<D>::kThreads, 1)
 bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmdO,   // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmK,    // box 64 x 64 rows
@@ -69,6 +139,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               __nv_bfloat16 *__restrict__ dQ, __nv_bfloat16 *__restrict__ Zneg, float2 *__restrict__ stats,
               int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
+  constexpr int NB = C::kNB, LAG = C::kLag;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;
@@ -76,19 +147,19 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   uint8_t *sKV = sdO + C::kBigTileBytes;    // stage s: K step tile, then V step tile
 
   __shared__ uint64_t bar_q, bar_kv_full[C::kDqStages], bar_kv_empty[C::kDqStages];
-  __shared__ uint64_t bar_sdp_full[2], bar_tr_ready[2], bar_acc_done;
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_acc_done;
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
-  __shared__ float s_rho[128], s_m[128], s_lam[128];
+  __shared__ float s_rho[NB - 1][128], s_m[NB - 1][128], s_lam[128];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
   __syncthreads();
-  if (cta_skip != 0) return;
+  if (cta_skip != 0) return;   // an earlier wait gave up: drain the rest of the grid quickly
 
   const int n_qt = N / 128;
   const int lin = blockIdx.x;
-  const int qt = CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH);
+  const int qt = CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH);   // causal: longest rows first
   const int bh = lin % BH;
   const int T = CAUSAL ? 2 * (qt + 1) : N / C::kStepRows;       // 64-key steps
   const int row0 = bh * N + qt * 128;
@@ -98,7 +169,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     cta_abort = 0;
     mbar_init(&bar_q, 1);
     for (int s = 0; s < C::kDqStages; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
+    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
     mbar_init(&bar_acc_done, 1);
     fence_mbar_init();
   }
@@ -109,7 +180,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = tmem_base_smem;
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);   // the shuffle marks it warp-uniform
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -130,6 +201,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
           tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow);
         }
       }
+      // Every load is consumed by an MMA the epilogue waits for, so nothing is in flight at exit unless the
+      // CTA aborted; then give the copies a bounded chance to land before shared memory is released.
       if (cta_abort) {
         for (int n = (T > C::kDqStages ? T - C::kDqStages : 0); n < T; ++n)
           for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_kv_full[n % C::kDqStages], (n / C::kDqStages) & 1); ++spin) {}
@@ -137,49 +210,57 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- tensor-core issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 queries] x [64 keys], contraction over d
-      constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 queries] x [d], contraction over 64 keys
-      const uint32_t aQ = smem_u32(sQ), adO = smem_u32(sdO);
-      mbar_wait(&bar_q, 0, ab, kDqWaitQ);
-      for (int n = 0; n <= T; ++n) {
-        if (n < T) {
-          const int st = n % C::kDqStages, b = n & 1;
-          mbar_wait(&bar_kv_full[st], (n / C::kDqStages) & 1, ab, kDqWaitKV);
-          tc_fence_after();
-          const uint32_t aK = smem_u32(sKV + st * C::kDqStageBytes), aV = aK + C::kStepTileBytes;
-          const uint32_t tS = tmem_base + C::kColS + 64 * b, tdP = tmem_base + C::kColDP + 64 * b;
+    // The whole warp runs this loop so that every address stays provably warp-uniform (descriptor operands
+    // then live in uniform registers); one elected lane issues the MMAs and commits.
+    constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 queries] x [64 keys], contraction over d
+    constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 queries] x [d], contraction over 64 keys
+    const SmemDesc dscQ = make_smem_desc(smem_u32(sQ), 16, 1024), dscdO = make_smem_desc(smem_u32(sdO), 16, 1024);
+    const SmemDesc dscK0 = make_smem_desc(smem_u32(sKV), 16, 1024);                          // K-major view of stage 0
+    const SmemDesc dscK0mn = make_smem_desc(smem_u32(sKV), C::kStepSlabBytes, 1024);       // MN-major view of stage 0
+    mbar_wait(&bar_q, 0, ab, kDqWaitQ);
+    for (int n = 0; n < T + LAG; ++n) {
+      if (n < T) {
+        const int st = n % C::kDqStages, b = n % NB;
+        mbar_wait(&bar_kv_full[st], (n / C::kDqStages) & 1, ab, kDqWaitKV);
+        tc_fence_after();
+        const SmemDesc dscK = dscK0.advanced(st * C::kDqStageBytes), dscV = dscK.advanced(C::kStepTileBytes);
+        const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
+        if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tS, smem_desc_sw128(aQ + oa, 16, 1024), smem_desc_sw128(aK + ob, 16, 1024), idesc_s, k > 0);
+            umma_ss(tS, dscQ.at(oa), dscK.at(ob), idesc_s, k > 0);
           }
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tdP, smem_desc_sw128(adO + oa, 16, 1024), smem_desc_sw128(aV + ob, 16, 1024), idesc_s, k > 0);
+            umma_ss(tdP, dscdO.at(oa), dscV.at(ob), idesc_s, k > 0);
           }
           umma_commit(&bar_sdp_full[b]);
         }
-        if (n >= 1) {
-          const int p = n - 1, st = p % C::kDqStages, b = p & 1;
-          mbar_wait(&bar_tr_ready[b], (p >> 1) & 1, ab, kDqWaitTR);
-          tc_fence_after();
-          const uint32_t aK = smem_u32(sKV + st * C::kDqStageBytes);
-          const uint32_t tR = tmem_base + C::kColS + 64 * b, tT = tmem_base + C::kColDP + 64 * b;   // packed BF16 over S / dP
+        __syncwarp();
+      }
+      if (n >= LAG) {
+        const int p = n - LAG, st = p % C::kDqStages, b = p % NB;
+        mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDqWaitTR);
+        tc_fence_after();
+        const SmemDesc dscK = dscK0mn.advanced(st * C::kDqStageBytes);
+        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;     // packed BF16 r / t over the S / dP columns
+        const uint32_t acc = (p > 0) ? 1u : 0u;
+        if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)
-            umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, smem_desc_sw128(aK + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
-                    (p > 0) || (k > 0));
+            umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)
-            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, smem_desc_sw128(aK + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
-                    (p > 0) || (k > 0));
+            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
           umma_commit(&bar_kv_empty[st]);
         }
+        __syncwarp();
       }
-      umma_commit(&bar_acc_done);
     }
+    if (elect_one_sync()) umma_commit(&bar_acc_done);
+    __syncwarp();
   } else {
     // ---------------------------------------------------------------- compute: thread <-> query row
     const int wg = (warp - 2) >> 2;
@@ -206,61 +287,37 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     const float neg_lse2 = -LSE[grow] * 1.4426950408889634f;
     if (wg == 0) stats[grow] = make_float2(neg_lse2, Dv);
 
-    float rho = 0.f, msum = 0.f;
-    for (int n = wg; n < T; n += 2) {
-      mbar_wait(&bar_sdp_full[wg], (n >> 1) & 1, ab, kDqWaitSdP);
+    float rho[2] = {0.f, 0.f}, msum[2] = {0.f, 0.f};
+    const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
+    for (int n = wg, k = 0; n < T; n += NB, ++k) {
+      mbar_wait(&bar_sdp_full[wg], k & 1, ab, kDqWaitSdP);
       tc_fence_after();
-      const uint32_t tS = tmem_base + C::kColS + 64 * wg + lane_addr, tdP = tmem_base + C::kColDP + 64 * wg + lane_addr;
-      const bool diag = CAUSAL && (n >= T - 2);
-      const int kcol0 = n * C::kStepRows - qt * 128;      // key index of column 0 relative to this tile's first query
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t xs[32], xp[32];
-        tmem_ld32(tS + 32 * c, xs);
-        tmem_ld32(tdP + 32 * c, xp);
-        tmem_wait_ld();
-        uint32_t pr[16], pt[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, neg_lse2));
-          float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, neg_lse2));
-          if (diag) {
-            if (kcol0 + 32 * c + 2 * i > row) p0 = 0.f;
-            if (kcol0 + 32 * c + 2 * i + 1 > row) p1 = 0.f;
-          }
-          const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), Dv));
-          const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), Dv));
-          const uint32_t rp = pack_bf16x2(p0, p1), tp = pack_bf16x2(t0, t1);
-          msum += bf16_lo_to_f32(rp); msum += bf16_hi_to_f32(rp);
-          rho += bf16_lo_to_f32(tp); rho += bf16_hi_to_f32(tp);
-          pr[i] = rp; pt[i] = tp;
-        }
-        tmem_st16(tS + 16 * c, pr);      // r over the consumed S columns
-        tmem_st16(tdP + 16 * c, pt);     // t over the consumed dP columns
-      }
+      if (CAUSAL && n >= T - 2) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho, msum);
+      else                      dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho, msum);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bar_tr_ready[wg]);
     }
 
-    // ---- row statistics of both warpgroups, lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
-    if (wg == 1) { s_rho[row] = rho; s_m[row] = msum; }
-    named_bar_sync(1, 256);
+    // ---- row statistics of all warpgroups (fixed order), lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
+    float rho_t = rho[0] + rho[1], m_t = msum[0] + msum[1];
+    if (wg > 0) { s_rho[wg - 1][row] = rho_t; s_m[wg - 1][row] = m_t; }
+    named_bar_sync(1, 128 * NB);
     if (wg == 0) {
-      rho += s_rho[row]; msum += s_m[row];
-      s_lam[row] = (msum != 0.f) ? __fdiv_rn(rho, msum) : 0.f;
+#pragma unroll
+      for (int w = 0; w < NB - 1; ++w) { rho_t += s_rho[w][row]; m_t += s_m[w][row]; }
+      s_lam[row] = (m_t != 0.f) ? __fdiv_rn(rho_t, m_t) : 0.f;
     }
-    named_bar_sync(1, 256);
+    named_bar_sync(1, 128 * NB);
     const float lam = s_lam[row];
     const float lam_q = (flags & kFlagNoQCorrection) ? 0.f : lam;
     const float lam_k = (flags & kFlagNoKCorrection) ? 0.f : lam;
 
     mbar_wait(&bar_acc_done, 0, ab, kDqWaitAcc);
     tc_fence_after();
-    // each warpgroup finishes half of the d columns
-#pragma unroll
-    for (int cc = 0; cc < D / 64; ++cc) {
-      const int col = wg * (D / 2) + 32 * cc;
+    // the 32-column chunks of the epilogue are dealt round-robin to the warpgroups
+    for (int cc = wg; cc < D / 32; cc += NB) {
+      const int col = 32 * cc;
       uint32_t a[32], b[32];
       tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
       tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);
@@ -297,7 +354,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 // dK / dV side
 // ============================================================================================
 template <int D, bool CAUSAL>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(BwdCfg<D>::kThreads, 1)
 bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmV,    // box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmQ,    // box 64 x 64 rows
@@ -306,6 +363,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const float2 *__restrict__ stats, __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV,
                int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
+  constexpr int NB = C::kNB, LAG = C::kLag;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sK = smem;
@@ -313,7 +371,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   uint8_t *sStage = sV + C::kBigTileBytes;   // stage s: Q, dO, Z step tiles, then 64 x float2 {-LSE log2 e, D}
 
   __shared__ uint64_t bar_kv, bar_q_full[C::kDkvStages], bar_q_empty[C::kDkvStages];
-  __shared__ uint64_t bar_sdp_full[2], bar_tr_ready[2], bar_acc_done;
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_acc_done;
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -322,7 +380,6 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   __syncthreads();
   if (cta_skip != 0) return;
 
-  const int n_kt = N / 128;
   const int lin = blockIdx.x;
   const int kt = lin / BH;                                   // causal: key tile 0 has the most query steps -> first
   const int bh = lin % BH;
@@ -331,14 +388,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   const int krow0 = bh * N + kt * 128;
   const bool use_z = (flags & kFlagNoKCorrection) == 0;
   const uint32_t stage_tx = (use_z ? 3 : 2) * C::kStepTileBytes + 512;
-  (void)n_kt;
 
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
     mbar_init(&bar_kv, 1);
     for (int s = 0; s < C::kDkvStages; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
+    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
     mbar_init(&bar_acc_done, 1);
     fence_mbar_init();
   }
@@ -349,7 +405,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = tmem_base_smem;
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -378,105 +434,97 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       }
     }
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- tensor-core issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 keys] x [64 queries], contraction over d
-      constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 keys] x [d], contraction over 64 queries
-      const uint32_t aK = smem_u32(sK), aV = smem_u32(sV);
-      mbar_wait(&bar_kv, 0, ab, kDkvWaitKV);
-      for (int n = 0; n <= T; ++n) {
-        if (n < T) {
-          const int st = n % C::kDkvStages, b = n & 1;
-          mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);
-          tc_fence_after();
-          const uint32_t aQ = smem_u32(sStage + st * C::kDkvStageBytes), adO = aQ + C::kStepTileBytes;
-          const uint32_t tS = tmem_base + C::kColS + 64 * b, tdP = tmem_base + C::kColDP + 64 * b;
+    // ---------------------------------------------------------------- tensor-core issuer (warp-uniform loop, elected issue)
+    constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 keys] x [64 queries], contraction over d
+    constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 keys] x [d], contraction over 64 queries
+    const SmemDesc dscK = make_smem_desc(smem_u32(sK), 16, 1024), dscV = make_smem_desc(smem_u32(sV), 16, 1024);
+    const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);                       // K-major view of stage 0
+    const SmemDesc dscQ0mn = make_smem_desc(smem_u32(sStage), C::kStepSlabBytes, 1024);    // MN-major view of stage 0
+    mbar_wait(&bar_kv, 0, ab, kDkvWaitKV);
+    for (int n = 0; n < T + LAG; ++n) {
+      if (n < T) {
+        const int st = n % C::kDkvStages, b = n % NB;
+        if (lane == 0) trace_stamp(0, n, 0);
+        mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);
+        tc_fence_after();
+        if (lane == 0) trace_stamp(0, n, 1);
+        const SmemDesc dscQ = dscQ0.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes);
+        const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
+        if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tS, smem_desc_sw128(aK + oa, 16, 1024), smem_desc_sw128(aQ + ob, 16, 1024), idesc_s, k > 0);
+            umma_ss(tS, dscK.at(oa), dscQ.at(ob), idesc_s, k > 0);
           }
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tdP, smem_desc_sw128(aV + oa, 16, 1024), smem_desc_sw128(adO + ob, 16, 1024), idesc_s, k > 0);
+            umma_ss(tdP, dscV.at(oa), dscdO.at(ob), idesc_s, k > 0);
           }
           umma_commit(&bar_sdp_full[b]);
+          trace_stamp(0, n, 2);
         }
-        if (n >= 1) {
-          const int p = n - 1, st = p % C::kDkvStages, b = p & 1;
-          mbar_wait(&bar_tr_ready[b], (p >> 1) & 1, ab, kDkvWaitTR);
-          tc_fence_after();
-          const uint32_t aQ = smem_u32(sStage + st * C::kDkvStageBytes), adO = aQ + C::kStepTileBytes, aZ = adO + C::kStepTileBytes;
-          const uint32_t tR = tmem_base + C::kColS + 64 * b, tT = tmem_base + C::kColDP + 64 * b;
+        __syncwarp();
+      }
+      if (n >= LAG) {
+        const int p = n - LAG, st = p % C::kDkvStages, b = p % NB;
+        mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDkvWaitTR);
+        tc_fence_after();
+        if (lane == 0) trace_stamp(0, p, 3);
+        const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes),
+                       dscZ = dscdO.advanced(C::kStepTileBytes);
+        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;
+        const uint32_t acc = (p > 0) ? 1u : 0u;
+        if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
-            umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, smem_desc_sw128(adO + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
-                    (p > 0) || (k > 0));
+            umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
-            umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, smem_desc_sw128(aQ + k * 2048, C::kStepSlabBytes, 1024), idesc_a,
-                    (p > 0) || (k > 0));
+            umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
           if (use_z) {
 #pragma unroll
             for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
-              umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, smem_desc_sw128(aZ + k * 2048, C::kStepSlabBytes, 1024), idesc_a, 1);
+              umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscZ.at(k * 2048), idesc_a, 1u);
           }
           umma_commit(&bar_q_empty[st]);
+          trace_stamp(0, p, 4);
         }
+        __syncwarp();
       }
-      umma_commit(&bar_acc_done);
     }
+    if (elect_one_sync()) umma_commit(&bar_acc_done);
+    __syncwarp();
   } else {
     // ---------------------------------------------------------------- compute: thread <-> key row
     const int wg = (warp - 2) >> 2;
     const int row = 32 * (warp & 3) + lane;                  // key row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
+    const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
+    const bool tracer = (threadIdx.x & 127) == 64;
 
-    for (int n = wg; n < T; n += 2) {
+    for (int n = wg, k = 0; n < T; n += NB, ++k) {
       const int st = n % C::kDkvStages;
+      if (tracer) trace_stamp(1 + wg, n, 0);
       mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);      // row statistics of this step landed
-      mbar_wait(&bar_sdp_full[wg], (n >> 1) & 1, ab, kDkvWaitSdP);
+      mbar_wait(&bar_sdp_full[wg], k & 1, ab, kDkvWaitSdP);
       tc_fence_after();
+      if (tracer) trace_stamp(1 + wg, n, 1);
       const float4 *st4 = reinterpret_cast<const float4 *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
-      const uint32_t tS = tmem_base + C::kColS + 64 * wg + lane_addr, tdP = tmem_base + C::kColDP + 64 * wg + lane_addr;
-      const bool diag = CAUSAL && (n < 2);
-      const int qcol0 = n * C::kStepRows;                     // query index of column 0 relative to this tile's first key
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t xs[32], xp[32];
-        tmem_ld32(tS + 32 * c, xs);
-        tmem_ld32(tdP + 32 * c, xp);
-        tmem_wait_ld();
-        uint32_t pr[16], pt[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float4 sd = st4[16 * c + i];                  // {-lse2, D} of columns 32c+2i and 32c+2i+1
-          float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, sd.x));
-          float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, sd.z));
-          if (diag) {
-            if (row > qcol0 + 32 * c + 2 * i) p0 = 0.f;
-            if (row > qcol0 + 32 * c + 2 * i + 1) p1 = 0.f;
-          }
-          const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), sd.y));
-          const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), sd.w));
-          pr[i] = pack_bf16x2(p0, p1);
-          pt[i] = pack_bf16x2(t0, t1);
-        }
-        tmem_st16(tS + 16 * c, pr);
-        tmem_st16(tdP + 16 * c, pt);
-      }
+      if (CAUSAL && n < 2) dkv_step<true>(tS, tdP, st4, scale_log2, row - n * C::kStepRows);
+      else                 dkv_step<false>(tS, tdP, st4, scale_log2, 0);
+      if (tracer) trace_stamp(1 + wg, n, 5);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bar_tr_ready[wg]);
+      if (tracer) trace_stamp(1 + wg, n, 7);
     }
 
     mbar_wait(&bar_acc_done, 0, ab, kDkvWaitAcc);
     tc_fence_after();
     const size_t grow = static_cast<size_t>(krow0 + row);
-#pragma unroll
-    for (int cc = 0; cc < D / 64; ++cc) {
-      const int col = wg * (D / 2) + 32 * cc;
+    for (int cc = wg; cc < D / 32; cc += NB) {
+      const int col = 32 * cc;
       uint32_t a[32], b[32];
       tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
       tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);

@@ -72,7 +72,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = tmem_base_smem;
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);   // shuffle marks it warp-uniform
   const uint32_t tS = tmem_base, tO = tmem_base + 128;
 
   if (warp == 0) {
@@ -101,29 +101,40 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- tensor-core issuer
-    if (lane == 0) {
+    // The whole warp runs this loop so that every address stays provably warp-uniform (descriptor operands
+    // then live in uniform registers); one elected lane issues the MMAs and commits.
+    {
       constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);   // S = Q K^T, both operands K-major
       constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, 0, 1);     // O += P V, V is MN-major (d contiguous)
+      const SmemDesc dscQ = make_smem_desc(smem_u32(sQ), 16, 1024);
+      const SmemDesc dscK0 = make_smem_desc(smem_u32(sK), 16, 1024);                  // K-major view of K stage 0
+      const SmemDesc dscV0 = make_smem_desc(smem_u32(sV), C::kSlabBytes, 1024);       // MN-major view of V stage 0
       mbar_wait(&bar_q, 0, ab, kFwdWaitQ);
       for (int j = 0; j < n_kv; ++j) {
         const int st = j % C::kStages;
         mbar_wait(&bar_kv_full[st], (j / C::kStages) & 1, ab, kFwdWaitKV);
         tc_fence_after();
-        const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK + st * C::kTileBytes), aV = smem_u32(sV + st * C::kTileBytes);
+        const SmemDesc dscK = dscK0.advanced(st * C::kTileBytes), dscV = dscV0.advanced(st * C::kTileBytes);
+        if (elect_one_sync()) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = (k / 4) * C::kSlabBytes + (k % 4) * 32;
-          umma_ss(tS, smem_desc_sw128(aQ + off, 16, 1024), smem_desc_sw128(aK + off, 16, 1024), idesc_s, k > 0);
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k / 4) * C::kSlabBytes + (k % 4) * 32;
+            umma_ss(tS, dscQ.at(off), dscK.at(off), idesc_s, k > 0);
+          }
+          umma_commit(&bar_s_full);
         }
-        umma_commit(&bar_s_full);
+        __syncwarp();
         mbar_wait(&bar_p_ready, j & 1, ab, kFwdWaitP);
         tc_fence_after();
+        const uint32_t acc = (j > 0) ? 1u : 0u;
+        if (elect_one_sync()) {
 #pragma unroll
-        for (int k = 0; k < C::kBlockN / 16; ++k) {
-          umma_ts(tO, tS + 8 * k, smem_desc_sw128(aV + k * 2048, C::kSlabBytes, 1024), idesc_o, (j > 0) || (k > 0));
+          for (int k = 0; k < C::kBlockN / 16; ++k) umma_ts(tO, tS + 8 * k, dscV.at(k * 2048), idesc_o, k > 0 ? 1u : acc);
+          umma_commit(&bar_kv_empty[st]);
         }
-        umma_commit(&bar_kv_empty[st]);
+        __syncwarp();
       }
+      if (elect_one_sync())
       umma_commit(&bar_o_done);
     }
   } else {

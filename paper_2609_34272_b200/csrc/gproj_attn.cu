@@ -231,4 +231,14 @@ const char *gproj_status_string(int status) {
 
 int gproj_last_launch_count(void) { return tl_launch_count; }
 
+#ifdef GPROJ_TRACE
+// Debug builds only: copy the phase stamps of CTA 0 to the host (after a device synchronize).
+int gproj_debug_read_trace(long long *out, int count) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return GPROJ_ERR_CUDA;
+  const int n = gproj::kTraceRoles * gproj::kTraceSteps * gproj::kTraceSlots;
+  if (count < n) return GPROJ_ERR_SHAPE;
+  return cudaMemcpyFromSymbol(out, gproj::g_trace, n * sizeof(long long)) == cudaSuccess ? n : GPROJ_ERR_CUDA;
+}
+#endif
+
 }  // extern "C"

@@ -21,6 +21,18 @@ struct AbortState {
   volatile int *cta_abort;   // shared-memory flag of this CTA
 };
 
+// Optional phase stamps (compiled in only with -DGPROJ_TRACE): CTA 0 records clock64() at named points
+// of each role's loop into a device array that a debug entry point copies out.
+#ifdef GPROJ_TRACE
+constexpr int kTraceRoles = 4, kTraceSteps = 96, kTraceSlots = 8;
+__device__ long long g_trace[kTraceRoles * kTraceSteps * kTraceSlots];
+__device__ __forceinline__ void trace_stamp(int role, int step, int slot) {
+  if (blockIdx.x == 0 && step < kTraceSteps) g_trace[(role * kTraceSteps + step) * kTraceSlots + slot] = clock64();
+}
+#else
+__device__ __forceinline__ void trace_stamp(int, int, int) {}
+#endif
+
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
@@ -145,6 +157,22 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   d |= static_cast<uint64_t>(1) << 46;
   d |= static_cast<uint64_t>(2) << 61;
   return d;
+}
+
+// The same descriptor split into its two 32-bit words.  The issuing thread builds it once per operand
+// tile; moving the start address by a byte offset is then a single 32-bit add on the low word (shared
+// memory addresses stay below 2^18, so the 14-bit field cannot carry).  Keeping the per-instruction
+// arithmetic this short matters: one thread issues every MMA of the CTA.
+struct SmemDesc {
+  uint32_t lo, hi;
+  __device__ __forceinline__ uint64_t at(uint32_t byte_offset) const {
+    return (static_cast<uint64_t>(hi) << 32) | static_cast<uint64_t>(lo + (byte_offset >> 4));
+  }
+  __device__ __forceinline__ SmemDesc advanced(uint32_t byte_offset) const { return SmemDesc{lo + (byte_offset >> 4), hi}; }
+};
+__device__ __forceinline__ SmemDesc make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  const uint64_t d = smem_desc_sw128(saddr, lbo_bytes, sbo_bytes);
+  return SmemDesc{static_cast<uint32_t>(d), static_cast<uint32_t>(d >> 32)};
 }
 
 // Instruction descriptor for kind::f16 with BF16 A/B and FP32 accumulation.

@@ -21,8 +21,11 @@
 // Pipeline.  TMEM holds kNB score buffers (S and dP of one 64-wide step each) next to the two FP32
 // accumulators: 3 buffers at d = 64, 2 at d = 128 (512 columns either way).  Compute warpgroup w owns
 // buffer w and the steps n = w (mod kNB); it overwrites the consumed S / dP columns with the packed BF16
-// operands r / t.  One warp issues every MMA: scores of step n first, then the second-stage products of
-// step n - (kNB - 1), so up to kNB steps are in flight and the tensor core works while the ALUs do.
+// operands r / t.  The tensor-core queue is only one or two instructions deep, so an issuing warp is stalled
+// for as long as its MMAs execute and anything else it does (barrier polls, commits) would idle the pipe.
+// Two warps therefore issue: warp 1 the score products of every step, warp 2 the second-stage products; each
+// one's bookkeeping overlaps the other's MMAs.  Reuse of a score buffer is ordered by an explicit barrier
+// (second-stage MMAs of step n committed -> scores of step n + kNB may be issued).
 #pragma once
 #include "sm100_primitives.cuh"
 
@@ -40,8 +43,7 @@ struct BwdCfg {
   static constexpr int kStepSlabBytes = kStepRows * 128;
   static constexpr int kStepTileBytes = kSlabs * kStepSlabBytes;
   static constexpr int kNB = (D == 64) ? 3 : 2;                   // score buffers = compute warpgroups
-  static constexpr int kLag = kNB - 1;                            // second-stage MMAs trail the scores by this many steps
-  static constexpr int kThreads = 64 + 128 * kNB;                 // producer warp, MMA warp, kNB compute warpgroups
+  static constexpr int kThreads = 128 + 128 * kNB;                // producer, 2 MMA warps, 1 spare; kNB compute warpgroups
   // TMEM columns: buffer b holds S at 128 b and dP at 128 b + 64; accumulators follow
   static constexpr int kTmemCols = 512;
   static constexpr uint32_t kColAcc0 = 128 * kNB, kColAcc1 = 128 * kNB + D;
@@ -52,76 +54,98 @@ struct BwdCfg {
   static constexpr int kDqSmemBytes = 2 * kBigTileBytes + kDqStages * kDqStageBytes + 1024;
   // dK/dV-side kernel: K, V resident; ring of (Q, dO, Z, stats) step tiles
   static constexpr int kDkvStages = (D == 64) ? 5 : 3;
-  static constexpr int kDkvStageBytes = 3 * kStepTileBytes + 1024;   // + 64 x float2 row statistics (512 B used)
+  static constexpr int kDkvStageBytes = 3 * kStepTileBytes + 1024;   // + 2 x 64 floats of row statistics (512 B used)
   static constexpr int kDkvSmemBytes = 2 * kBigTileBytes + kDkvStages * kDkvStageBytes + 1024;
   static_assert(kDqStages >= kNB + 1 && kDkvStages >= kNB + 1, "a stage stays busy until its second-stage MMAs finish");
 };
 
 enum BwdWaitCode {
-  kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26,
-  kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36
+  kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26, kDqWaitBuf = 0x27,
+  kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36, kDkvWaitBuf = 0x37
 };
 
+// Arithmetic of one pair of adjacent score columns, shared by both kernels (Algorithm 1 lines 5-8):
+//   p = exp2(x * (alpha log2 e) - LSE log2 e),  r = BF16(p),  t = BF16(fl32[p * fl32(dP - D)]).
+// x2 / dp2 are the raw TMEM words of the two columns; nl2 = {-LSE log2 e} and nd2 = {-D} per column.
+// keep0 / keep1 zero a probability beyond the causal diagonal.
+template <bool MASKED>
+__device__ __forceinline__ void score_pair(uint32_t x0, uint32_t x1, uint32_t dp0, uint32_t dp1, uint64_t scale2, uint64_t nl2,
+                                           uint64_t nd2, bool keep0, bool keep1, uint32_t &r_packed, uint32_t &t_packed) {
+  float a0, a1;
+  f32x2_split(fma2(f32x2_bits(x0, x1), scale2, nl2), a0, a1);
+  float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
+  if (MASKED) {
+    if (!keep0) p0 = 0.f;
+    if (!keep1) p1 = 0.f;
+  }
+  float t0, t1;
+  f32x2_split(mul2(f32x2(p0, p1), add2(f32x2_bits(dp0, dp1), nd2)), t0, t1);
+  r_packed = pack_bf16x2(p0, p1);
+  t_packed = pack_bf16x2(t0, t1);
+}
+
 // One 64-column step of the dQ side for one query row.  `lim` = (row index) - (key index of column 0):
-// with MASKED, column c is beyond the causal diagonal when c > lim.
+// with MASKED, column c is beyond the causal diagonal when c > lim.  TMEM is read in 16-column chunks and the
+// next chunk's load is in flight while the current one is in the ALUs; the packed r / t overwrite columns
+// whose scores were consumed at least one chunk earlier.
 template <bool MASKED>
 __device__ __forceinline__ void dq_step(uint32_t tS, uint32_t tdP, float scale_log2, float neg_lse2, float Dv, int lim,
-                                        float (&rho)[2], float (&msum)[2]) {
+                                        uint64_t &rho2, uint64_t &msum2) {
+  const uint64_t scale2 = f32x2(scale_log2, scale_log2), nl2 = f32x2(neg_lse2, neg_lse2), nd2 = f32x2(-Dv, -Dv);
+  uint32_t xs[2][16], xp[2][16];
+  tmem_ld16(tS, xs[0]);
+  tmem_ld16(tdP, xp[0]);
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    uint32_t xs[32], xp[32];
-    tmem_ld32(tS + 32 * c, xs);
-    tmem_ld32(tdP + 32 * c, xp);
+  for (int c = 0; c < 4; ++c) {
     tmem_wait_ld();
-    uint32_t pr[16], pt[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, neg_lse2));
-      float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, neg_lse2));
-      if (MASKED) {
-        if (32 * c + 2 * i > lim) p0 = 0.f;
-        if (32 * c + 2 * i + 1 > lim) p1 = 0.f;
-      }
-      const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), Dv));
-      const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), Dv));
-      const uint32_t rp = pack_bf16x2(p0, p1), tp = pack_bf16x2(t0, t1);
-      // row masses of the operands as rounded (two chains each, to keep the adds off one dependency chain)
-      msum[0] += bf16_lo_to_f32(rp); msum[1] += bf16_hi_to_f32(rp);
-      rho[0] += bf16_lo_to_f32(tp); rho[1] += bf16_hi_to_f32(tp);
-      pr[i] = rp; pt[i] = tp;
+    if (c < 3) {
+      tmem_ld16(tS + 16 * (c + 1), xs[(c + 1) & 1]);
+      tmem_ld16(tdP + 16 * (c + 1), xp[(c + 1) & 1]);
     }
-    tmem_st16(tS + 16 * c, pr);      // r over the consumed S columns
-    tmem_st16(tdP + 16 * c, pt);     // t over the consumed dP columns
+    uint32_t pr[8], pt[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int col = 16 * c + 2 * i;
+      score_pair<MASKED>(xs[c & 1][2 * i], xs[c & 1][2 * i + 1], xp[c & 1][2 * i], xp[c & 1][2 * i + 1], scale2, nl2, nd2,
+                         col <= lim, col + 1 <= lim, pr[i], pt[i]);
+      // row masses of the operands AS ROUNDED (Eq. "gproj-row-mass"): re-expand the BF16 pairs and add in FP32
+      msum2 = add2(msum2, f32x2_bits(pr[i] << 16, pr[i] & 0xffff0000u));
+      rho2 = add2(rho2, f32x2_bits(pt[i] << 16, pt[i] & 0xffff0000u));
+    }
+    tmem_st8(tS + 8 * c, pr);      // r over consumed S columns
+    tmem_st8(tdP + 8 * c, pt);     // t over consumed dP columns
   }
 }
 
 // One 64-column step of the dK/dV side for one key row.  `lim` = (key row) - (query index of column 0):
-// with MASKED, column c is a query before this key when c < lim.
+// with MASKED, column c is a query before this key when c < lim.  nl / nd: per-column -LSE log2 e and -D.
 template <bool MASKED>
-__device__ __forceinline__ void dkv_step(uint32_t tS, uint32_t tdP, const float4 *st4, float scale_log2, int lim) {
+__device__ __forceinline__ void dkv_step(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim) {
+  const uint64_t scale2 = f32x2(scale_log2, scale_log2);
+  uint32_t xs[2][16], xp[2][16];
+  tmem_ld16(tS, xs[0]);
+  tmem_ld16(tdP, xp[0]);
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    uint32_t xs[32], xp[32];
-    tmem_ld32(tS + 32 * c, xs);
-    tmem_ld32(tdP + 32 * c, xp);
+  for (int c = 0; c < 4; ++c) {
     tmem_wait_ld();
-    uint32_t pr[16], pt[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float4 sd = st4[16 * c + i];                  // {-LSE log2 e, D} of columns 32c+2i and 32c+2i+1
-      float p0 = fast_exp2(fmaf(__uint_as_float(xs[2 * i]), scale_log2, sd.x));
-      float p1 = fast_exp2(fmaf(__uint_as_float(xs[2 * i + 1]), scale_log2, sd.z));
-      if (MASKED) {
-        if (32 * c + 2 * i < lim) p0 = 0.f;
-        if (32 * c + 2 * i + 1 < lim) p1 = 0.f;
-      }
-      const float t0 = __fmul_rn(p0, __fsub_rn(__uint_as_float(xp[2 * i]), sd.y));
-      const float t1 = __fmul_rn(p1, __fsub_rn(__uint_as_float(xp[2 * i + 1]), sd.w));
-      pr[i] = pack_bf16x2(p0, p1);
-      pt[i] = pack_bf16x2(t0, t1);
+    if (c < 3) {
+      tmem_ld16(tS + 16 * (c + 1), xs[(c + 1) & 1]);
+      tmem_ld16(tdP + 16 * (c + 1), xp[(c + 1) & 1]);
     }
-    tmem_st16(tS + 16 * c, pr);
-    tmem_st16(tdP + 16 * c, pt);
+    uint32_t pr[8], pt[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      // statistics of four columns per 16-byte shared-memory read (same address for every lane: broadcast)
+      const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);
+      const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
+      const int col = 16 * c + 4 * i;
+      score_pair<MASKED>(xs[c & 1][4 * i], xs[c & 1][4 * i + 1], xp[c & 1][4 * i], xp[c & 1][4 * i + 1], scale2, l4.x, d4.x,
+                         col >= lim, col + 1 >= lim, pr[2 * i], pt[2 * i]);
+      score_pair<MASKED>(xs[c & 1][4 * i + 2], xs[c & 1][4 * i + 3], xp[c & 1][4 * i + 2], xp[c & 1][4 * i + 3], scale2, l4.y, d4.y,
+                         col + 2 >= lim, col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
+    }
+    tmem_st8(tS + 8 * c, pr);
+    tmem_st8(tdP + 8 * c, pt);
   }
 }
 
@@ -136,10 +160,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmV,    // box 64 x 64 rows
               const __nv_bfloat16 *__restrict__ Qg, const __nv_bfloat16 *__restrict__ Og,
               const __nv_bfloat16 *__restrict__ dOg, const float *__restrict__ LSE,
-              __nv_bfloat16 *__restrict__ dQ, __nv_bfloat16 *__restrict__ Zneg, float2 *__restrict__ stats,
+              __nv_bfloat16 *__restrict__ dQ, __nv_bfloat16 *__restrict__ Zneg, float *__restrict__ stats,
               int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
-  constexpr int NB = C::kNB, LAG = C::kLag;
+  constexpr int NB = C::kNB;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;
@@ -147,7 +171,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   uint8_t *sKV = sdO + C::kBigTileBytes;    // stage s: K step tile, then V step tile
 
   __shared__ uint64_t bar_q, bar_kv_full[C::kDqStages], bar_kv_empty[C::kDqStages];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_acc_done;
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done;
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
   __shared__ float s_rho[NB - 1][128], s_m[NB - 1][128], s_lam[128];
@@ -169,7 +193,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     cta_abort = 0;
     mbar_init(&bar_q, 1);
     for (int s = 0; s < C::kDqStages; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
-    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
+    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
     fence_mbar_init();
   }
@@ -209,61 +233,64 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
     }
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- tensor-core issuer
+    // ---------------------------------------------------------------- tensor-core issuer 1: scores
     // The whole warp runs this loop so that every address stays provably warp-uniform (descriptor operands
     // then live in uniform registers); one elected lane issues the MMAs and commits.
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 queries] x [64 keys], contraction over d
-    constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 queries] x [d], contraction over 64 keys
     const SmemDesc dscQ = make_smem_desc(smem_u32(sQ), 16, 1024), dscdO = make_smem_desc(smem_u32(sdO), 16, 1024);
     const SmemDesc dscK0 = make_smem_desc(smem_u32(sKV), 16, 1024);                          // K-major view of stage 0
-    const SmemDesc dscK0mn = make_smem_desc(smem_u32(sKV), C::kStepSlabBytes, 1024);       // MN-major view of stage 0
     mbar_wait(&bar_q, 0, ab, kDqWaitQ);
-    for (int n = 0; n < T + LAG; ++n) {
-      if (n < T) {
-        const int st = n % C::kDqStages, b = n % NB;
-        mbar_wait(&bar_kv_full[st], (n / C::kDqStages) & 1, ab, kDqWaitKV);
-        tc_fence_after();
-        const SmemDesc dscK = dscK0.advanced(st * C::kDqStageBytes), dscV = dscK.advanced(C::kStepTileBytes);
-        const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
-        if (elect_one_sync()) {
+    for (int n = 0; n < T; ++n) {
+      const int st = n % C::kDqStages, b = n % NB;
+      mbar_wait(&bar_kv_full[st], (n / C::kDqStages) & 1, ab, kDqWaitKV);
+      if (n >= NB) mbar_wait(&bar_buf_free[b], ((n / NB) - 1) & 1, ab, kDqWaitBuf);   // r, t of step n - NB consumed
+      tc_fence_after();
+      const SmemDesc dscK = dscK0.advanced(st * C::kDqStageBytes), dscV = dscK.advanced(C::kStepTileBytes);
+      const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
+      if (elect_one_sync()) {
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tS, dscQ.at(oa), dscK.at(ob), idesc_s, k > 0);
-          }
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tdP, dscdO.at(oa), dscV.at(ob), idesc_s, k > 0);
-          }
-          umma_commit(&bar_sdp_full[b]);
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+          umma_ss(tS, dscQ.at(oa), dscK.at(ob), idesc_s, k > 0);
         }
-        __syncwarp();
-      }
-      if (n >= LAG) {
-        const int p = n - LAG, st = p % C::kDqStages, b = p % NB;
-        mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDqWaitTR);
-        tc_fence_after();
-        const SmemDesc dscK = dscK0mn.advanced(st * C::kDqStageBytes);
-        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;     // packed BF16 r / t over the S / dP columns
-        const uint32_t acc = (p > 0) ? 1u : 0u;
-        if (elect_one_sync()) {
 #pragma unroll
-          for (int k = 0; k < C::kStepRows / 16; ++k)
-            umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-#pragma unroll
-          for (int k = 0; k < C::kStepRows / 16; ++k)
-            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-          umma_commit(&bar_kv_empty[st]);
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+          umma_ss(tdP, dscdO.at(oa), dscV.at(ob), idesc_s, k > 0);
         }
-        __syncwarp();
+        umma_commit(&bar_sdp_full[b]);
       }
+      __syncwarp();
     }
-    if (elect_one_sync()) umma_commit(&bar_acc_done);
-    __syncwarp();
+  } else if (warp == 2) {
+    // ---------------------------------------------------------------- tensor-core issuer 2: A += t K, B += r K
+    constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 queries] x [d], contraction over 64 keys
+    const SmemDesc dscK0mn = make_smem_desc(smem_u32(sKV), C::kStepSlabBytes, 1024);       // MN-major view of stage 0
+    for (int p = 0; p < T; ++p) {
+      const int st = p % C::kDqStages, b = p % NB;
+      mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDqWaitTR);
+      tc_fence_after();
+      const SmemDesc dscK = dscK0mn.advanced(st * C::kDqStageBytes);
+      const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;     // packed BF16 r / t over the S / dP columns
+      const uint32_t acc = (p > 0) ? 1u : 0u;
+      if (elect_one_sync()) {
+#pragma unroll
+        for (int k = 0; k < C::kStepRows / 16; ++k)
+          umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+#pragma unroll
+        for (int k = 0; k < C::kStepRows / 16; ++k)
+          umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+        umma_commit(&bar_buf_free[b]);
+        umma_commit(&bar_kv_empty[st]);
+        if (p == T - 1) umma_commit(&bar_acc_done);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 3) {
+    // spare warp: keeps the compute warpgroups aligned to TMEM lane quadrants
   } else {
     // ---------------------------------------------------------------- compute: thread <-> query row
-    const int wg = (warp - 2) >> 2;
+    const int wg = (warp - 4) >> 2;
     const int row = 32 * (warp & 3) + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
     const size_t grow = static_cast<size_t>(row0 + row);
@@ -285,22 +312,29 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
     }
     const float neg_lse2 = -LSE[grow] * 1.4426950408889634f;
-    if (wg == 0) stats[grow] = make_float2(neg_lse2, Dv);
+    if (wg == 0) {   // per 64-row block: 64 x {-LSE log2 e}, then 64 x {-D}
+      float *blk = stats + (grow >> 6) * 128 + (grow & 63);
+      blk[0] = neg_lse2;
+      blk[64] = -Dv;
+    }
 
-    float rho[2] = {0.f, 0.f}, msum[2] = {0.f, 0.f};
+    uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);
     const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
     for (int n = wg, k = 0; n < T; n += NB, ++k) {
       mbar_wait(&bar_sdp_full[wg], k & 1, ab, kDqWaitSdP);
       tc_fence_after();
-      if (CAUSAL && n >= T - 2) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho, msum);
-      else                      dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho, msum);
+      if (CAUSAL && n >= T - 2) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho2, msum2);
+      else                      dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bar_tr_ready[wg]);
     }
 
     // ---- row statistics of all warpgroups (fixed order), lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
-    float rho_t = rho[0] + rho[1], m_t = msum[0] + msum[1];
+    float rho_lo, rho_hi, m_lo, m_hi;
+    f32x2_split(rho2, rho_lo, rho_hi);
+    f32x2_split(msum2, m_lo, m_hi);
+    float rho_t = rho_lo + rho_hi, m_t = m_lo + m_hi;
     if (wg > 0) { s_rho[wg - 1][row] = rho_t; s_m[wg - 1][row] = m_t; }
     named_bar_sync(1, 128 * NB);
     if (wg == 0) {
@@ -360,18 +394,18 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmQ,    // box 64 x 64 rows
                const __grid_constant__ CUtensorMap tmdO,   // box 64 x 64 rows
                const __grid_constant__ CUtensorMap tmZ,    // box 64 x 64 rows
-               const float2 *__restrict__ stats, __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV,
+               const float *__restrict__ stats, __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV,
                int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
-  constexpr int NB = C::kNB, LAG = C::kLag;
+  constexpr int NB = C::kNB;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sK = smem;
   uint8_t *sV = sK + C::kBigTileBytes;
-  uint8_t *sStage = sV + C::kBigTileBytes;   // stage s: Q, dO, Z step tiles, then 64 x float2 {-LSE log2 e, D}
+  uint8_t *sStage = sV + C::kBigTileBytes;   // stage s: Q, dO, Z step tiles, then 64 x {-LSE log2 e} and 64 x {-D}
 
   __shared__ uint64_t bar_kv, bar_q_full[C::kDkvStages], bar_q_empty[C::kDkvStages];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_acc_done;
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done;
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -394,7 +428,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     cta_abort = 0;
     mbar_init(&bar_kv, 1);
     for (int s = 0; s < C::kDkvStages; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
-    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); }
+    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
     fence_mbar_init();
   }
@@ -426,7 +460,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
           tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow);
           if (use_z) tma_load_2d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow);
         }
-        bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + qrow, 512, &bar_q_full[st]);
+        bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + 2 * static_cast<size_t>(qrow), 512, &bar_q_full[st]);
       }
       if (cta_abort) {
         for (int n = (T > C::kDkvStages ? T - C::kDkvStages : 0); n < T; ++n)
@@ -434,70 +468,74 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       }
     }
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- tensor-core issuer (warp-uniform loop, elected issue)
+    // ---------------------------------------------------------------- tensor-core issuer 1: scores (warp-uniform loop, elected issue)
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 keys] x [64 queries], contraction over d
-    constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 keys] x [d], contraction over 64 queries
     const SmemDesc dscK = make_smem_desc(smem_u32(sK), 16, 1024), dscV = make_smem_desc(smem_u32(sV), 16, 1024);
     const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);                       // K-major view of stage 0
-    const SmemDesc dscQ0mn = make_smem_desc(smem_u32(sStage), C::kStepSlabBytes, 1024);    // MN-major view of stage 0
     mbar_wait(&bar_kv, 0, ab, kDkvWaitKV);
-    for (int n = 0; n < T + LAG; ++n) {
-      if (n < T) {
-        const int st = n % C::kDkvStages, b = n % NB;
-        if (lane == 0) trace_stamp(0, n, 0);
-        mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);
-        tc_fence_after();
-        if (lane == 0) trace_stamp(0, n, 1);
-        const SmemDesc dscQ = dscQ0.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes);
-        const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
-        if (elect_one_sync()) {
+    for (int n = 0; n < T; ++n) {
+      const int st = n % C::kDkvStages, b = n % NB;
+      if (lane == 0) trace_stamp(0, n, 0);
+      mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);
+      if (n >= NB) mbar_wait(&bar_buf_free[b], ((n / NB) - 1) & 1, ab, kDkvWaitBuf);   // r, t of step n - NB consumed
+      tc_fence_after();
+      if (lane == 0) trace_stamp(0, n, 1);
+      const SmemDesc dscQ = dscQ0.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes);
+      const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
+      if (elect_one_sync()) {
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tS, dscK.at(oa), dscQ.at(ob), idesc_s, k > 0);
-          }
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-            umma_ss(tdP, dscV.at(oa), dscdO.at(ob), idesc_s, k > 0);
-          }
-          umma_commit(&bar_sdp_full[b]);
-          trace_stamp(0, n, 2);
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+          umma_ss(tS, dscK.at(oa), dscQ.at(ob), idesc_s, k > 0);
         }
-        __syncwarp();
-      }
-      if (n >= LAG) {
-        const int p = n - LAG, st = p % C::kDkvStages, b = p % NB;
-        mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDkvWaitTR);
-        tc_fence_after();
-        if (lane == 0) trace_stamp(0, p, 3);
-        const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes),
-                       dscZ = dscdO.advanced(C::kStepTileBytes);
-        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;
-        const uint32_t acc = (p > 0) ? 1u : 0u;
-        if (elect_one_sync()) {
 #pragma unroll
-          for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
-            umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-#pragma unroll
-          for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
-            umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-          if (use_z) {
-#pragma unroll
-            for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
-              umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscZ.at(k * 2048), idesc_a, 1u);
-          }
-          umma_commit(&bar_q_empty[st]);
-          trace_stamp(0, p, 4);
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+          umma_ss(tdP, dscV.at(oa), dscdO.at(ob), idesc_s, k > 0);
         }
-        __syncwarp();
+        umma_commit(&bar_sdp_full[b]);
+        trace_stamp(0, n, 2);
       }
+      __syncwarp();
     }
-    if (elect_one_sync()) umma_commit(&bar_acc_done);
-    __syncwarp();
+  } else if (warp == 2) {
+    // ---------------------------------------------------------------- tensor-core issuer 2: dV += r^T dO, dK += t^T Q + r^T Z
+    constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 keys] x [d], contraction over 64 queries
+    const SmemDesc dscQ0mn = make_smem_desc(smem_u32(sStage), C::kStepSlabBytes, 1024);    // MN-major view of stage 0
+    for (int p = 0; p < T; ++p) {
+      const int st = p % C::kDkvStages, b = p % NB;
+      if (lane == 0) trace_stamp(3, p, 0);
+      mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDkvWaitTR);
+      tc_fence_after();
+      if (lane == 0) trace_stamp(3, p, 1);
+      const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes),
+                     dscZ = dscdO.advanced(C::kStepTileBytes);
+      const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;
+      const uint32_t acc = (p > 0) ? 1u : 0u;
+      if (elect_one_sync()) {
+#pragma unroll
+        for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
+          umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+#pragma unroll
+        for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
+          umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+        if (use_z) {
+#pragma unroll
+          for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
+            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscZ.at(k * 2048), idesc_a, 1u);
+        }
+        umma_commit(&bar_buf_free[b]);
+        umma_commit(&bar_q_empty[st]);
+        if (p == T - 1) umma_commit(&bar_acc_done);
+        trace_stamp(3, p, 2);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 3) {
+    // spare warp: keeps the compute warpgroups aligned to TMEM lane quadrants
   } else {
     // ---------------------------------------------------------------- compute: thread <-> key row
-    const int wg = (warp - 2) >> 2;
+    const int wg = (warp - 4) >> 2;
     const int row = 32 * (warp & 3) + lane;                  // key row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
     const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
@@ -510,9 +548,9 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       mbar_wait(&bar_sdp_full[wg], k & 1, ab, kDkvWaitSdP);
       tc_fence_after();
       if (tracer) trace_stamp(1 + wg, n, 1);
-      const float4 *st4 = reinterpret_cast<const float4 *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
-      if (CAUSAL && n < 2) dkv_step<true>(tS, tdP, st4, scale_log2, row - n * C::kStepRows);
-      else                 dkv_step<false>(tS, tdP, st4, scale_log2, 0);
+      const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
+      if (CAUSAL && n < 2) dkv_step<true>(tS, tdP, nl, nl + 64, scale_log2, row - n * C::kStepRows);
+      else                 dkv_step<false>(tS, tdP, nl, nl + 64, scale_log2, 0);
       if (tracer) trace_stamp(1 + wg, n, 5);
       tmem_wait_st();
       tc_fence_before();

@@ -165,7 +165,7 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
 
   const int BH = B * H;
   const uint64_t rows = static_cast<uint64_t>(BH) * N;
-  float2 *stats = static_cast<float2 *>(workspace);
+  float *stats = static_cast<float *>(workspace);   // per 64-row block: 64 x {-LSE log2 e}, 64 x {-D}
   __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + align256(rows * sizeof(float2)));
 
   CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64;

@@ -26,6 +26,8 @@ if ROOT not in sys.path:
 
 METRIC = "fused attn bwd TFLOP/s & % BF16 tensor peak; dQ/dK/dV rel-L2 vs FP64"
 UNIT = "TFLOP/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised under profiles/
+NCU_DRAM_BYTES_PER_LAUNCH = {("bwd_dkv_kernel", 2): 42.507e6 + 0.791e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -261,7 +263,8 @@ def main():
         "wall_ms_per_step_incl_l2_flush": 1e3 * wall / steps,
         "kernels_ms": {"bwd_dq_kernel": dq_ms, "bwd_dkv_kernel": dkv_ms},
         "roofline": {"bound": "tensor", "kernel": "bwd_dkv_kernel", "achieved": dkv_achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": dkv_achieved / peak, "traffic": None, "peak_source": peak_kind + " (burst bf16 GEMM)",
+                     "frac": dkv_achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(("bwd_dkv_kernel", args.workload)),
+                     "peak_source": peak_kind + " (burst bf16 GEMM)",
                      "algorithmic_flops_per_launch": fl["dkv_kernel"]},
         "e2e": {"value": world * fl["bwd7"] / (e2e_ms / 1e3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 4 * tensor_bytes, "d2h_bytes_per_step": 3 * tensor_bytes,

@@ -85,6 +85,29 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
                    void *workspace, size_t workspace_bytes, unsigned flags, void *stream);
 
 /*
+ * Backward for callers that must not allocate device memory (the paper has no counterpart: this is a
+ * convenience of this library).  Some hosts of this code cannot call cudaMalloc at the point where they
+ * need a gradient: a plugin running inside another framework's memory pool, a real-time or safety-audited
+ * process whose memory is fixed at start-up, or a callback in which the CUDA allocator may not be entered.
+ * This entry point takes no workspace: the scratch of gproj_attn_bwd lives in a fixed device array of
+ * GPROJ_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the library holds
+ * that much memory until the process exits.
+ *   - Same inputs, outputs, flags and arithmetic as gproj_attn_bwd; results are bitwise the same.
+ *   - Shapes whose gproj_attn_bwd_workspace_bytes() exceeds GPROJ_STATIC_SCRATCH_BYTES are rejected with
+ *     GPROJ_ERR_WORKSPACE (workloads up to B*H*N*d = 8 Mi elements at d = 64 fit); nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device current); make
+ *     that first call before any stream capture begins.  No call allocates or frees anything.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left there.  Nothing
+ *     in it has to start at zero (the first kernel writes every word the second one reads), but two calls
+ *     that overlap on the GPU (different streams, no dependency) race on it: serialise them.
+ */
+#define GPROJ_STATIC_SCRATCH_BYTES (16u << 20)
+int gproj_attn_bwd_static_scratch(const void *Q, const void *K, const void *V, const void *O, const float *LSE,
+                                  const void *dO, void *dQ, void *dK, void *dV,
+                                  int B, int H, int N, int d, float softmax_scale, int causal,
+                                  unsigned flags, void *stream);
+
+/*
  * Synchronises `stream`, then returns GPROJ_OK, GPROJ_ERR_TIMEOUT if any kernel launched by this
  * library on the current device since the last call recorded an abandoned wait, or GPROJ_ERR_CUDA.
  * If `detail` is non-NULL it receives the raw device code (0 when fine) and the code is cleared.

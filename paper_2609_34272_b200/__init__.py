@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     FLAG_ONLY_DQ_PASS,
     GprojError,
     gproj_attn_bwd,
+    gproj_attn_bwd_static_scratch,
     gproj_attn_bwd_workspace_bytes,
     gproj_attn_fwd,
     gproj_last_device_status,

@@ -18,7 +18,10 @@ FLAG_NO_K_CORRECTION = 2
 FLAG_ONLY_DQ_PASS = 4
 FLAG_ONLY_DKV_PASS = 8
 
-EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_last_device_status",
+STATIC_SCRATCH_BYTES = 16 << 20
+
+EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_bwd_static_scratch",
+           "gproj_last_device_status",
            "gproj_status_string", "gproj_last_launch_count")
 
 _lib = None
@@ -45,6 +48,8 @@ def load():
         lib.gproj_attn_bwd_workspace_bytes.argtypes = [i, i, i, i]
         lib.gproj_attn_bwd.restype = i
         lib.gproj_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, sz, u, vp]
+        lib.gproj_attn_bwd_static_scratch.restype = i
+        lib.gproj_attn_bwd_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, u, vp]
         lib.gproj_last_device_status.restype = i
         lib.gproj_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
         lib.gproj_status_string.restype = ctypes.c_char_p
@@ -113,6 +118,32 @@ def gproj_attn_bwd(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, workspac
                                    int(flags), _stream(Q.device))
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_bwd")
+    return dQ, dK, dV
+
+
+def gproj_attn_bwd_static_scratch(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, dQ=None, dK=None, dV=None):
+    """Backward that uses the library's built-in device scratch instead of a workspace tensor.
+
+    For callers that may not allocate device memory when the gradient is needed.  Shapes needing more than
+    ``STATIC_SCRATCH_BYTES`` of scratch raise ``GprojError`` (status -4).  Calls on one device share the scratch:
+    do not let two of them overlap on the GPU.  The output tensors are the caller's (pass dQ, dK, dV to avoid
+    even those allocations).
+    """
+    _check_bf16("Q", Q)
+    B, H, N, d = Q.shape
+    for name, t in (("K", K), ("V", V), ("O", O), ("dO", dO)):
+        _check_bf16(name, t, Q.shape)
+    if not (LSE.is_cuda and LSE.dtype == torch.float32 and LSE.is_contiguous() and tuple(LSE.shape) == (B, H, N)):
+        raise TypeError("LSE must be a contiguous CUDA float32 tensor [B, H, N]")
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(Q) if dK is None else dK
+    dV = torch.empty_like(Q) if dV is None else dV
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_bwd_static_scratch(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
+                                                  dO.data_ptr(), dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, N, d,
+                                                  float(softmax_scale), int(bool(causal)), int(flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_bwd_static_scratch")
     return dQ, dK, dV
 
 

@@ -199,6 +199,35 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
   return GPROJ_OK;
 }
 
+// ---- backward without a caller-supplied workspace -------------------------------------------------
+// The scratch is a file-scope device array.  In host code the array's name is only a handle: the
+// address a kernel or a TMA descriptor can use must be looked up per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[GPROJ_STATIC_SCRATCH_BYTES];
+
+int gproj_attn_bwd_static_scratch(const void *Q, const void *K, const void *V, const void *O, const float *LSE,
+                                  const void *dO, void *dQ, void *dK, void *dV, int B, int H, int N, int d,
+                                  float softmax_scale, int causal, unsigned flags, void *stream) {
+  static std::mutex scratch_mutex;
+  static void *scratch_addr[kMaxDevices] = {};
+  const size_t need = gproj_attn_bwd_workspace_bytes(B, H, N, d);
+  if (need == 0) return GPROJ_ERR_SHAPE;
+  if (need > GPROJ_STATIC_SCRATCH_BYTES) return GPROJ_ERR_WORKSPACE;   // beyond the built-in scratch
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GPROJ_ERR_CUDA;
+  void *scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(scratch_mutex);
+    if (!scratch_addr[dev]) {   // once per device, with that device current
+      void *p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+      scratch_addr[dev] = p;
+    }
+    scratch = scratch_addr[dev];
+  }
+  return gproj_attn_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, N, d, softmax_scale, causal, scratch,
+                        GPROJ_STATIC_SCRATCH_BYTES, flags, stream);
+}
+
 int gproj_last_device_status(void *stream, int *detail) {
   if (detail) *detail = 0;
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return GPROJ_ERR_CUDA;

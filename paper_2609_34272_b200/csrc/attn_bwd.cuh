@@ -123,26 +123,35 @@ template <bool MASKED>
 __device__ __forceinline__ void dkv_step(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2);
   uint32_t xs[2][16], xp[2][16];
+  ulonglong2 l4[2][4], d4[2][4];     // statistics of 16 columns, fetched one chunk ahead (shared-memory latency is long
+                                     // while the tensor core streams its operands from the same memory)
   tmem_ld16(tS, xs[0]);
   tmem_ld16(tdP, xp[0]);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    l4[0][i] = *reinterpret_cast<const ulonglong2 *>(nl + 4 * i);
+    d4[0][i] = *reinterpret_cast<const ulonglong2 *>(nd + 4 * i);
+  }
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     tmem_wait_ld();
     if (c < 3) {
       tmem_ld16(tS + 16 * (c + 1), xs[(c + 1) & 1]);
       tmem_ld16(tdP + 16 * (c + 1), xp[(c + 1) & 1]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        l4[(c + 1) & 1][i] = *reinterpret_cast<const ulonglong2 *>(nl + 16 * (c + 1) + 4 * i);
+        d4[(c + 1) & 1][i] = *reinterpret_cast<const ulonglong2 *>(nd + 16 * (c + 1) + 4 * i);
+      }
     }
     uint32_t pr[8], pt[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      // statistics of four columns per 16-byte shared-memory read (same address for every lane: broadcast)
-      const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);
-      const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
       const int col = 16 * c + 4 * i;
-      score_pair<MASKED>(xs[c & 1][4 * i], xs[c & 1][4 * i + 1], xp[c & 1][4 * i], xp[c & 1][4 * i + 1], scale2, l4.x, d4.x,
-                         col >= lim, col + 1 >= lim, pr[2 * i], pt[2 * i]);
-      score_pair<MASKED>(xs[c & 1][4 * i + 2], xs[c & 1][4 * i + 3], xp[c & 1][4 * i + 2], xp[c & 1][4 * i + 3], scale2, l4.y, d4.y,
-                         col + 2 >= lim, col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
+      score_pair<MASKED>(xs[c & 1][4 * i], xs[c & 1][4 * i + 1], xp[c & 1][4 * i], xp[c & 1][4 * i + 1], scale2, l4[c & 1][i].x,
+                         d4[c & 1][i].x, col >= lim, col + 1 >= lim, pr[2 * i], pt[2 * i]);
+      score_pair<MASKED>(xs[c & 1][4 * i + 2], xs[c & 1][4 * i + 3], xp[c & 1][4 * i + 2], xp[c & 1][4 * i + 3], scale2,
+                         l4[c & 1][i].y, d4[c & 1][i].y, col + 2 >= lim, col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
     }
     tmem_st8(tS + 8 * c, pr);
     tmem_st8(tdP + 8 * c, pt);
@@ -158,9 +167,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmdO,   // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmK,    // box 64 x 64 rows
               const __grid_constant__ CUtensorMap tmV,    // box 64 x 64 rows
-              const __nv_bfloat16 *__restrict__ Qg, const __nv_bfloat16 *__restrict__ Og,
-              const __nv_bfloat16 *__restrict__ dOg, const float *__restrict__ LSE,
-              __nv_bfloat16 *__restrict__ dQ, __nv_bfloat16 *__restrict__ Zneg, float *__restrict__ stats,
+              const __grid_constant__ CUtensorMap tmdQ,   // store, box 64 x 128 rows
+              const __grid_constant__ CUtensorMap tmZ,    // store, box 64 x 128 rows
+              const __nv_bfloat16 *__restrict__ Og, const __nv_bfloat16 *__restrict__ dOg,
+              const float *__restrict__ LSE, float *__restrict__ stats,
               int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
   constexpr int NB = C::kNB;
@@ -174,7 +184,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done;
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
-  __shared__ float s_rho[NB - 1][128], s_m[NB - 1][128], s_lam[128];
+  __shared__ float s_rho[NB - 1][128], s_m[NB - 1][128], s_lam[128], s_D[128];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
@@ -295,22 +305,30 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
     const size_t grow = static_cast<size_t>(row0 + row);
 
-    // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1)
-    float Dv = 0.f;
-    {
-      const uint4 *o4 = reinterpret_cast<const uint4 *>(Og + grow * D);
-      const uint4 *g4 = reinterpret_cast<const uint4 *>(dOg + grow * D);
+    // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1).  Warpgroup 0 computes the
+    // tile's 128 values with coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
+    if (wg == 0) {
+      constexpr int L = D / 8, RPI = 32 / L;           // lanes per row, rows per warp-wide load
+      const int sub = lane / L, part = lane % L;
 #pragma unroll 4
-      for (int v = 0; v < D / 8; ++v) {
-        const uint4 a = __ldg(o4 + v), b = __ldg(g4 + v);
+      for (int it = 0; it < 32 / RPI; ++it) {
+        const int r = 32 * (warp & 3) + it * RPI + sub;
+        const uint4 a = __ldg(reinterpret_cast<const uint4 *>(Og + static_cast<size_t>(row0 + r) * D) + part);
+        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(dOg + static_cast<size_t>(row0 + r) * D) + part);
         const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+        float acc = 0.f;
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-          Dv = fmaf(bf16_lo_to_f32(aw[w]), bf16_lo_to_f32(bw[w]), Dv);
-          Dv = fmaf(bf16_hi_to_f32(aw[w]), bf16_hi_to_f32(bw[w]), Dv);
+          acc = fmaf(bf16_lo_to_f32(aw[w]), bf16_lo_to_f32(bw[w]), acc);
+          acc = fmaf(bf16_hi_to_f32(aw[w]), bf16_hi_to_f32(bw[w]), acc);
         }
+#pragma unroll
+        for (int off = L / 2; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (part == 0) s_D[r] = acc;
       }
     }
+    named_bar_sync(2, 128 * NB);
+    const float Dv = s_D[row];
     const float neg_lse2 = -LSE[grow] * 1.4426950408889634f;
     if (wg == 0) {   // per 64-row block: 64 x {-LSE log2 e}, then 64 x {-D}
       float *blk = stats + (grow >> 6) * 128 + (grow & 63);
@@ -349,19 +367,20 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 
     mbar_wait(&bar_acc_done, 0, ab, kDqWaitAcc);
     tc_fence_after();
-    // the 32-column chunks of the epilogue are dealt round-robin to the warpgroups
+    // The 32-column chunks of the epilogue are dealt round-robin to the warpgroups.  Results are staged in the
+    // TMA (128-byte swizzled) layout over the Q and dO tiles, which no MMA reads any more, and written out by
+    // two TMA stores per slab: Z = -BF16(lambda q) in place over q, dQ over dO.
     for (int cc = wg; cc < D / 32; cc += NB) {
       const int col = 32 * cc;
       uint32_t a[32], b[32];
       tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
       tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);
       tmem_wait_ld();
-      const uint4 *q4 = reinterpret_cast<const uint4 *>(Qg + grow * D + col);
-      uint4 *dq4 = reinterpret_cast<uint4 *>(dQ + grow * D + col);
-      uint4 *z4 = reinterpret_cast<uint4 *>(Zneg + grow * D + col);
+      uint8_t *qslab = sQ + (cc >> 1) * C::kBigSlabBytes, *oslab = sdO + (cc >> 1) * C::kBigSlabBytes;
 #pragma unroll
       for (int v = 0; v < 4; ++v) {
-        const uint4 qv = __ldg(q4 + v);
+        const uint32_t off = swz128_offset(row, 4 * (cc & 1) + v);
+        const uint4 qv = *reinterpret_cast<const uint4 *>(qslab + off);
         const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
         uint32_t dqw[4], zw[4];
 #pragma unroll
@@ -373,9 +392,19 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
           // z = BF16(fl32[lambda q]); the sign flip is exact
           zw[w] = pack_bf16x2(__fmul_rn(lam_k, bf16_lo_to_f32(qw[w])), __fmul_rn(lam_k, bf16_hi_to_f32(qw[w]))) ^ 0x80008000u;
         }
-        dq4[v] = make_uint4(dqw[0], dqw[1], dqw[2], dqw[3]);
-        z4[v] = make_uint4(zw[0], zw[1], zw[2], zw[3]);
+        *reinterpret_cast<uint4 *>(oslab + off) = make_uint4(dqw[0], dqw[1], dqw[2], dqw[3]);
+        *reinterpret_cast<uint4 *>(qslab + off) = make_uint4(zw[0], zw[1], zw[2], zw[3]);
       }
+    }
+    fence_proxy_async_smem();
+    named_bar_sync(1, 128 * NB);
+    if (threadIdx.x == 128) {
+      for (int sl = 0; sl < C::kSlabs; ++sl) {
+        tma_store_2d(&tmdQ, sdO + sl * C::kBigSlabBytes, sl * 64, row0);
+        tma_store_2d(&tmZ, sQ + sl * C::kBigSlabBytes, sl * 64, row0);
+      }
+      bulk_commit_group();
+      bulk_wait_group_read0();
     }
   }
 
@@ -394,7 +423,9 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmQ,    // box 64 x 64 rows
                const __grid_constant__ CUtensorMap tmdO,   // box 64 x 64 rows
                const __grid_constant__ CUtensorMap tmZ,    // box 64 x 64 rows
-               const float *__restrict__ stats, __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV,
+               const __grid_constant__ CUtensorMap tmdK,   // store, box 64 x 128 rows
+               const __grid_constant__ CUtensorMap tmdV,   // store, box 64 x 128 rows
+               const float *__restrict__ stats,
                int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
   constexpr int NB = C::kNB;
@@ -560,17 +591,17 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
 
     mbar_wait(&bar_acc_done, 0, ab, kDkvWaitAcc);
     tc_fence_after();
-    const size_t grow = static_cast<size_t>(krow0 + row);
+    // staged in the TMA layout over the K and V tiles (no MMA reads them any more), then stored by TMA
     for (int cc = wg; cc < D / 32; cc += NB) {
       const int col = 32 * cc;
       uint32_t a[32], b[32];
       tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
       tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);
       tmem_wait_ld();
-      uint4 *dv4 = reinterpret_cast<uint4 *>(dV + grow * D + col);
-      uint4 *dk4 = reinterpret_cast<uint4 *>(dK + grow * D + col);
+      uint8_t *vslab = sV + (cc >> 1) * C::kBigSlabBytes, *kslab = sK + (cc >> 1) * C::kBigSlabBytes;
 #pragma unroll
       for (int v = 0; v < 4; ++v) {
+        const uint32_t off = swz128_offset(row, 4 * (cc & 1) + v);
         uint32_t vw[4], kw[4];
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
@@ -578,9 +609,19 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
           vw[w] = pack_bf16x2(__uint_as_float(a[i]), __uint_as_float(a[i + 1]));
           kw[w] = pack_bf16x2(__fmul_rn(alpha, __uint_as_float(b[i])), __fmul_rn(alpha, __uint_as_float(b[i + 1])));
         }
-        dv4[v] = make_uint4(vw[0], vw[1], vw[2], vw[3]);
-        dk4[v] = make_uint4(kw[0], kw[1], kw[2], kw[3]);
+        *reinterpret_cast<uint4 *>(vslab + off) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
+        *reinterpret_cast<uint4 *>(kslab + off) = make_uint4(kw[0], kw[1], kw[2], kw[3]);
       }
+    }
+    fence_proxy_async_smem();
+    named_bar_sync(1, 128 * NB);
+    if (threadIdx.x == 128) {
+      for (int sl = 0; sl < C::kSlabs; ++sl) {
+        tma_store_2d(&tmdV, sV + sl * C::kBigSlabBytes, sl * 64, krow0);
+        tma_store_2d(&tmdK, sK + sl * C::kBigSlabBytes, sl * 64, krow0);
+      }
+      bulk_commit_group();
+      bulk_wait_group_read0();
     }
   }
 

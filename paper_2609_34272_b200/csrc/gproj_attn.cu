@@ -168,28 +168,27 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
   float *stats = static_cast<float *>(workspace);   // per 64-row block: 64 x {-LSE log2 e}, 64 x {-D}
   __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + align256(rows * sizeof(float2)));
 
-  CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64;
+  CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64, mdQst, mZst, mdKst, mdVst;
   bool ok = make_map(&mQ128, Q, rows, d, 128) && make_map(&mdO128, dO, rows, d, 128) && make_map(&mK64, K, rows, d, 64) &&
             make_map(&mV64, V, rows, d, 64) && make_map(&mK128, K, rows, d, 128) && make_map(&mV128, V, rows, d, 128) &&
-            make_map(&mQ64, Q, rows, d, 64) && make_map(&mdO64, dO, rows, d, 64) && make_map(&mZ64, Zneg, rows, d, 64);
+            make_map(&mQ64, Q, rows, d, 64) && make_map(&mdO64, dO, rows, d, 64) && make_map(&mZ64, Zneg, rows, d, 64) &&
+            make_map(&mdQst, dQ, rows, d, 128) && make_map(&mZst, Zneg, rows, d, 128) && make_map(&mdKst, dK, rows, d, 128) &&
+            make_map(&mdVst, dV, rows, d, 128);
   if (!ok) return GPROJ_ERR_CUDA;
 
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
   const dim3 grid(static_cast<unsigned>(BH * (N / 128)));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const __nv_bfloat16 *Qb = static_cast<const __nv_bfloat16 *>(Q), *Ob = static_cast<const __nv_bfloat16 *>(O),
-                      *dOb = static_cast<const __nv_bfloat16 *>(dO);
-  __nv_bfloat16 *dQb = static_cast<__nv_bfloat16 *>(dQ), *dKb = static_cast<__nv_bfloat16 *>(dK),
-                *dVb = static_cast<__nv_bfloat16 *>(dV);
+  const __nv_bfloat16 *Ob = static_cast<const __nv_bfloat16 *>(O), *dOb = static_cast<const __nv_bfloat16 *>(dO);
 #define GPROJ_LAUNCH_BWD(DD, CC)                                                                                        \
   do {                                                                                                                  \
     if (run_dq)                                                                                                         \
       bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                               \
-          mQ128, mdO128, mK64, mV64, Qb, Ob, dOb, LSE, dQb, Zneg, stats, N, BH, scale_log2, softmax_scale, flags,       \
+          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, N, BH, scale_log2, softmax_scale, flags,         \
           st->status_ptr);                                                                                              \
     if (run_dkv)                                                                                                        \
       bwd_dkv_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
-          mK128, mV128, mQ64, mdO64, mZ64, stats, dKb, dVb, N, BH, scale_log2, softmax_scale, flags, st->status_ptr);   \
+          mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, N, BH, scale_log2, softmax_scale, flags, st->status_ptr); \
   } while (0)
   if (d == 64) { if (causal) GPROJ_LAUNCH_BWD(64, true); else GPROJ_LAUNCH_BWD(64, false); }
   else         { if (causal) GPROJ_LAUNCH_BWD(128, true); else GPROJ_LAUNCH_BWD(128, false); }

@@ -119,6 +119,21 @@ __device__ __forceinline__ void bulk_load_1d(void *smem_dst, const void *gmem_sr
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// TMA: 2-D tiled store shared -> global (bulk-group completion).  x must be a multiple of 8 BF16 elements; y >= 0.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, const void *smem_src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all committed bulk stores of this thread have finished READING shared memory (it may be reused or released)
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+// Byte offset of 16-byte chunk `chunk16` (0..7) of row `row` inside a 128-byte-row slab laid out with the
+// 128-byte swizzle TMA uses (chunk index XOR row mod 8).  Slab bases are 1024-byte aligned.
+__device__ __forceinline__ uint32_t swz128_offset(int row, int chunk16) {
+  return static_cast<uint32_t>(row) * 128u + (static_cast<uint32_t>(chunk16 ^ (row & 7)) << 4);
+}
 
 // ------------------------------------------------------------------------------------------
 // TMEM allocation (one full warp executes these)

@@ -26,6 +26,13 @@
 // Two warps therefore issue: warp 1 the score products of every step, warp 2 the second-stage products; each
 // one's bookkeeping overlaps the other's MMAs.  Reuse of a score buffer is ordered by an explicit barrier
 // (second-stage MMAs of step n committed -> scores of step n + kNB may be issued).
+//
+// Persistence.  One CTA per SM walks a static list of tiles: tiles are ordered by decreasing work and dealt
+// to the CTAs in boustrophedon rounds, which balances causal work as well as a greedy scheduler would while
+// staying deterministic and needing no counter.  Barrier set-up, the TMEM allocation and the launch latency
+// are paid once; the step pipeline (stage ring, score buffers) runs on across tile boundaries, the stationary
+// tile of the next work item is fetched by its own warp as soon as the last score product of the current one
+// has been issued and completed, and the epilogue of one tile overlaps the first steps of the next.
 #pragma once
 #include "sm100_primitives.cuh"
 
@@ -43,7 +50,9 @@ struct BwdCfg {
   static constexpr int kStepSlabBytes = kStepRows * 128;
   static constexpr int kStepTileBytes = kSlabs * kStepSlabBytes;
   static constexpr int kNB = (D == 64) ? 3 : 2;                   // score buffers = compute warpgroups
-  static constexpr int kThreads = 128 + 128 * kNB;                // producer, 2 MMA warps, 1 spare; kNB compute warpgroups
+  static constexpr int kThreads = 128 + 128 * kNB;                // stage producer, 2 MMA warps, tile loader; kNB compute warpgroups
+  // Output staging for the TMA stores: its own buffer where shared memory allows (d = 64), else over the stationary tile.
+  static constexpr bool kSepStaging = (D == 64);
   // TMEM columns: buffer b holds S at 128 b and dP at 128 b + 64; accumulators follow
   static constexpr int kTmemCols = 512;
   static constexpr uint32_t kColAcc0 = 128 * kNB, kColAcc1 = 128 * kNB + D;
@@ -51,17 +60,31 @@ struct BwdCfg {
   // dQ-side kernel: Q, dO resident; ring of (K, V) step tiles
   static constexpr int kDqStages = (D == 64) ? 6 : 4;
   static constexpr int kDqStageBytes = 2 * kStepTileBytes;
-  static constexpr int kDqSmemBytes = 2 * kBigTileBytes + kDqStages * kDqStageBytes + 1024;
+  static constexpr int kDqResBufs = (D == 64) ? 2 : 1;             // stationary (Q, dO) buffers
+  static constexpr int kDqSmemBytes = kDqResBufs * 2 * kBigTileBytes + kDqStages * kDqStageBytes + (kSepStaging ? 2 * kBigTileBytes : 0) + 1024;
   // dK/dV-side kernel: K, V resident; ring of (Q, dO, Z, stats) step tiles
   static constexpr int kDkvStages = (D == 64) ? 5 : 3;
   static constexpr int kDkvStageBytes = 3 * kStepTileBytes + 1024;   // + 2 x 64 floats of row statistics (512 B used)
-  static constexpr int kDkvSmemBytes = 2 * kBigTileBytes + kDkvStages * kDkvStageBytes + 1024;
+  static constexpr int kDkvSmemBytes = 2 * kBigTileBytes + kDkvStages * kDkvStageBytes + (kSepStaging ? 2 * kBigTileBytes : 0) + 1024;
   static_assert(kDqStages >= kNB + 1 && kDkvStages >= kNB + 1, "a stage stays busy until its second-stage MMAs finish");
 };
 
+// Static persistent schedule: work items are numbered by decreasing work; round r hands item r G + c to CTA c
+// on even rounds and item r G + (G - 1 - c) on odd rounds (G = number of CTAs).
+struct TileSched {
+  int total, G, c, round;
+  __device__ __forceinline__ explicit TileSched(int total_tiles)
+      : total(total_tiles), G(static_cast<int>(gridDim.x)), c(static_cast<int>(blockIdx.x)), round(0) {}
+  __device__ __forceinline__ int next() {
+    const int idx = round * G + ((round & 1) ? (G - 1 - c) : c);
+    ++round;
+    return idx < total ? idx : -1;
+  }
+};
+
 enum BwdWaitCode {
-  kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26, kDqWaitBuf = 0x27,
-  kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36, kDkvWaitBuf = 0x37
+  kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26, kDqWaitBuf = 0x27, kDqWaitResFree = 0x28, kDqWaitAccFree = 0x29,
+  kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36, kDkvWaitBuf = 0x37, kDkvWaitResFree = 0x38, kDkvWaitAccFree = 0x39
 };
 
 // Arithmetic of one pair of adjacent score columns, shared by both kernels (Algorithm 1 lines 5-8):
@@ -123,35 +146,26 @@ template <bool MASKED>
 __device__ __forceinline__ void dkv_step(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2);
   uint32_t xs[2][16], xp[2][16];
-  ulonglong2 l4[2][4], d4[2][4];     // statistics of 16 columns, fetched one chunk ahead (shared-memory latency is long
-                                     // while the tensor core streams its operands from the same memory)
   tmem_ld16(tS, xs[0]);
   tmem_ld16(tdP, xp[0]);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    l4[0][i] = *reinterpret_cast<const ulonglong2 *>(nl + 4 * i);
-    d4[0][i] = *reinterpret_cast<const ulonglong2 *>(nd + 4 * i);
-  }
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     tmem_wait_ld();
     if (c < 3) {
       tmem_ld16(tS + 16 * (c + 1), xs[(c + 1) & 1]);
       tmem_ld16(tdP + 16 * (c + 1), xp[(c + 1) & 1]);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        l4[(c + 1) & 1][i] = *reinterpret_cast<const ulonglong2 *>(nl + 16 * (c + 1) + 4 * i);
-        d4[(c + 1) & 1][i] = *reinterpret_cast<const ulonglong2 *>(nd + 16 * (c + 1) + 4 * i);
-      }
     }
     uint32_t pr[8], pt[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
+      // statistics of four columns per 16-byte shared-memory read (same address for every lane: broadcast)
+      const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);
+      const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
       const int col = 16 * c + 4 * i;
-      score_pair<MASKED>(xs[c & 1][4 * i], xs[c & 1][4 * i + 1], xp[c & 1][4 * i], xp[c & 1][4 * i + 1], scale2, l4[c & 1][i].x,
-                         d4[c & 1][i].x, col >= lim, col + 1 >= lim, pr[2 * i], pt[2 * i]);
-      score_pair<MASKED>(xs[c & 1][4 * i + 2], xs[c & 1][4 * i + 3], xp[c & 1][4 * i + 2], xp[c & 1][4 * i + 3], scale2,
-                         l4[c & 1][i].y, d4[c & 1][i].y, col + 2 >= lim, col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
+      score_pair<MASKED>(xs[c & 1][4 * i], xs[c & 1][4 * i + 1], xp[c & 1][4 * i], xp[c & 1][4 * i + 1], scale2, l4.x, d4.x,
+                         col >= lim, col + 1 >= lim, pr[2 * i], pt[2 * i]);
+      score_pair<MASKED>(xs[c & 1][4 * i + 2], xs[c & 1][4 * i + 3], xp[c & 1][4 * i + 2], xp[c & 1][4 * i + 3], scale2, l4.y, d4.y,
+                         col + 2 >= lim, col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
     }
     tmem_st8(tS + 8 * c, pr);
     tmem_st8(tdP + 8 * c, pt);
@@ -171,17 +185,17 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmZ,    // store, box 64 x 128 rows
               const __nv_bfloat16 *__restrict__ Og, const __nv_bfloat16 *__restrict__ dOg,
               const float *__restrict__ LSE, float *__restrict__ stats,
-              int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
+              int N, int BH, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
-  constexpr int NB = C::kNB;
+  constexpr int NB = C::kNB, R = C::kDqResBufs, S = C::kDqStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t *sQ = smem;
-  uint8_t *sdO = sQ + C::kBigTileBytes;
-  uint8_t *sKV = sdO + C::kBigTileBytes;    // stage s: K step tile, then V step tile
+  uint8_t *sRes = smem;                                        // buffer rb: Q tile, then dO tile
+  uint8_t *sKV = sRes + R * 2 * C::kBigTileBytes;              // stage s: K step tile, then V step tile
+  uint8_t *sOut = sKV + S * C::kDqStageBytes;                  // staging (dQ tile, then Z tile) when separate
 
-  __shared__ uint64_t bar_q, bar_kv_full[C::kDqStages], bar_kv_empty[C::kDqStages];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done;
+  __shared__ uint64_t bar_res_full[R], bar_res_free[R], bar_kv_full[S], bar_kv_empty[S];
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free;
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
   __shared__ float s_rho[NB - 1][128], s_m[NB - 1][128], s_lam[128], s_D[128];
@@ -192,54 +206,73 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   if (cta_skip != 0) return;   // an earlier wait gave up: drain the rest of the grid quickly
 
   const int n_qt = N / 128;
-  const int lin = blockIdx.x;
-  const int qt = CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH);   // causal: longest rows first
-  const int bh = lin % BH;
-  const int T = CAUSAL ? 2 * (qt + 1) : N / C::kStepRows;       // 64-key steps
-  const int row0 = bh * N + qt * 128;
-
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
-    mbar_init(&bar_q, 1);
-    for (int s = 0; s < C::kDqStages; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
+    for (int r = 0; r < R; ++r) { mbar_init(&bar_res_full[r], 1); mbar_init(&bar_res_free[r], 2); }
+    for (int s = 0; s < S; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
     for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
+    mbar_init(&bar_acc_free, 128 * NB);
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
   if (warp == 0 && lane == 0) {
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmdO); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+    tma_prefetch_desc(&tmdQ); tma_prefetch_desc(&tmZ);
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);   // the shuffle marks it warp-uniform
 
+  TileSched sched(total_tiles);
+  // tile decode: causal -> longest rows first
+  auto tile_qt = [&](int lin) { return CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH); };
+  auto tile_steps = [&](int qt) { return CAUSAL ? 2 * (qt + 1) : N / C::kStepRows; };
+
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producer of the streamed (K, V) step tiles
     if (lane == 0) {
-      mbar_expect_tx(&bar_q, 2 * C::kBigTileBytes);
-      for (int s = 0; s < C::kSlabs; ++s) {
-        tma_load_2d(sQ + s * C::kBigSlabBytes, &tmQ, &bar_q, s * 64, row0);
-        tma_load_2d(sdO + s * C::kBigSlabBytes, &tmdO, &bar_q, s * 64, row0);
-      }
-      for (int n = 0; n < T; ++n) {
-        const int st = n % C::kDqStages;
-        if (n >= C::kDqStages) mbar_wait(&bar_kv_empty[st], ((n / C::kDqStages) - 1) & 1, ab, kDqWaitKVEmpty);
-        mbar_expect_tx(&bar_kv_full[st], C::kDqStageBytes);
-        uint8_t *dst = sKV + st * C::kDqStageBytes;
-        const int krow = bh * N + n * C::kStepRows;
-        for (int s = 0; s < C::kSlabs; ++s) {
-          tma_load_2d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow);
-          tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow);
+      int g = 0;
+      for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
+        const int qt = tile_qt(lin), bh = lin % BH, T = tile_steps(qt);
+        for (int n = 0; n < T; ++n, ++g) {
+          const int st = g % S;
+          if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kDqWaitKVEmpty);
+          mbar_expect_tx(&bar_kv_full[st], C::kDqStageBytes);
+          uint8_t *dst = sKV + st * C::kDqStageBytes;
+          const int krow = bh * N + n * C::kStepRows;
+          for (int s = 0; s < C::kSlabs; ++s) {
+            tma_load_2d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow);
+            tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow);
+          }
         }
       }
       // Every load is consumed by an MMA the epilogue waits for, so nothing is in flight at exit unless the
       // CTA aborted; then give the copies a bounded chance to land before shared memory is released.
       if (cta_abort) {
-        for (int n = (T > C::kDqStages ? T - C::kDqStages : 0); n < T; ++n)
-          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_kv_full[n % C::kDqStages], (n / C::kDqStages) & 1); ++spin) {}
+        for (int q = (g > S ? g - S : 0); q < g; ++q)
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_kv_full[q % S], (q / S) & 1); ++spin) {}
+      }
+    }
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- TMA loader of the stationary (Q, dO) tiles
+    if (lane == 0) {
+      int ti = 0;
+      for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+        const int rb = ti % R, row0 = (lin % BH) * N + tile_qt(lin) * 128;
+        if (ti >= R) mbar_wait(&bar_res_free[rb], ((ti / R) - 1) & 1, ab, kDqWaitResFree);
+        mbar_expect_tx(&bar_res_full[rb], 2 * C::kBigTileBytes);
+        uint8_t *dst = sRes + rb * 2 * C::kBigTileBytes;
+        for (int s = 0; s < C::kSlabs; ++s) {
+          tma_load_2d(dst + s * C::kBigSlabBytes, &tmQ, &bar_res_full[rb], s * 64, row0);
+          tma_load_2d(dst + C::kBigTileBytes + s * C::kBigSlabBytes, &tmdO, &bar_res_full[rb], s * 64, row0);
+        }
+      }
+      if (cta_abort) {
+        for (int q = (ti > R ? ti - R : 0); q < ti; ++q)
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_res_full[q % R], (q / R) & 1); ++spin) {}
       }
     }
   } else if (warp == 1) {
@@ -247,165 +280,195 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     // The whole warp runs this loop so that every address stays provably warp-uniform (descriptor operands
     // then live in uniform registers); one elected lane issues the MMAs and commits.
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 queries] x [64 keys], contraction over d
-    const SmemDesc dscQ = make_smem_desc(smem_u32(sQ), 16, 1024), dscdO = make_smem_desc(smem_u32(sdO), 16, 1024);
+    const SmemDesc dscRes0 = make_smem_desc(smem_u32(sRes), 16, 1024);
     const SmemDesc dscK0 = make_smem_desc(smem_u32(sKV), 16, 1024);                          // K-major view of stage 0
-    mbar_wait(&bar_q, 0, ab, kDqWaitQ);
-    for (int n = 0; n < T; ++n) {
-      const int st = n % C::kDqStages, b = n % NB;
-      mbar_wait(&bar_kv_full[st], (n / C::kDqStages) & 1, ab, kDqWaitKV);
-      if (n >= NB) mbar_wait(&bar_buf_free[b], ((n / NB) - 1) & 1, ab, kDqWaitBuf);   // r, t of step n - NB consumed
-      tc_fence_after();
-      const SmemDesc dscK = dscK0.advanced(st * C::kDqStageBytes), dscV = dscK.advanced(C::kStepTileBytes);
-      const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
-      if (elect_one_sync()) {
+    int g = 0, ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int T = tile_steps(tile_qt(lin)), rb = ti % R;
+      mbar_wait(&bar_res_full[rb], (ti / R) & 1, ab, kDqWaitQ);
+      const SmemDesc dscQ = dscRes0.advanced(rb * 2 * C::kBigTileBytes), dscdO = dscQ.advanced(C::kBigTileBytes);
+      for (int n = 0; n < T; ++n, ++g) {
+        const int st = g % S, b = g % NB;
+        mbar_wait(&bar_kv_full[st], (g / S) & 1, ab, kDqWaitKV);
+        if (g >= NB) mbar_wait(&bar_buf_free[b], ((g / NB) - 1) & 1, ab, kDqWaitBuf);   // r, t of step g - NB consumed
+        tc_fence_after();
+        const SmemDesc dscK = dscK0.advanced(st * C::kDqStageBytes), dscV = dscK.advanced(C::kStepTileBytes);
+        const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
+        if (elect_one_sync()) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-          umma_ss(tS, dscQ.at(oa), dscK.at(ob), idesc_s, k > 0);
-        }
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tS, dscQ.at(oa), dscK.at(ob), idesc_s, k > 0);
+          }
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-          umma_ss(tdP, dscdO.at(oa), dscV.at(ob), idesc_s, k > 0);
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tdP, dscdO.at(oa), dscV.at(ob), idesc_s, k > 0);
+          }
+          umma_commit(&bar_sdp_full[b]);
+          if (n == T - 1) umma_commit(&bar_res_free[rb]);   // no MMA reads this Q / dO buffer any more
         }
-        umma_commit(&bar_sdp_full[b]);
+        __syncwarp();
       }
-      __syncwarp();
     }
   } else if (warp == 2) {
     // ---------------------------------------------------------------- tensor-core issuer 2: A += t K, B += r K
     constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 queries] x [d], contraction over 64 keys
     const SmemDesc dscK0mn = make_smem_desc(smem_u32(sKV), C::kStepSlabBytes, 1024);       // MN-major view of stage 0
-    for (int p = 0; p < T; ++p) {
-      const int st = p % C::kDqStages, b = p % NB;
-      mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDqWaitTR);
-      tc_fence_after();
-      const SmemDesc dscK = dscK0mn.advanced(st * C::kDqStageBytes);
-      const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;     // packed BF16 r / t over the S / dP columns
-      const uint32_t acc = (p > 0) ? 1u : 0u;
-      if (elect_one_sync()) {
+    int g = 0, ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int T = tile_steps(tile_qt(lin));
+      if (ti > 0) mbar_wait(&bar_acc_free, (ti - 1) & 1, ab, kDqWaitAccFree);   // the previous epilogue has read A, B
+      for (int p = 0; p < T; ++p, ++g) {
+        const int st = g % S, b = g % NB;
+        mbar_wait(&bar_tr_ready[b], (g / NB) & 1, ab, kDqWaitTR);
+        tc_fence_after();
+        const SmemDesc dscK = dscK0mn.advanced(st * C::kDqStageBytes);
+        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;     // packed BF16 r / t over the S / dP columns
+        const uint32_t acc = (p > 0) ? 1u : 0u;
+        if (elect_one_sync()) {
 #pragma unroll
-        for (int k = 0; k < C::kStepRows / 16; ++k)
-          umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+          for (int k = 0; k < C::kStepRows / 16; ++k)
+            umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
 #pragma unroll
-        for (int k = 0; k < C::kStepRows / 16; ++k)
-          umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-        umma_commit(&bar_buf_free[b]);
-        umma_commit(&bar_kv_empty[st]);
-        if (p == T - 1) umma_commit(&bar_acc_done);
+          for (int k = 0; k < C::kStepRows / 16; ++k)
+            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+          umma_commit(&bar_buf_free[b]);
+          umma_commit(&bar_kv_empty[st]);
+          if (p == T - 1) umma_commit(&bar_acc_done);
+        }
+        __syncwarp();
       }
-      __syncwarp();
     }
-  } else if (warp == 3) {
-    // spare warp: keeps the compute warpgroups aligned to TMEM lane quadrants
   } else {
     // ---------------------------------------------------------------- compute: thread <-> query row
     const int wg = (warp - 4) >> 2;
     const int row = 32 * (warp & 3) + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
-    const size_t grow = static_cast<size_t>(row0 + row);
-
-    // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1).  Warpgroup 0 computes the
-    // tile's 128 values with coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
-    if (wg == 0) {
-      constexpr int L = D / 8, RPI = 32 / L;           // lanes per row, rows per warp-wide load
-      const int sub = lane / L, part = lane % L;
-#pragma unroll 4
-      for (int it = 0; it < 32 / RPI; ++it) {
-        const int r = 32 * (warp & 3) + it * RPI + sub;
-        const uint4 a = __ldg(reinterpret_cast<const uint4 *>(Og + static_cast<size_t>(row0 + r) * D) + part);
-        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(dOg + static_cast<size_t>(row0 + r) * D) + part);
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-        float acc = 0.f;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          acc = fmaf(bf16_lo_to_f32(aw[w]), bf16_lo_to_f32(bw[w]), acc);
-          acc = fmaf(bf16_hi_to_f32(aw[w]), bf16_hi_to_f32(bw[w]), acc);
-        }
-#pragma unroll
-        for (int off = L / 2; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (part == 0) s_D[r] = acc;
-      }
-    }
-    named_bar_sync(2, 128 * NB);
-    const float Dv = s_D[row];
-    const float neg_lse2 = -LSE[grow] * 1.4426950408889634f;
-    if (wg == 0) {   // per 64-row block: 64 x {-LSE log2 e}, then 64 x {-D}
-      float *blk = stats + (grow >> 6) * 128 + (grow & 63);
-      blk[0] = neg_lse2;
-      blk[64] = -Dv;
-    }
-
-    uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);
     const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
-    for (int n = wg, k = 0; n < T; n += NB, ++k) {
-      mbar_wait(&bar_sdp_full[wg], k & 1, ab, kDqWaitSdP);
-      tc_fence_after();
-      if (CAUSAL && n >= T - 2) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho2, msum2);
-      else                      dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bar_tr_ready[wg]);
-    }
+    int g0 = 0, ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int qt = tile_qt(lin), bh = lin % BH, T = tile_steps(qt), rb = ti % R;
+      const int row0 = bh * N + qt * 128;
+      const size_t grow = static_cast<size_t>(row0 + row);
 
-    // ---- row statistics of all warpgroups (fixed order), lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
-    float rho_lo, rho_hi, m_lo, m_hi;
-    f32x2_split(rho2, rho_lo, rho_hi);
-    f32x2_split(msum2, m_lo, m_hi);
-    float rho_t = rho_lo + rho_hi, m_t = m_lo + m_hi;
-    if (wg > 0) { s_rho[wg - 1][row] = rho_t; s_m[wg - 1][row] = m_t; }
-    named_bar_sync(1, 128 * NB);
-    if (wg == 0) {
+      // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1).  Warpgroup 0 computes the
+      // tile's 128 values with coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
+      if (wg == 0) {
+        constexpr int L = D / 8, RPI = 32 / L;           // lanes per row, rows per warp-wide load
+        const int sub = lane / L, part = lane % L;
+#pragma unroll 4
+        for (int it = 0; it < 32 / RPI; ++it) {
+          const int r = 32 * (warp & 3) + it * RPI + sub;
+          const uint4 a = __ldg(reinterpret_cast<const uint4 *>(Og + static_cast<size_t>(row0 + r) * D) + part);
+          const uint4 b = __ldg(reinterpret_cast<const uint4 *>(dOg + static_cast<size_t>(row0 + r) * D) + part);
+          const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+          float acc = 0.f;
 #pragma unroll
-      for (int w = 0; w < NB - 1; ++w) { rho_t += s_rho[w][row]; m_t += s_m[w][row]; }
-      s_lam[row] = (m_t != 0.f) ? __fdiv_rn(rho_t, m_t) : 0.f;
-    }
-    named_bar_sync(1, 128 * NB);
-    const float lam = s_lam[row];
-    const float lam_q = (flags & kFlagNoQCorrection) ? 0.f : lam;
-    const float lam_k = (flags & kFlagNoKCorrection) ? 0.f : lam;
-
-    mbar_wait(&bar_acc_done, 0, ab, kDqWaitAcc);
-    tc_fence_after();
-    // The 32-column chunks of the epilogue are dealt round-robin to the warpgroups.  Results are staged in the
-    // TMA (128-byte swizzled) layout over the Q and dO tiles, which no MMA reads any more, and written out by
-    // two TMA stores per slab: Z = -BF16(lambda q) in place over q, dQ over dO.
-    for (int cc = wg; cc < D / 32; cc += NB) {
-      const int col = 32 * cc;
-      uint32_t a[32], b[32];
-      tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
-      tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);
-      tmem_wait_ld();
-      uint8_t *qslab = sQ + (cc >> 1) * C::kBigSlabBytes, *oslab = sdO + (cc >> 1) * C::kBigSlabBytes;
+          for (int w = 0; w < 4; ++w) {
+            acc = fmaf(bf16_lo_to_f32(aw[w]), bf16_lo_to_f32(bw[w]), acc);
+            acc = fmaf(bf16_hi_to_f32(aw[w]), bf16_hi_to_f32(bw[w]), acc);
+          }
 #pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        const uint32_t off = swz128_offset(row, 4 * (cc & 1) + v);
-        const uint4 qv = *reinterpret_cast<const uint4 *>(qslab + off);
-        const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
-        uint32_t dqw[4], zw[4];
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const int i = 8 * v + 2 * w;
-          const float g0 = __fmul_rn(alpha, __fsub_rn(__uint_as_float(a[i]), __fmul_rn(lam_q, __uint_as_float(b[i]))));
-          const float g1 = __fmul_rn(alpha, __fsub_rn(__uint_as_float(a[i + 1]), __fmul_rn(lam_q, __uint_as_float(b[i + 1]))));
-          dqw[w] = pack_bf16x2(g0, g1);
-          // z = BF16(fl32[lambda q]); the sign flip is exact
-          zw[w] = pack_bf16x2(__fmul_rn(lam_k, bf16_lo_to_f32(qw[w])), __fmul_rn(lam_k, bf16_hi_to_f32(qw[w]))) ^ 0x80008000u;
+          for (int off = L / 2; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+          if (part == 0) s_D[r] = acc;
         }
-        *reinterpret_cast<uint4 *>(oslab + off) = make_uint4(dqw[0], dqw[1], dqw[2], dqw[3]);
-        *reinterpret_cast<uint4 *>(qslab + off) = make_uint4(zw[0], zw[1], zw[2], zw[3]);
       }
-    }
-    fence_proxy_async_smem();
-    named_bar_sync(1, 128 * NB);
-    if (threadIdx.x == 128) {
-      for (int sl = 0; sl < C::kSlabs; ++sl) {
-        tma_store_2d(&tmdQ, sdO + sl * C::kBigSlabBytes, sl * 64, row0);
-        tma_store_2d(&tmZ, sQ + sl * C::kBigSlabBytes, sl * 64, row0);
+      named_bar_sync(2, 128 * NB);
+      const float Dv = s_D[row];
+      const float neg_lse2 = -LSE[grow] * 1.4426950408889634f;
+      if (wg == 0) {   // per 64-row block: 64 x {-LSE log2 e}, then 64 x {-D}
+        float *blk = stats + (grow >> 6) * 128 + (grow & 63);
+        blk[0] = neg_lse2;
+        blk[64] = -Dv;
       }
-      bulk_commit_group();
-      bulk_wait_group_read0();
+
+      uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);
+      for (int n = (wg - g0 % NB + NB) % NB; n < T; n += NB) {
+        mbar_wait(&bar_sdp_full[wg], ((g0 + n) / NB) & 1, ab, kDqWaitSdP);
+        tc_fence_after();
+        if (CAUSAL && n >= T - 2) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho2, msum2);
+        else                      dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bar_tr_ready[wg]);
+      }
+
+      // ---- row statistics of all warpgroups (fixed order), lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
+      float rho_lo, rho_hi, m_lo, m_hi;
+      f32x2_split(rho2, rho_lo, rho_hi);
+      f32x2_split(msum2, m_lo, m_hi);
+      float rho_t = rho_lo + rho_hi, m_t = m_lo + m_hi;
+      if (wg > 0) { s_rho[wg - 1][row] = rho_t; s_m[wg - 1][row] = m_t; }
+      if (C::kSepStaging && threadIdx.x == 128) bulk_wait_group_read0();   // the previous tile's stores have left the staging buffer
+      named_bar_sync(1, 128 * NB);
+      if (wg == 0) {
+#pragma unroll
+        for (int w = 0; w < NB - 1; ++w) { rho_t += s_rho[w][row]; m_t += s_m[w][row]; }
+        s_lam[row] = (m_t != 0.f) ? __fdiv_rn(rho_t, m_t) : 0.f;
+      }
+      named_bar_sync(1, 128 * NB);
+      const float lam = s_lam[row];
+      const float lam_q = (flags & kFlagNoQCorrection) ? 0.f : lam;
+      const float lam_k = (flags & kFlagNoKCorrection) ? 0.f : lam;
+
+      mbar_wait(&bar_acc_done, ti & 1, ab, kDqWaitAcc);
+      tc_fence_after();
+      // The 32-column chunks of the epilogue are dealt round-robin to the warpgroups.  Results are staged in the
+      // TMA (128-byte swizzled) layout and written out by TMA stores: Z = -BF16(lambda q), dQ.
+      uint8_t *sQt = sRes + rb * 2 * C::kBigTileBytes, *sdOt = sQt + C::kBigTileBytes;
+      uint8_t *stage_dq = C::kSepStaging ? sOut : sdOt, *stage_z = C::kSepStaging ? sOut + C::kBigTileBytes : sQt;
+      constexpr int kMaxCh = (D / 32 + NB - 1) / NB;       // epilogue chunks per warpgroup
+      uint32_t a[kMaxCh][32], b[kMaxCh][32];
+#pragma unroll
+      for (int nch = 0; nch < kMaxCh; ++nch) {
+        const int cc = wg + nch * NB;
+        if (cc < D / 32) {
+          tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + 32 * cc, a[nch]);
+          tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + 32 * cc, b[nch]);
+        }
+      }
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(&bar_acc_free);          // the accumulators may be overwritten by the next tile
+#pragma unroll
+      for (int nch = 0; nch < kMaxCh; ++nch) {
+        const int cc = wg + nch * NB;
+        if (cc >= D / 32) break;
+        const uint32_t slab = (cc >> 1) * C::kBigSlabBytes;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const uint32_t off = slab + swz128_offset(row, 4 * (cc & 1) + v);
+          const uint4 qv = *reinterpret_cast<const uint4 *>(sQt + off);
+          const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
+          uint32_t dqw[4], zw[4];
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const int i = 8 * v + 2 * w;
+            const float g0v = __fmul_rn(alpha, __fsub_rn(__uint_as_float(a[nch][i]), __fmul_rn(lam_q, __uint_as_float(b[nch][i]))));
+            const float g1v = __fmul_rn(alpha, __fsub_rn(__uint_as_float(a[nch][i + 1]), __fmul_rn(lam_q, __uint_as_float(b[nch][i + 1]))));
+            dqw[w] = pack_bf16x2(g0v, g1v);
+            // z = BF16(fl32[lambda q]); the sign flip is exact
+            zw[w] = pack_bf16x2(__fmul_rn(lam_k, bf16_lo_to_f32(qw[w])), __fmul_rn(lam_k, bf16_hi_to_f32(qw[w]))) ^ 0x80008000u;
+          }
+          *reinterpret_cast<uint4 *>(stage_dq + off) = make_uint4(dqw[0], dqw[1], dqw[2], dqw[3]);
+          *reinterpret_cast<uint4 *>(stage_z + off) = make_uint4(zw[0], zw[1], zw[2], zw[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      named_bar_sync(1, 128 * NB);
+      if (threadIdx.x == 128) {
+        for (int sl = 0; sl < C::kSlabs; ++sl) {
+          tma_store_2d(&tmdQ, stage_dq + sl * C::kBigSlabBytes, sl * 64, row0);
+          tma_store_2d(&tmZ, stage_z + sl * C::kBigSlabBytes, sl * 64, row0);
+        }
+        bulk_commit_group();
+        if (!C::kSepStaging) bulk_wait_group_read0();     // staging shares the Q / dO buffer: reads must finish first
+        mbar_arrive(&bar_res_free[rb]);                   // second arrival: the epilogue no longer needs this buffer
+      }
+      g0 += T;
     }
+    if (threadIdx.x == 128) bulk_wait_group_read0();
   }
 
   tc_fence_before();
@@ -426,17 +489,18 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmdK,   // store, box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmdV,   // store, box 64 x 128 rows
                const float *__restrict__ stats,
-               int N, int BH, float scale_log2, float alpha, unsigned flags, int *status) {
+               int N, int BH, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
-  constexpr int NB = C::kNB;
+  constexpr int NB = C::kNB, S = C::kDkvStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sK = smem;
   uint8_t *sV = sK + C::kBigTileBytes;
   uint8_t *sStage = sV + C::kBigTileBytes;   // stage s: Q, dO, Z step tiles, then 64 x {-LSE log2 e} and 64 x {-D}
+  uint8_t *sOut = sStage + S * C::kDkvStageBytes;   // staging (dK tile, then dV tile) when separate
 
-  __shared__ uint64_t bar_kv, bar_q_full[C::kDkvStages], bar_q_empty[C::kDkvStages];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done;
+  __shared__ uint64_t bar_res_full, bar_res_free, bar_q_full[S], bar_q_empty[S];
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free;
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -445,184 +509,245 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   __syncthreads();
   if (cta_skip != 0) return;
 
-  const int lin = blockIdx.x;
-  const int kt = lin / BH;                                   // causal: key tile 0 has the most query steps -> first
-  const int bh = lin % BH;
-  const int q_start = CAUSAL ? kt * 128 : 0;
-  const int T = (N - q_start) / C::kStepRows;                 // 64-query steps
-  const int krow0 = bh * N + kt * 128;
   const bool use_z = (flags & kFlagNoKCorrection) == 0;
   const uint32_t stage_tx = (use_z ? 3 : 2) * C::kStepTileBytes + 512;
 
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
-    mbar_init(&bar_kv, 1);
-    for (int s = 0; s < C::kDkvStages; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
+    mbar_init(&bar_res_full, 1);
+    mbar_init(&bar_res_free, 2);
+    for (int s = 0; s < S; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
     for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
+    mbar_init(&bar_acc_free, 128 * NB);
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
   if (warp == 0 && lane == 0) {
     tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmdO); tma_prefetch_desc(&tmZ);
+    tma_prefetch_desc(&tmdK); tma_prefetch_desc(&tmdV);
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);
 
+  TileSched sched(total_tiles);
+  // tile decode: causal -> key tile 0 has the most query steps and comes first
+  auto tile_q_start = [&](int kt) { return CAUSAL ? kt * 128 : 0; };
+  auto tile_steps = [&](int kt) { return (N - tile_q_start(kt)) / C::kStepRows; };
+
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producer of the streamed (Q, dO, Z, stats) step tiles
     if (lane == 0) {
-      mbar_expect_tx(&bar_kv, 2 * C::kBigTileBytes);
-      for (int s = 0; s < C::kSlabs; ++s) {
-        tma_load_2d(sK + s * C::kBigSlabBytes, &tmK, &bar_kv, s * 64, krow0);
-        tma_load_2d(sV + s * C::kBigSlabBytes, &tmV, &bar_kv, s * 64, krow0);
-      }
-      for (int n = 0; n < T; ++n) {
-        const int st = n % C::kDkvStages;
-        if (n >= C::kDkvStages) mbar_wait(&bar_q_empty[st], ((n / C::kDkvStages) - 1) & 1, ab, kDkvWaitQEmpty);
-        mbar_expect_tx(&bar_q_full[st], stage_tx);
-        uint8_t *dst = sStage + st * C::kDkvStageBytes;
-        const int qrow = bh * N + q_start + n * C::kStepRows;
-        for (int s = 0; s < C::kSlabs; ++s) {
-          tma_load_2d(dst + s * C::kStepSlabBytes, &tmQ, &bar_q_full[st], s * 64, qrow);
-          tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow);
-          if (use_z) tma_load_2d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow);
+      int g = 0;
+      for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
+        const int kt = lin / BH, bh = lin % BH, T = tile_steps(kt), q_start = tile_q_start(kt);
+        for (int n = 0; n < T; ++n, ++g) {
+          const int st = g % S;
+          if (g >= S) mbar_wait(&bar_q_empty[st], ((g / S) - 1) & 1, ab, kDkvWaitQEmpty);
+          mbar_expect_tx(&bar_q_full[st], stage_tx);
+          uint8_t *dst = sStage + st * C::kDkvStageBytes;
+          const int qrow = bh * N + q_start + n * C::kStepRows;
+          for (int s = 0; s < C::kSlabs; ++s) {
+            tma_load_2d(dst + s * C::kStepSlabBytes, &tmQ, &bar_q_full[st], s * 64, qrow);
+            tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow);
+            if (use_z) tma_load_2d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow);
+          }
+          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + 2 * static_cast<size_t>(qrow), 512, &bar_q_full[st]);
         }
-        bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + 2 * static_cast<size_t>(qrow), 512, &bar_q_full[st]);
       }
       if (cta_abort) {
-        for (int n = (T > C::kDkvStages ? T - C::kDkvStages : 0); n < T; ++n)
-          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full[n % C::kDkvStages], (n / C::kDkvStages) & 1); ++spin) {}
+        for (int q = (g > S ? g - S : 0); q < g; ++q)
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full[q % S], (q / S) & 1); ++spin) {}
       }
+    }
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- TMA loader of the stationary (K, V) tiles
+    if (lane == 0) {
+      int ti = 0;
+      for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+        const int krow0 = (lin % BH) * N + (lin / BH) * 128;
+        if (ti >= 1) mbar_wait(&bar_res_free, (ti - 1) & 1, ab, kDkvWaitResFree);
+        mbar_expect_tx(&bar_res_full, 2 * C::kBigTileBytes);
+        for (int s = 0; s < C::kSlabs; ++s) {
+          tma_load_2d(sK + s * C::kBigSlabBytes, &tmK, &bar_res_full, s * 64, krow0);
+          tma_load_2d(sV + s * C::kBigSlabBytes, &tmV, &bar_res_full, s * 64, krow0);
+        }
+      }
+      if (cta_abort && ti > 0)
+        for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_res_full, (ti - 1) & 1); ++spin) {}
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- tensor-core issuer 1: scores (warp-uniform loop, elected issue)
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 keys] x [64 queries], contraction over d
     const SmemDesc dscK = make_smem_desc(smem_u32(sK), 16, 1024), dscV = make_smem_desc(smem_u32(sV), 16, 1024);
     const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);                       // K-major view of stage 0
-    mbar_wait(&bar_kv, 0, ab, kDkvWaitKV);
-    for (int n = 0; n < T; ++n) {
-      const int st = n % C::kDkvStages, b = n % NB;
-      if (lane == 0) trace_stamp(0, n, 0);
-      mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);
-      if (n >= NB) mbar_wait(&bar_buf_free[b], ((n / NB) - 1) & 1, ab, kDkvWaitBuf);   // r, t of step n - NB consumed
-      tc_fence_after();
-      if (lane == 0) trace_stamp(0, n, 1);
-      const SmemDesc dscQ = dscQ0.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes);
-      const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
-      if (elect_one_sync()) {
+    int g = 0, ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int T = tile_steps(lin / BH);
+      mbar_wait(&bar_res_full, ti & 1, ab, kDkvWaitKV);
+      for (int n = 0; n < T; ++n, ++g) {
+        const int st = g % S, b = g % NB;
+        mbar_wait(&bar_q_full[st], (g / S) & 1, ab, kDkvWaitQ);
+        if (g >= NB) mbar_wait(&bar_buf_free[b], ((g / NB) - 1) & 1, ab, kDkvWaitBuf);   // r, t of step g - NB consumed
+        tc_fence_after();
+        const SmemDesc dscQ = dscQ0.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes);
+        const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
+        if (elect_one_sync()) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-          umma_ss(tS, dscK.at(oa), dscQ.at(ob), idesc_s, k > 0);
-        }
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tS, dscK.at(oa), dscQ.at(ob), idesc_s, k > 0);
+          }
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
-          umma_ss(tdP, dscV.at(oa), dscdO.at(ob), idesc_s, k > 0);
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
+            umma_ss(tdP, dscV.at(oa), dscdO.at(ob), idesc_s, k > 0);
+          }
+          umma_commit(&bar_sdp_full[b]);
+          if (n == T - 1) umma_commit(&bar_res_free);   // no MMA reads this K / V tile any more
         }
-        umma_commit(&bar_sdp_full[b]);
-        trace_stamp(0, n, 2);
+        __syncwarp();
       }
-      __syncwarp();
     }
   } else if (warp == 2) {
     // ---------------------------------------------------------------- tensor-core issuer 2: dV += r^T dO, dK += t^T Q + r^T Z
     constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 keys] x [d], contraction over 64 queries
+    constexpr uint32_t idesc_fused = idesc_bf16_f32(128, 128, 0, 1);   // d = 64 only: [128 keys] x [dO | Z]
     const SmemDesc dscQ0mn = make_smem_desc(smem_u32(sStage), C::kStepSlabBytes, 1024);    // MN-major view of stage 0
-    for (int p = 0; p < T; ++p) {
-      const int st = p % C::kDkvStages, b = p % NB;
-      if (lane == 0) trace_stamp(3, p, 0);
-      mbar_wait(&bar_tr_ready[b], (p / NB) & 1, ab, kDkvWaitTR);
-      tc_fence_after();
-      if (lane == 0) trace_stamp(3, p, 1);
-      const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes),
-                     dscZ = dscdO.advanced(C::kStepTileBytes);
-      const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;
-      const uint32_t acc = (p > 0) ? 1u : 0u;
-      if (elect_one_sync()) {
+    int g = 0, ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int T = tile_steps(lin / BH);
+      if (ti > 0) mbar_wait(&bar_acc_free, (ti - 1) & 1, ab, kDkvWaitAccFree);   // the previous epilogue has read dV, dK
+      for (int p = 0; p < T; ++p, ++g) {
+        const int st = g % S, b = g % NB;
+        mbar_wait(&bar_tr_ready[b], (g / NB) & 1, ab, kDkvWaitTR);
+        tc_fence_after();
+        const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes),
+                       dscZ = dscdO.advanced(C::kStepTileBytes);
+        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;
+        const uint32_t acc = (p > 0) ? 1u : 0u;
+        if (elect_one_sync()) {
+          if (D == 64 && use_z) {
+            // d = 64: the dO and Z step tiles are adjacent 64-column atoms of one MN-major operand and the dV and dK
+            // accumulators are adjacent TMEM columns, so r^T [dO | Z] is ONE full-rate N = 128 product
+            // (an N = 64 instruction costs as much as 0.7 of an N = 128 one).  dK gets its main term t^T Q afterwards.
 #pragma unroll
-        for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
-          umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+            for (int k = 0; k < C::kStepRows / 16; ++k)    // [dV | dK] += r^T [dO | -BF16(lambda Q)]
+              umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_fused, k > 0 ? 1u : acc);
 #pragma unroll
-        for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
-          umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-        if (use_z) {
+            for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += t^T Q
+              umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, 1u);
+          } else {
 #pragma unroll
-          for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
-            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscZ.at(k * 2048), idesc_a, 1u);
+            for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
+              umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+#pragma unroll
+            for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
+              umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+            if (use_z) {
+#pragma unroll
+              for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
+                umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscZ.at(k * 2048), idesc_a, 1u);
+            }
+          }
+          umma_commit(&bar_buf_free[b]);
+          umma_commit(&bar_q_empty[st]);
+          if (p == T - 1) umma_commit(&bar_acc_done);
         }
-        umma_commit(&bar_buf_free[b]);
-        umma_commit(&bar_q_empty[st]);
-        if (p == T - 1) umma_commit(&bar_acc_done);
-        trace_stamp(3, p, 2);
+        __syncwarp();
       }
-      __syncwarp();
     }
-  } else if (warp == 3) {
-    // spare warp: keeps the compute warpgroups aligned to TMEM lane quadrants
   } else {
     // ---------------------------------------------------------------- compute: thread <-> key row
     const int wg = (warp - 4) >> 2;
     const int row = 32 * (warp & 3) + lane;                  // key row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
     const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
-    const bool tracer = (threadIdx.x & 127) == 64;
+    int g0 = 0, ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int kt = lin / BH, bh = lin % BH, T = tile_steps(kt);
+      const int krow0 = bh * N + kt * 128;
+#ifdef GPROJ_TRACE
+      const unsigned long long tile_t0 = global_ns();
+#endif
+      for (int n = (wg - g0 % NB + NB) % NB; n < T; n += NB) {
+        const int g = g0 + n, st = g % S;
+        mbar_wait(&bar_q_full[st], (g / S) & 1, ab, kDkvWaitQ);      // row statistics of this step landed
+        mbar_wait(&bar_sdp_full[wg], (g / NB) & 1, ab, kDkvWaitSdP);
+        tc_fence_after();
+        const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
+        if (CAUSAL && n < 2) dkv_step<true>(tS, tdP, nl, nl + 64, scale_log2, row - n * C::kStepRows);
+        else                 dkv_step<false>(tS, tdP, nl, nl + 64, scale_log2, 0);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bar_tr_ready[wg]);
+      }
 
-    for (int n = wg, k = 0; n < T; n += NB, ++k) {
-      const int st = n % C::kDkvStages;
-      if (tracer) trace_stamp(1 + wg, n, 0);
-      mbar_wait(&bar_q_full[st], (n / C::kDkvStages) & 1, ab, kDkvWaitQ);      // row statistics of this step landed
-      mbar_wait(&bar_sdp_full[wg], k & 1, ab, kDkvWaitSdP);
+      mbar_wait(&bar_acc_done, ti & 1, ab, kDkvWaitAcc);
       tc_fence_after();
-      if (tracer) trace_stamp(1 + wg, n, 1);
-      const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
-      if (CAUSAL && n < 2) dkv_step<true>(tS, tdP, nl, nl + 64, scale_log2, row - n * C::kStepRows);
-      else                 dkv_step<false>(tS, tdP, nl, nl + 64, scale_log2, 0);
-      if (tracer) trace_stamp(1 + wg, n, 5);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bar_tr_ready[wg]);
-      if (tracer) trace_stamp(1 + wg, n, 7);
-    }
-
-    mbar_wait(&bar_acc_done, 0, ab, kDkvWaitAcc);
-    tc_fence_after();
-    // staged in the TMA layout over the K and V tiles (no MMA reads them any more), then stored by TMA
-    for (int cc = wg; cc < D / 32; cc += NB) {
-      const int col = 32 * cc;
-      uint32_t a[32], b[32];
-      tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + col, a);
-      tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + col, b);
-      tmem_wait_ld();
-      uint8_t *vslab = sV + (cc >> 1) * C::kBigSlabBytes, *kslab = sK + (cc >> 1) * C::kBigSlabBytes;
+      uint8_t *stage_dk = C::kSepStaging ? sOut : sK, *stage_dv = C::kSepStaging ? sOut + C::kBigTileBytes : sV;
+      constexpr int kMaxCh = (D / 32 + NB - 1) / NB;       // epilogue chunks per warpgroup
+      uint32_t a[kMaxCh][32], b[kMaxCh][32];
 #pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        const uint32_t off = swz128_offset(row, 4 * (cc & 1) + v);
-        uint32_t vw[4], kw[4];
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const int i = 8 * v + 2 * w;
-          vw[w] = pack_bf16x2(__uint_as_float(a[i]), __uint_as_float(a[i + 1]));
-          kw[w] = pack_bf16x2(__fmul_rn(alpha, __uint_as_float(b[i])), __fmul_rn(alpha, __uint_as_float(b[i + 1])));
+      for (int nch = 0; nch < kMaxCh; ++nch) {
+        const int cc = wg + nch * NB;
+        if (cc < D / 32) {
+          tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + 32 * cc, a[nch]);
+          tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + 32 * cc, b[nch]);
         }
-        *reinterpret_cast<uint4 *>(vslab + off) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
-        *reinterpret_cast<uint4 *>(kslab + off) = make_uint4(kw[0], kw[1], kw[2], kw[3]);
       }
-    }
-    fence_proxy_async_smem();
-    named_bar_sync(1, 128 * NB);
-    if (threadIdx.x == 128) {
-      for (int sl = 0; sl < C::kSlabs; ++sl) {
-        tma_store_2d(&tmdV, sV + sl * C::kBigSlabBytes, sl * 64, krow0);
-        tma_store_2d(&tmdK, sK + sl * C::kBigSlabBytes, sl * 64, krow0);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(&bar_acc_free);          // the accumulators may be overwritten by the next tile
+      if (C::kSepStaging) {
+        if (threadIdx.x == 128) {
+          mbar_arrive(&bar_res_free);      // second arrival: with its own staging buffer the epilogue never touches K / V
+          bulk_wait_group_read0();         // the previous tile's stores have left the staging buffer
+        }
+        named_bar_sync(1, 128 * NB);
       }
-      bulk_commit_group();
-      bulk_wait_group_read0();
+      // staged in the TMA (128-byte swizzled) layout, then stored by TMA
+#pragma unroll
+      for (int nch = 0; nch < kMaxCh; ++nch) {
+        const int cc = wg + nch * NB;
+        if (cc >= D / 32) break;
+        const uint32_t slab = (cc >> 1) * C::kBigSlabBytes;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const uint32_t off = slab + swz128_offset(row, 4 * (cc & 1) + v);
+          uint32_t vw[4], kw[4];
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const int i = 8 * v + 2 * w;
+            vw[w] = pack_bf16x2(__uint_as_float(a[nch][i]), __uint_as_float(a[nch][i + 1]));
+            kw[w] = pack_bf16x2(__fmul_rn(alpha, __uint_as_float(b[nch][i])), __fmul_rn(alpha, __uint_as_float(b[nch][i + 1])));
+          }
+          *reinterpret_cast<uint4 *>(stage_dv + off) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
+          *reinterpret_cast<uint4 *>(stage_dk + off) = make_uint4(kw[0], kw[1], kw[2], kw[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      named_bar_sync(1, 128 * NB);
+      if (threadIdx.x == 128) {
+        for (int sl = 0; sl < C::kSlabs; ++sl) {
+          tma_store_2d(&tmdV, stage_dv + sl * C::kBigSlabBytes, sl * 64, krow0);
+          tma_store_2d(&tmdK, stage_dk + sl * C::kBigSlabBytes, sl * 64, krow0);
+        }
+        bulk_commit_group();
+        if (!C::kSepStaging) {             // staging shares the K / V tile: its reads must finish before the next load
+          bulk_wait_group_read0();
+          mbar_arrive(&bar_res_free);
+        }
+#ifdef GPROJ_TRACE
+        tile_trace(lin, tile_t0, global_ns());
+#endif
+      }
+      g0 += T;
     }
+    if (threadIdx.x == 128) bulk_wait_group_read0();
   }
 
   tc_fence_before();

@@ -26,6 +26,7 @@ struct DeviceState {
   bool ready = false;
   bool arch_ok = false;
   int *status_ptr = nullptr;
+  int sm_count = 0;
 };
 
 std::mutex g_mutex;
@@ -48,6 +49,8 @@ int device_state(DeviceState **out) {
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return GPROJ_ERR_CUDA;
     st.arch_ok = (major == 10);
+    if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || st.sm_count <= 0)
+      return GPROJ_ERR_CUDA;
     if (st.arch_ok) {
       if (!g_encode) {
         cudaDriverEntryPointQueryResult q;
@@ -177,18 +180,20 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
   if (!ok) return GPROJ_ERR_CUDA;
 
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
-  const dim3 grid(static_cast<unsigned>(BH * (N / 128)));
+  const int total_tiles = BH * (N / 128);
+  const dim3 grid(static_cast<unsigned>(total_tiles < st->sm_count ? total_tiles : st->sm_count));   // persistent: one CTA per SM
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16 *Ob = static_cast<const __nv_bfloat16 *>(O), *dOb = static_cast<const __nv_bfloat16 *>(dO);
 #define GPROJ_LAUNCH_BWD(DD, CC)                                                                                        \
   do {                                                                                                                  \
     if (run_dq)                                                                                                         \
       bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                               \
-          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, N, BH, scale_log2, softmax_scale, flags,         \
+          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, N, BH, total_tiles, scale_log2, softmax_scale, flags, \
           st->status_ptr);                                                                                              \
     if (run_dkv)                                                                                                        \
       bwd_dkv_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
-          mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, N, BH, scale_log2, softmax_scale, flags, st->status_ptr); \
+          mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, N, BH, total_tiles, scale_log2, softmax_scale, flags,       \
+          st->status_ptr);                                                                                              \
   } while (0)
   if (d == 64) { if (causal) GPROJ_LAUNCH_BWD(64, true); else GPROJ_LAUNCH_BWD(64, false); }
   else         { if (causal) GPROJ_LAUNCH_BWD(128, true); else GPROJ_LAUNCH_BWD(128, false); }
@@ -260,6 +265,18 @@ const char *gproj_status_string(int status) {
 int gproj_last_launch_count(void) { return tl_launch_count; }
 
 #ifdef GPROJ_TRACE
+// Debug builds only: per-tile timeline of the most recent launches (count, then {cta, tile, start ns, end ns} records).
+int gproj_debug_read_tile_trace(unsigned long long *out, int max_records, int reset) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return GPROJ_ERR_CUDA;
+  int n = 0;
+  if (cudaMemcpyFromSymbol(&n, gproj::g_tile_trace_count, sizeof(int)) != cudaSuccess) return GPROJ_ERR_CUDA;
+  if (n > gproj::kTileTraceMax) n = gproj::kTileTraceMax;
+  if (n > max_records) n = max_records;
+  if (n > 0 && cudaMemcpyFromSymbol(out, gproj::g_tile_trace, static_cast<size_t>(n) * 4 * sizeof(unsigned long long)) != cudaSuccess)
+    return GPROJ_ERR_CUDA;
+  if (reset) { const int zero = 0; cudaMemcpyToSymbol(gproj::g_tile_trace_count, &zero, sizeof(int)); }
+  return n;
+}
 // Debug builds only: copy the phase stamps of CTA 0 to the host (after a device synchronize).
 int gproj_debug_read_trace(long long *out, int count) {
   if (cudaDeviceSynchronize() != cudaSuccess) return GPROJ_ERR_CUDA;

@@ -29,6 +29,21 @@ __device__ long long g_trace[kTraceRoles * kTraceSteps * kTraceSlots];
 __device__ __forceinline__ void trace_stamp(int role, int step, int slot) {
   if (blockIdx.x == 0 && step < kTraceSteps) g_trace[(role * kTraceSteps + step) * kTraceSlots + slot] = clock64();
 }
+// per-tile timeline: {cta, tile, start ns, end ns} for every tile of a persistent launch
+constexpr int kTileTraceMax = 16384;
+__device__ unsigned long long g_tile_trace[kTileTraceMax * 4];
+__device__ int g_tile_trace_count;
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void tile_trace(int tile, unsigned long long t0, unsigned long long t1) {
+  const int i = atomicAdd(&g_tile_trace_count, 1);
+  if (i < kTileTraceMax) {
+    g_tile_trace[4 * i] = blockIdx.x; g_tile_trace[4 * i + 1] = tile; g_tile_trace[4 * i + 2] = t0; g_tile_trace[4 * i + 3] = t1;
+  }
+}
 #else
 __device__ __forceinline__ void trace_stamp(int, int, int) {}
 #endif

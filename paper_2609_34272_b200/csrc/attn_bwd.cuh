@@ -195,7 +195,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   uint8_t *sOut = sKV + S * C::kDqStageBytes;                  // staging (dQ tile, then Z tile) when separate
 
   __shared__ uint64_t bar_res_full[R], bar_res_free[R], bar_kv_full[S], bar_kv_empty[S];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free;
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
   __shared__ float s_rho[NB - 1][128], s_m[NB - 1][128], s_lam[128], s_D[128];
@@ -214,6 +214,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
     mbar_init(&bar_acc_free, 128 * NB);
+    mbar_init(&bar_drain[0], 1);
+    mbar_init(&bar_drain[1], 1);
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
@@ -311,6 +313,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         __syncwarp();
       }
     }
+    drain_mmas_if_aborted(&bar_drain[0], ab);
   } else if (warp == 2) {
     // ---------------------------------------------------------------- tensor-core issuer 2: A += t K, B += r K
     constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 queries] x [d], contraction over 64 keys
@@ -340,6 +343,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         __syncwarp();
       }
     }
+    drain_mmas_if_aborted(&bar_drain[1], ab);
   } else {
     // ---------------------------------------------------------------- compute: thread <-> query row
     const int wg = (warp - 4) >> 2;
@@ -500,7 +504,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   uint8_t *sOut = sStage + S * C::kDkvStageBytes;   // staging (dK tile, then dV tile) when separate
 
   __shared__ uint64_t bar_res_full, bar_res_free, bar_q_full[S], bar_q_empty[S];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free;
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -521,6 +525,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
     mbar_init(&bar_acc_free, 128 * NB);
+    mbar_init(&bar_drain[0], 1);
+    mbar_init(&bar_drain[1], 1);
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
@@ -612,6 +618,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         __syncwarp();
       }
     }
+    drain_mmas_if_aborted(&bar_drain[0], ab);
   } else if (warp == 2) {
     // ---------------------------------------------------------------- tensor-core issuer 2: dV += r^T dO, dK += t^T Q + r^T Z
     constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);     // [128 keys] x [d], contraction over 64 queries
@@ -660,6 +667,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         __syncwarp();
       }
     }
+    drain_mmas_if_aborted(&bar_drain[1], ab);
   } else {
     // ---------------------------------------------------------------- compute: thread <-> key row
     const int wg = (warp - 4) >> 2;

@@ -1,48 +1,64 @@
 // Fused attention forward for sm_100a: O = softmax(alpha Q K^T) V and the row log-sum-exp.
 //
-// One CTA owns a tile of 128 query rows of one (batch, head) and walks the key tiles.
-// Roles (warp-specialised, 192 threads):
-//   warp 0      TMA producer: Q tile once, then K_j / V_j tiles through a ring of stages
-//   warp 1      tensor-core issuer: S = Q K_j^T (FP32 in TMEM), then O += P~ V_j with the BF16
-//               probabilities read straight from TMEM; owns the TMEM allocation
-//   warps 2..5  softmax: thread <-> query row (TMEM lane), so every row statistic is a private
-//               register; online softmax on the UNSCALED logits with the subtract-before-scale
-//               rounding of Eq. "gproj-forward": z = exp2(fl32[ fl32(x - x_max) * (alpha log2 e) ]);
-//               l accumulates the FP32 z, the value product uses BF16(z).
-// The saved state is BF16 O and FP32 LSE = alpha x_max + ln l  (Algorithm 1, "Input").
+// A persistent CTA (one per SM) walks a static list of work items; one item = a PAIR of 128-row query tiles of
+// one (batch, head), processed against the key tiles they attend to.  Roles (384 threads):
+//   warp 0        TMA producer of the streamed K_j / V_j tiles (separate barriers: S needs only K, P~V only V)
+//   warp 1        tensor-core issuer 1: S_t = Q_t K_j^T for both query tiles (N = 128, FP32 in TMEM); owns TMEM
+//   warp 2        tensor-core issuer 2: O_t += P~_t V_j with the BF16 probabilities read straight from TMEM
+//   warp 3        TMA loader of the stationary Q pair
+//   warps 4..7    softmax warpgroup of query tile 0, warps 8..11 of query tile 1: thread <-> query row (TMEM lane),
+//                 so every row statistic is a private register.  While one warpgroup is in the ALUs the tensor
+//                 core works for the other one (the tensor-core queue is only 1-2 instructions deep, hence two
+//                 issuing warps: each one's barrier polls overlap the other's MMAs).
+// Softmax arithmetic: online softmax on the UNSCALED logits with the subtract-before-scale rounding of
+// Eq. "gproj-forward": z = exp2(fl32[ fl32(x - x_max) * (alpha log2 e) ]); l accumulates the FP32 z, the value
+// product uses BF16(z); the accumulator is rescaled whenever the running maximum of any row of the warp moved.
+// The saved state is BF16 O (staged in the TMA layout over the consumed Q tile, written by a TMA store) and
+// FP32 LSE = alpha x_max + ln l  (Algorithm 1, "Input").
+// TMEM: S_0, S_1 (128 columns each), O_0, O_1 (d each); at d = 64 the packed P~_t have their own 64 columns, so
+// S_t of the next key tile can be issued as soon as the softmax has read the current one; at d = 128 TMEM is full
+// and P~_t overwrites the first half of S_t.
 #pragma once
+#include "attn_bwd.cuh"   // TileSched
 #include "sm100_primitives.cuh"
 
 namespace gproj {
 
 template <int D>
 struct FwdCfg {
-  static constexpr int kBlockM = 128;
+  static constexpr int kBlockM = 128;                  // rows of one query tile (two per work item)
   static constexpr int kBlockN = 128;
-  static constexpr int kSlabs = D / 64;               // 64-column (128-byte) swizzle slabs per tile
+  static constexpr int kSlabs = D / 64;                // 64-column (128-byte) swizzle slabs per tile
   static constexpr int kSlabBytes = 128 * 128;         // 128 rows x 128 B
   static constexpr int kTileBytes = kSlabs * kSlabBytes;
-  static constexpr int kStages = (D == 64) ? 3 : 2;
-  static constexpr int kSmemBytes = kTileBytes * (1 + 2 * kStages) + 1024;
-  static constexpr int kTmemCols = 256;                // S: [0,128)  (P~ aliases its first 64)   O: [128,128+D)
-  static constexpr int kThreads = 192;
+  static constexpr int kStages = (D == 64) ? 4 : 2;    // ring of (K, V) tile pairs
+  static constexpr int kSmemBytes = 2 * kTileBytes + kStages * 2 * kTileBytes + 1024;
+  static constexpr int kTmemCols = 512;
+  static constexpr bool kSepP = (D == 64);             // P~ in its own TMEM columns
+  static constexpr uint32_t kColS = 0, kColO = 256, kColP = 256 + 2 * D;   // S_t at 128 t, O_t at 256 + D t, P_t at kColP + 64 t
+  static constexpr int kThreads = 384;
 };
 
-enum FwdWaitCode { kFwdWaitQ = 0x11, kFwdWaitKV = 0x12, kFwdWaitKVEmpty = 0x13, kFwdWaitS = 0x14, kFwdWaitP = 0x15, kFwdWaitO = 0x16 };
+enum FwdWaitCode {
+  kFwdWaitQ = 0x11, kFwdWaitK = 0x12, kFwdWaitV = 0x13, kFwdWaitKVEmpty = 0x14, kFwdWaitS = 0x15, kFwdWaitP = 0x16,
+  kFwdWaitPV = 0x17, kFwdWaitSFree = 0x18, kFwdWaitOFree = 0x19, kFwdWaitQFree = 0x1a
+};
 
 template <int D, bool CAUSAL>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV, __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE,
-                int N, int BH, float scale_log2, float alpha, int *status) {
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                float *__restrict__ LSE, int N, int BH, int tiles_per_item, int total_items, float scale_log2, float alpha,
+                int *status) {
   using C = FwdCfg<D>;
+  constexpr int S = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t *sQ = smem;
-  uint8_t *sK = sQ + C::kTileBytes;
-  uint8_t *sV = sK + C::kStages * C::kTileBytes;
+  uint8_t *sQ = smem;                              // tile 0, then tile 1 (each later reused to stage O_t)
+  uint8_t *sKV = sQ + 2 * C::kTileBytes;            // stage s: K tile, then V tile
 
-  __shared__ uint64_t bar_q, bar_kv_full[C::kStages], bar_kv_empty[C::kStages], bar_s_full, bar_p_ready, bar_o_done;
+  __shared__ uint64_t bar_q_full, bar_q_free, bar_k_full[S], bar_v_full[S], bar_kv_empty[S];
+  __shared__ uint64_t bar_s_full[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -50,170 +66,262 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
   __syncthreads();
   if (cta_skip != 0) return;   // an earlier wait gave up: drain the rest of the grid quickly
-  const int n_qt = N / C::kBlockM;
-  const int lin = blockIdx.x;
-  const int qt = CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH);   // causal: longest rows first
-  const int bh = lin % BH;
-  const int n_kv = CAUSAL ? qt + 1 : n_qt;
-  const int row0 = bh * N + qt * C::kBlockM;                      // first row of this tile in the [BH*N, d] view
 
+  const int n_qt = N / C::kBlockM;
+  const int TPI = tiles_per_item;                  // 2: a pair of query tiles per work item; 1: single tiles (small grids)
+  const int n_pairs = (n_qt + TPI - 1) / TPI;
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
-    mbar_init(&bar_q, 1);
-    for (int s = 0; s < C::kStages; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
-    mbar_init(&bar_s_full, 1);
-    mbar_init(&bar_p_ready, 128);
-    mbar_init(&bar_o_done, 1);
+    mbar_init(&bar_q_full, 1);
+    mbar_init(&bar_q_free, tiles_per_item);         // one arrival per query tile slot: its O store has left shared memory
+    for (int s = 0; s < S; ++s) { mbar_init(&bar_k_full[s], 1); mbar_init(&bar_v_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(&bar_drain[t], 1);
+      mbar_init(&bar_s_full[t], 1); mbar_init(&bar_p_ready[t], 128); mbar_init(&bar_pv_done[t], 1); mbar_init(&bar_o_free[t], 128);
+    }
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
-  if (warp == 0 && lane == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); }
+  if (warp == 0 && lane == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);   // shuffle marks it warp-uniform
-  const uint32_t tS = tmem_base, tO = tmem_base + 128;
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);   // the shuffle marks it warp-uniform
+
+  // Work items ordered by decreasing work (causal: last pair first).  Item -> (pair index, head).
+  TileSched sched(total_items);
+  auto item_pair = [&](int lin) { return CAUSAL ? (n_pairs - 1 - lin / BH) : (lin / BH); };
+  auto n_steps = [&](int pair) { return CAUSAL ? min(TPI * pair + TPI, n_qt) : n_qt; };   // key tiles walked by the item
+  // query tile t of the item takes part in key step j?
+  auto active = [&](int pair, int t, int j) { return t < TPI && (TPI * pair + t < n_qt) && (!CAUSAL || j <= TPI * pair + t); };
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producer of K_j, V_j
     if (lane == 0) {
-      mbar_expect_tx(&bar_q, C::kTileBytes);
-      for (int s = 0; s < C::kSlabs; ++s) tma_load_2d(sQ + s * C::kSlabBytes, &tmQ, &bar_q, s * 64, row0);
-      for (int j = 0; j < n_kv; ++j) {
-        const int st = j % C::kStages;
-        if (j >= C::kStages) mbar_wait(&bar_kv_empty[st], ((j / C::kStages) - 1) & 1, ab, kFwdWaitKVEmpty);
-        mbar_expect_tx(&bar_kv_full[st], 2 * C::kTileBytes);
-        const int krow = bh * N + j * C::kBlockN;
-        for (int s = 0; s < C::kSlabs; ++s) {
-          tma_load_2d(sK + st * C::kTileBytes + s * C::kSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow);
-          tma_load_2d(sV + st * C::kTileBytes + s * C::kSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow);
+      int g = 0;
+      for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
+        const int pair = item_pair(lin), bh = lin % BH, T = n_steps(pair);
+        for (int j = 0; j < T; ++j, ++g) {
+          const int st = g % S;
+          if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kFwdWaitKVEmpty);
+          uint8_t *dK = sKV + st * 2 * C::kTileBytes, *dV = dK + C::kTileBytes;
+          const int krow = bh * N + j * C::kBlockN;
+          mbar_expect_tx(&bar_k_full[st], C::kTileBytes);
+          for (int s = 0; s < C::kSlabs; ++s) tma_load_2d(dK + s * C::kSlabBytes, &tmK, &bar_k_full[st], s * 64, krow);
+          mbar_expect_tx(&bar_v_full[st], C::kTileBytes);
+          for (int s = 0; s < C::kSlabs; ++s) tma_load_2d(dV + s * C::kSlabBytes, &tmV, &bar_v_full[st], s * 64, krow);
         }
       }
-      // every load above is consumed by an MMA that the epilogue waits for, so nothing is in flight at exit
-      // unless the CTA aborted; then give the copies a bounded chance to land before shared memory is released.
+      // Every load is consumed by an MMA the epilogue waits for, so nothing is in flight at exit unless the
+      // CTA aborted; then give the copies a bounded chance to land before shared memory is released.
       if (cta_abort) {
-        for (int j = (n_kv > C::kStages ? n_kv - C::kStages : 0); j < n_kv; ++j) {
-          const int st = j % C::kStages;
-          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_kv_full[st], (j / C::kStages) & 1); ++spin) {}
+        for (int q = (g > S ? g - S : 0); q < g; ++q) {
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_k_full[q % S], (q / S) & 1); ++spin) {}
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_v_full[q % S], (q / S) & 1); ++spin) {}
         }
       }
+    }
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- TMA loader of the stationary Q pair
+    if (lane == 0) {
+      int ti = 0;
+      for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+        const int pair = item_pair(lin), bh = lin % BH;
+        const int tiles = (TPI == 2 && 2 * pair + 1 < n_qt) ? 2 : 1;
+        if (ti >= 1) mbar_wait(&bar_q_free, (ti - 1) & 1, ab, kFwdWaitQFree);
+        mbar_expect_tx(&bar_q_full, tiles * C::kTileBytes);
+        for (int t = 0; t < tiles; ++t)
+          for (int s = 0; s < C::kSlabs; ++s)
+            tma_load_2d(sQ + t * C::kTileBytes + s * C::kSlabBytes, &tmQ, &bar_q_full, s * 64, bh * N + (TPI * pair + t) * C::kBlockM);
+      }
+      if (cta_abort && ti > 0)
+        for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full, (ti - 1) & 1); ++spin) {}
     }
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- tensor-core issuer
+    // ---------------------------------------------------------------- tensor-core issuer 1: S_t = Q_t K_j^T
     // The whole warp runs this loop so that every address stays provably warp-uniform (descriptor operands
     // then live in uniform registers); one elected lane issues the MMAs and commits.
-    {
-      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);   // S = Q K^T, both operands K-major
-      constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, 0, 1);     // O += P V, V is MN-major (d contiguous)
-      const SmemDesc dscQ = make_smem_desc(smem_u32(sQ), 16, 1024);
-      const SmemDesc dscK0 = make_smem_desc(smem_u32(sK), 16, 1024);                  // K-major view of K stage 0
-      const SmemDesc dscV0 = make_smem_desc(smem_u32(sV), C::kSlabBytes, 1024);       // MN-major view of V stage 0
-      mbar_wait(&bar_q, 0, ab, kFwdWaitQ);
-      for (int j = 0; j < n_kv; ++j) {
-        const int st = j % C::kStages;
-        mbar_wait(&bar_kv_full[st], (j / C::kStages) & 1, ab, kFwdWaitKV);
-        tc_fence_after();
-        const SmemDesc dscK = dscK0.advanced(st * C::kTileBytes), dscV = dscV0.advanced(st * C::kTileBytes);
-        if (elect_one_sync()) {
+    constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);   // both operands K-major
+    const SmemDesc dscQ0 = make_smem_desc(smem_u32(sQ), 16, 1024);
+    const SmemDesc dscK0 = make_smem_desc(smem_u32(sKV), 16, 1024);
+    int g = 0, ti = 0, cnt[2] = {0, 0};
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int pair = item_pair(lin), T = n_steps(pair);
+      mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
+      for (int j = 0; j < T; ++j, ++g) {
+        const int st = g % S;
+        mbar_wait(&bar_k_full[st], (g / S) & 1, ab, kFwdWaitK);
+        const SmemDesc dscK = dscK0.advanced(st * 2 * C::kTileBytes);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k / 4) * C::kSlabBytes + (k % 4) * 32;
-            umma_ss(tS, dscQ.at(off), dscK.at(off), idesc_s, k > 0);
+        for (int t = 0; t < 2; ++t) {
+          if (!active(pair, t, j)) continue;
+          // S_t may be overwritten once its previous contents are dead: read by the softmax (P~ elsewhere), or,
+          // when P~ lives in the same columns, consumed by the previous P~V product.
+          if (cnt[t] > 0) {
+            if (C::kSepP) mbar_wait(&bar_p_ready[t], (cnt[t] - 1) & 1, ab, kFwdWaitSFree);
+            else          mbar_wait(&bar_pv_done[t], (cnt[t] - 1) & 1, ab, kFwdWaitSFree);
           }
-          umma_commit(&bar_s_full);
-        }
-        __syncwarp();
-        mbar_wait(&bar_p_ready, j & 1, ab, kFwdWaitP);
-        tc_fence_after();
-        const uint32_t acc = (j > 0) ? 1u : 0u;
-        if (elect_one_sync()) {
+          tc_fence_after();
+          const SmemDesc dscQ = dscQ0.advanced(t * C::kTileBytes);
+          if (elect_one_sync()) {
 #pragma unroll
-          for (int k = 0; k < C::kBlockN / 16; ++k) umma_ts(tO, tS + 8 * k, dscV.at(k * 2048), idesc_o, k > 0 ? 1u : acc);
-          umma_commit(&bar_kv_empty[st]);
+            for (int k = 0; k < D / 16; ++k) {
+              const uint32_t off = (k / 4) * C::kSlabBytes + (k % 4) * 32;
+              umma_ss(tmem_base + C::kColS + 128 * t, dscQ.at(off), dscK.at(off), idesc_s, k > 0);
+            }
+            umma_commit(&bar_s_full[t]);
+          }
+          __syncwarp();
+          ++cnt[t];
         }
+      }
+    }
+    drain_mmas_if_aborted(&bar_drain[0], ab);
+  } else if (warp == 2) {
+    // ---------------------------------------------------------------- tensor-core issuer 2: O_t += P~_t V_j
+    constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, 0, 1);     // V is MN-major (d contiguous)
+    const SmemDesc dscV0 = make_smem_desc(smem_u32(sKV + C::kTileBytes), C::kSlabBytes, 1024);
+    int g = 0, ti = 0, cnt[2] = {0, 0};
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int pair = item_pair(lin), T = n_steps(pair);
+      for (int j = 0; j < T; ++j, ++g) {
+        const int st = g % S;
+        mbar_wait(&bar_v_full[st], (g / S) & 1, ab, kFwdWaitV);
+        const SmemDesc dscV = dscV0.advanced(st * 2 * C::kTileBytes);
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (!active(pair, t, j)) continue;
+          if (j == 0 && ti > 0) mbar_wait(&bar_o_free[t], (ti - 1) & 1, ab, kFwdWaitOFree);   // previous epilogue has read O_t
+          mbar_wait(&bar_p_ready[t], cnt[t] & 1, ab, kFwdWaitP);
+          tc_fence_after();
+          const uint32_t tP = tmem_base + (C::kSepP ? C::kColP + 64 * t : C::kColS + 128 * t);
+          const uint32_t acc = (j > 0) ? 1u : 0u;
+          if (elect_one_sync()) {
+#pragma unroll
+            for (int k = 0; k < C::kBlockN / 16; ++k)
+              umma_ts(tmem_base + C::kColO + D * t, tP + 8 * k, dscV.at(k * 2048), idesc_o, k > 0 ? 1u : acc);
+            umma_commit(&bar_pv_done[t]);
+          }
+          __syncwarp();
+          ++cnt[t];
+        }
+        if (elect_one_sync()) umma_commit(&bar_kv_empty[st]);    // every MMA that reads this K / V stage has been issued
         __syncwarp();
       }
-      if (elect_one_sync())
-      umma_commit(&bar_o_done);
     }
+    drain_mmas_if_aborted(&bar_drain[1], ab);
   } else {
-    // ---------------------------------------------------------------- softmax: one thread per query row
+    // ---------------------------------------------------------------- softmax: warpgroup t <-> query tile t, thread <-> row
+    const int t = (warp - 4) >> 2;
     const int row = 32 * (warp & 3) + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
-    float m_run = -INFINITY, l_run = 0.f;
-    for (int j = 0; j < n_kv; ++j) {
-      mbar_wait(&bar_s_full, j & 1, ab, kFwdWaitS);
-      tc_fence_after();
-      uint32_t xr[4][32];
+    const uint32_t tS = tmem_base + C::kColS + 128 * t + lane_addr;
+    const uint32_t tO = tmem_base + C::kColO + D * t + lane_addr;
+    const uint32_t tP = tmem_base + (C::kSepP ? C::kColP + 64 * t : C::kColS + 128 * t) + lane_addr;
+    int ti = 0, cnt = 0;
+    // With single-tile items the second warpgroup has nothing to do for the whole launch (and bar_q_free expects one
+    // arrival per item only).
+    for (int lin = (t < TPI) ? sched.next() : -1; lin >= 0; lin = sched.next(), ++ti) {
+      const int pair = item_pair(lin), bh = lin % BH, T = n_steps(pair);
+      const int qt = TPI * pair + t;
+      if (qt >= n_qt) {
+        // Odd number of query tiles: the last pair has no second tile.  Stay in step with the item (its Q has landed)
+        // before handing back this slot, so that no barrier runs ahead of the roles that wait on it.
+        mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
+        if (row == 0) mbar_arrive(&bar_q_free);
+        mbar_arrive(&bar_o_free[t]);
+        continue;
+      }
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int j = 0; j < T; ++j) {
+        if (!active(pair, t, j)) continue;
+        mbar_wait(&bar_s_full[t], cnt & 1, ab, kFwdWaitS);
+        tc_fence_after();
+        uint32_t xr[4][32];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_addr + 32 * c, xr[c]);
-      tmem_wait_ld();
-      float mx = -INFINITY;
-      if (CAUSAL && j == n_kv - 1) {
+        for (int c = 0; c < 4; ++c) tmem_ld32(tS + 32 * c, xr[c]);
+        tmem_wait_ld();
+        if (CAUSAL && j == qt) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (32 * c + i > row) xr[c][i] = 0xff800000u;   // -inf: key beyond the diagonal
+        }
+        float mx = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (32 * c + i > row) xr[c][i] = 0xff800000u;   // -inf: key beyond the diagonal
-      }
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(xr[c][i]));
+        const float m_new = fmaxf(m_run, mx);
+        const float corr = fast_exp2(__fmul_rn(__fsub_rn(m_run, m_new), scale_log2));
+        // P~ of the previous key tile must have been consumed (and O_t updated) before either is touched
+        if (j > 0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
+        float rs = 0.f;
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(xr[c][i]));
-      const float m_new = fmaxf(m_run, mx);
-      const float corr = fast_exp2(__fmul_rn(__fsub_rn(m_run, m_new), scale_log2));
-      float rs = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float z0 = fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i]), m_new), scale_log2));
-          const float z1 = fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i + 1]), m_new), scale_log2));
-          rs += z0 + z1;
-          pk[i] = pack_bf16x2(z0, z1);
+          for (int i = 0; i < 16; ++i) {
+            const float z0 = fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i]), m_new), scale_log2));
+            const float z1 = fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i + 1]), m_new), scale_log2));
+            rs += z0 + z1;
+            pk[i] = pack_bf16x2(z0, z1);
+          }
+          tmem_st16(tP + 16 * c, pk);
         }
-        tmem_st16(tS + lane_addr + 16 * c, pk);   // P~ overwrites the S columns already consumed
+        l_run = l_run * corr + rs;
+        if (j > 0 && __any_sync(0xffffffffu, m_new != m_run)) {
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + 32 * c, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+            tmem_st32(tO + 32 * c, o);
+          }
+        }
+        m_run = m_new;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bar_p_ready[t]);
+        ++cnt;
       }
-      l_run = l_run * corr + rs;
-      // The accumulator may be rescaled now: bar_s_full also covers the previous P~ V product
-      // (a commit tracks every MMA issued before it).
-      if (j > 0 && __any_sync(0xffffffffu, m_new != m_run)) {
+      // ---- epilogue: O = BF16(acc / l) staged in the TMA layout over this tile's Q, LSE = alpha x_max + ln l
+      mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV);
+      tc_fence_after();
+      const float inv_l = 1.0f / l_run;
+      uint8_t *stage = sQ + t * C::kTileBytes;         // no MMA reads this Q tile any more
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tO + lane_addr + 32 * c, o);
-          tmem_wait_ld();
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tO + 32 * c, o);
+        tmem_wait_ld();
+        const uint32_t slab = (c >> 1) * C::kSlabBytes;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
-          tmem_st32(tO + lane_addr + 32 * c, o);
+        for (int v = 0; v < 4; ++v) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int w = 0; w < 4; ++w)
+            pk[w] = pack_bf16x2(__uint_as_float(o[8 * v + 2 * w]) * inv_l, __uint_as_float(o[8 * v + 2 * w + 1]) * inv_l);
+          *reinterpret_cast<uint4 *>(stage + slab + swz128_offset(row, 4 * (c & 1) + v)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
       }
-      m_run = m_new;
-      tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bar_p_ready);
+      mbar_arrive(&bar_o_free[t]);                     // O_t may be overwritten by the next work item
+      const int grow = bh * N + qt * C::kBlockM;
+      LSE[grow + row] = fmaf(m_run, alpha, logf(l_run));
+      fence_proxy_async_smem();
+      named_bar_sync(1 + t, 128);
+      if (row == 0) {
+        for (int sl = 0; sl < C::kSlabs; ++sl) tma_store_2d(&tmO, stage + sl * C::kSlabBytes, sl * 64, grow);
+        bulk_commit_group();
+        bulk_wait_group_read0();
+        mbar_arrive(&bar_q_free);                      // this tile's half of the Q buffer may be reloaded
+      }
     }
-    // ---- epilogue: O = BF16(acc / l), LSE = alpha x_max + ln l
-    mbar_wait(&bar_o_done, 0, ab, kFwdWaitO);
-    tc_fence_after();
-    const float inv_l = 1.0f / l_run;
-    __nv_bfloat16 *orow = O + static_cast<size_t>(row0 + row) * D;
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t o[32];
-      tmem_ld32(tO + lane_addr + 32 * c, o);
-      tmem_wait_ld();
-      uint32_t pk[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i)
-        pk[i] = pack_bf16x2(__uint_as_float(o[2 * i]) * inv_l, __uint_as_float(o[2 * i + 1]) * inv_l);
-      uint4 *dst = reinterpret_cast<uint4 *>(orow + 32 * c);
-#pragma unroll
-      for (int v = 0; v < 4; ++v) dst[v] = make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
-    }
-    LSE[row0 + row] = fmaf(m_run, alpha, logf(l_run));
   }
 
   tc_fence_before();

@@ -123,15 +123,20 @@ int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *
 
   const int BH = B * H;
   const uint64_t rows = static_cast<uint64_t>(BH) * N;
-  CUtensorMap mQ, mK, mV;
-  if (!make_map(&mQ, Q, rows, d, 128) || !make_map(&mK, K, rows, d, 128) || !make_map(&mV, V, rows, d, 128))
+  CUtensorMap mQ, mK, mV, mO;
+  if (!make_map(&mQ, Q, rows, d, 128) || !make_map(&mK, K, rows, d, 128) || !make_map(&mV, V, rows, d, 128) ||
+      !make_map(&mO, O, rows, d, 128))
     return GPROJ_ERR_CUDA;
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
-  const dim3 grid(static_cast<unsigned>(BH * (N / 128)));
+  // One work item = a pair of query tiles of one head (two softmax warpgroups ping-pong on the tensor core); when
+  // that leaves too few items to balance the SMs, items are single tiles.
+  const int n_qt = N / 128;
+  const int tiles_per_item = (static_cast<long long>(BH) * ((n_qt + 1) / 2) * 2 >= 3LL * st->sm_count) ? 2 : 1;
+  const int total_items = BH * ((n_qt + tiles_per_item - 1) / tiles_per_item);
+  const dim3 grid(static_cast<unsigned>(total_items < st->sm_count ? total_items : st->sm_count));   // persistent
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  __nv_bfloat16 *Ob = static_cast<__nv_bfloat16 *>(O);
-#define GPROJ_LAUNCH_FWD(DD, CC)                                                                              \
-  attn_fwd_kernel<DD, CC><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(mQ, mK, mV, Ob, LSE, N, BH, \
+#define GPROJ_LAUNCH_FWD(DD, CC)                                                                                    \
+  attn_fwd_kernel<DD, CC><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(mQ, mK, mV, mO, LSE, N, BH, tiles_per_item, total_items, \
                                                                                       scale_log2, softmax_scale, st->status_ptr)
   if (d == 64) { if (causal) GPROJ_LAUNCH_FWD(64, true); else GPROJ_LAUNCH_FWD(64, false); }
   else         { if (causal) GPROJ_LAUNCH_FWD(128, true); else GPROJ_LAUNCH_FWD(128, false); }

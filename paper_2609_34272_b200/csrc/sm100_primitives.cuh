@@ -238,6 +238,18 @@ __device__ __forceinline__ void umma_commit(uint64_t *bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// Called by a whole MMA-issuing warp when its loop is over.  In the normal flow every MMA has been waited for by a
+// consumer before the CTA frees TMEM.  If the CTA aborted (a bounded wait gave up and later waits fell through) MMAs
+// may still be executing: commit them to a spare barrier and give them a bounded time to finish before TMEM goes.
+__device__ __forceinline__ void drain_mmas_if_aborted(uint64_t *spare_bar, const AbortState &ab) {
+  if (*ab.cta_abort) {
+    if (elect_one_sync()) umma_commit(spare_bar);
+    __syncwarp();
+    for (int spin = 0; spin < 2000000 && !mbar_try_wait(spare_bar, 0); ++spin) {}
+  }
+  __syncwarp();
+}
+
 // ------------------------------------------------------------------------------------------
 // TMEM <-> registers.  Shape 32x32b: lane l of the warp owns TMEM lane (32*(warp%4) + l) and
 // receives / supplies one 32-bit word per column.  taddr = base + (lane << 16) + column.

@@ -85,6 +85,22 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
                    void *workspace, size_t workspace_bytes, unsigned flags, void *stream);
 
 /*
+ * Grouped-query variants: Q, O, dO, dQ have H query heads ([B][H][N][d], LSE [B][H][N]); K, V, dK, dV have Hkv heads
+ * ([B][Hkv][N][d]) with H a multiple of Hkv; query head h reads key / value head h / (H / Hkv).  Key and value
+ * gradients sum over the query heads that share a KV head (Section 3.1, text after Eq. "row-gradients"; Appendix
+ * "Rounding in the implemented key correction": grouped queries only enlarge the set of contributing query heads); the
+ * sum is taken in the FP32 accumulators, before the single final BF16 cast.  Everything else, including the workspace
+ * size (gproj_attn_bwd_workspace_bytes(B, H, N, d) with the QUERY head count), is as for the functions above, which are
+ * the case Hkv = H.  This is the paper's own layout (16 query / 4 KV heads, d = 64).
+ */
+int gproj_attn_fwd_gqa(const void *Q, const void *K, const void *V, void *O, float *LSE,
+                       int B, int H, int Hkv, int N, int d, float softmax_scale, int causal, void *stream);
+int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                       void *dQ, void *dK, void *dV,
+                       int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+                       void *workspace, size_t workspace_bytes, unsigned flags, void *stream);
+
+/*
  * Backward for callers that must not allocate device memory (the paper has no counterpart: this is a
  * convenience of this library).  Some hosts of this code cannot call cudaMalloc at the point where they
  * need a gradient: a plugin running inside another framework's memory pool, a real-time or safety-audited

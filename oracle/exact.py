@@ -86,29 +86,43 @@ def head_keys_f64(q, k, v, u, alpha, causal, LSE, MUA, keys):
 
 
 def attn_fwd_bwd_f64(Q, K, V, dO, alpha, causal, heads=None):
-    """Exact forward and VJP for ``[B, H, N, d]`` BF16-bit inputs.
+    """Exact forward and VJP for BF16-bit inputs Q, dO ``[B, H, N, d]`` and K, V ``[B, Hkv, N, d]`` (H % Hkv == 0).
 
-    ``heads`` optionally restricts the work to a list of flat (b*H + h) indices;
-    the returned arrays then have that many leading entries.  Returns a dict with
-    O, LSE, MUA, dQ, dK, dV (FP64, uncast).
+    Query head h reads key / value head h // (H // Hkv); dK and dV sum over the query heads that share a KV head
+    (Section 3.1, text after Eq. "row-gradients").  ``heads`` optionally restricts the work to a list of flat
+    (b*H + h) query-head indices (only for Hkv == H); the returned arrays then have that many leading entries.
+    Returns a dict with O, LSE, MUA, dQ ([.., H, ..]) and dK, dV ([.., Hkv, ..]) in FP64, uncast.
     """
     Q, K, V, dO = map(_u16, (Q, K, V, dO))
     B, H, N, d = Q.shape
-    flat = lambda x: x.reshape(B * H, N, d)
-    Qf, Kf, Vf, Uf = map(flat, (Q, K, V, dO))
+    Hkv = K.shape[1]
+    if K.shape != (B, Hkv, N, d) or V.shape != K.shape or dO.shape != Q.shape or H % Hkv != 0:
+        raise ValueError("shape mismatch")
+    G = H // Hkv
+    Qf, Uf = Q.reshape(B * H, N, d), dO.reshape(B * H, N, d)
+    Kf, Vf = K.reshape(B * Hkv, N, d), V.reshape(B * Hkv, N, d)
+    kv_of = lambda bh: (bh // H) * Hkv + (bh % H) // G
+    if heads is not None and G != 1:
+        raise ValueError("a head subset is only supported without grouped queries")
     idx = list(range(B * H)) if heads is None else list(heads)
     n = len(idx)
-    out = {"O": np.empty((n, N, d)), "LSE": np.empty((n, N)), "MUA": np.empty((n, N)),
-           "dQ": np.empty((n, N, d)), "dK": np.empty((n, N, d)), "dV": np.empty((n, N, d))}
+    out = {"O": np.empty((n, N, d)), "LSE": np.empty((n, N)), "MUA": np.empty((n, N)), "dQ": np.empty((n, N, d))}
+    nkv = B * Hkv if heads is None else n
+    out["dK"] = np.zeros((nkv, N, d)); out["dV"] = np.zeros((nkv, N, d))
     allrows = np.arange(N, dtype=np.int32)
     for t, bh in enumerate(idx):
-        O, LSE, MUA, dQ = head_rows_f64(Qf[bh], Kf[bh], Vf[bh], Uf[bh], alpha, causal, allrows)
-        dK, dV = head_keys_f64(Qf[bh], Kf[bh], Vf[bh], Uf[bh], alpha, causal, LSE, MUA, allrows)
-        out["O"][t], out["LSE"][t], out["MUA"][t] = O, LSE, MUA
-        out["dQ"][t], out["dK"][t], out["dV"][t] = dQ, dK, dV
+        kv = kv_of(bh)
+        O, LSE, MUA, dQ = head_rows_f64(Qf[bh], Kf[kv], Vf[kv], Uf[bh], alpha, causal, allrows)
+        dK, dV = head_keys_f64(Qf[bh], Kf[kv], Vf[kv], Uf[bh], alpha, causal, LSE, MUA, allrows)
+        out["O"][t], out["LSE"][t], out["MUA"][t], out["dQ"][t] = O, LSE, MUA, dQ
+        slot = kv if heads is None else t
+        out["dK"][slot] += dK
+        out["dV"][slot] += dV
     if heads is None:
-        for key in out:
+        for key in ("O", "LSE", "MUA", "dQ"):
             out[key] = out[key].reshape((B, H) + out[key].shape[1:])
+        for key in ("dK", "dV"):
+            out[key] = out[key].reshape((B, Hkv) + out[key].shape[1:])
     return out
 
 

@@ -20,7 +20,8 @@ FLAG_ONLY_DKV_PASS = 8
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
-EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_bwd_static_scratch",
+EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_fwd_gqa", "gproj_attn_bwd_gqa",
+           "gproj_attn_bwd_static_scratch",
            "gproj_last_device_status",
            "gproj_status_string", "gproj_last_launch_count")
 
@@ -48,6 +49,10 @@ def load():
         lib.gproj_attn_bwd_workspace_bytes.argtypes = [i, i, i, i]
         lib.gproj_attn_bwd.restype = i
         lib.gproj_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, sz, u, vp]
+        lib.gproj_attn_fwd_gqa.restype = i
+        lib.gproj_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+        lib.gproj_attn_bwd_gqa.restype = i
+        lib.gproj_attn_bwd_gqa.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, sz, u, vp]
         lib.gproj_attn_bwd_static_scratch.restype = i
         lib.gproj_attn_bwd_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, u, vp]
         lib.gproj_last_device_status.restype = i
@@ -71,6 +76,13 @@ def _check_bf16(name, t, shape=None):
         raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
 
 
+def _kv_heads(Q, K):
+    B, H, N, d = Q.shape
+    if K.dim() != 4 or K.shape[0] != B or K.shape[2] != N or K.shape[3] != d or H % K.shape[1] != 0:
+        raise ValueError(f"K/V shape {tuple(K.shape)} does not match Q {tuple(Q.shape)} (need [B, Hkv, N, d], H % Hkv == 0)")
+    return K.shape[1]
+
+
 def _stream(device):
     return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
 
@@ -80,28 +92,37 @@ def gproj_attn_bwd_workspace_bytes(B, H, N, d) -> int:
 
 
 def gproj_attn_fwd(Q, K, V, softmax_scale, causal, O=None, LSE=None):
-    """O, LSE = attention forward.  Q, K, V: CUDA bfloat16 [B, H, N, d]."""
+    """O, LSE = attention forward.  Q: CUDA bfloat16 [B, H, N, d]; K, V: [B, Hkv, N, d] with H a multiple of Hkv
+    (Hkv < H = grouped-query attention)."""
     _check_bf16("Q", Q)
     B, H, N, d = Q.shape
-    _check_bf16("K", K, Q.shape); _check_bf16("V", V, Q.shape)
+    _check_bf16("K", K); _check_bf16("V", V, K.shape)
+    Hkv = _kv_heads(Q, K)
     if O is None:
         O = torch.empty_like(Q)
     if LSE is None:
         LSE = torch.empty((B, H, N), dtype=torch.float32, device=Q.device)
     _check_bf16("O", O, Q.shape)
     with torch.cuda.device(Q.device):
-        rc = load().gproj_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
-                                   B, H, N, d, float(softmax_scale), int(bool(causal)), _stream(Q.device))
+        if Hkv == H:
+            rc = load().gproj_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
+                                       B, H, N, d, float(softmax_scale), int(bool(causal)), _stream(Q.device))
+        else:
+            rc = load().gproj_attn_fwd_gqa(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
+                                           B, H, Hkv, N, d, float(softmax_scale), int(bool(causal)), _stream(Q.device))
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_fwd")
     return O, LSE
 
 
 def gproj_attn_bwd(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, workspace=None, dQ=None, dK=None, dV=None):
-    """dQ, dK, dV = attention backward with the GProj correction (flags: FLAG_NO_*_CORRECTION)."""
+    """dQ, dK, dV = attention backward with the GProj correction (flags: FLAG_NO_*_CORRECTION).
+    K, V (and dK, dV) may have fewer heads than Q (grouped-query attention)."""
     _check_bf16("Q", Q)
     B, H, N, d = Q.shape
-    for name, t in (("K", K), ("V", V), ("O", O), ("dO", dO)):
+    _check_bf16("K", K); _check_bf16("V", V, K.shape)
+    Hkv = _kv_heads(Q, K)
+    for name, t in (("O", O), ("dO", dO)):
         _check_bf16(name, t, Q.shape)
     if not (LSE.is_cuda and LSE.dtype == torch.float32 and LSE.is_contiguous() and tuple(LSE.shape) == (B, H, N)):
         raise TypeError("LSE must be a contiguous CUDA float32 tensor [B, H, N]")
@@ -109,13 +130,19 @@ def gproj_attn_bwd(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, workspac
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device)
     dQ = torch.empty_like(Q) if dQ is None else dQ
-    dK = torch.empty_like(Q) if dK is None else dK
-    dV = torch.empty_like(Q) if dV is None else dV
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(K) if dV is None else dV
     with torch.cuda.device(Q.device):
-        rc = load().gproj_attn_bwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
-                                   dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, N, d, float(softmax_scale),
-                                   int(bool(causal)), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
-                                   int(flags), _stream(Q.device))
+        if Hkv == H:
+            rc = load().gproj_attn_bwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
+                                       dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, N, d, float(softmax_scale),
+                                       int(bool(causal)), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                       int(flags), _stream(Q.device))
+        else:
+            rc = load().gproj_attn_bwd_gqa(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
+                                           dO.data_ptr(), dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, Hkv, N, d,
+                                           float(softmax_scale), int(bool(causal)), workspace.data_ptr(),
+                                           workspace.numel() * workspace.element_size(), int(flags), _stream(Q.device))
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_bwd")
     return dQ, dK, dV

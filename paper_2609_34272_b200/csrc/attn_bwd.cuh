@@ -185,7 +185,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmZ,    // store, box 64 x 128 rows
               const __nv_bfloat16 *__restrict__ Og, const __nv_bfloat16 *__restrict__ dOg,
               const float *__restrict__ LSE, float *__restrict__ stats,
-              int N, int BH, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+              int N, int BH, int Hq, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
   constexpr int NB = C::kNB, R = C::kDqResBufs, S = C::kDqStages;
   extern __shared__ uint8_t smem_raw[];
@@ -244,7 +244,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kDqWaitKVEmpty);
           mbar_expect_tx(&bar_kv_full[st], C::kDqStageBytes);
           uint8_t *dst = sKV + st * C::kDqStageBytes;
-          const int krow = bh * N + n * C::kStepRows;
+          const int krow = kv_head_of(bh, Hq, G) * N + n * C::kStepRows;   // grouped-query: the group's shared K / V head
           for (int s = 0; s < C::kSlabs; ++s) {
             tma_load_2d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow);
             tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow);
@@ -493,7 +493,10 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmdK,   // store, box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmdV,   // store, box 64 x 128 rows
                const float *__restrict__ stats,
-               int N, int BH, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+               int N, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+  // BH counts (batch, KV head) pairs here.  With grouped queries (G > 1) one work item walks the query steps of all G
+  // query heads of its KV head, so their contributions are summed in the FP32 accumulators (Section 3.1: key and value
+  // contributions also sum over the query heads that share a KV head).
   using C = BwdCfg<D>;
   constexpr int NB = C::kNB, S = C::kDkvStages;
   extern __shared__ uint8_t smem_raw[];
@@ -550,12 +553,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
         const int kt = lin / BH, bh = lin % BH, T = tile_steps(kt), q_start = tile_q_start(kt);
-        for (int n = 0; n < T; ++n, ++g) {
+        const int q_head0 = (bh / Hkv) * (Hkv * G) + (bh % Hkv) * G;     // first query head of the group (flat index)
+        for (int n = 0; n < G * T; ++n, ++g) {
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_q_empty[st], ((g / S) - 1) & 1, ab, kDkvWaitQEmpty);
           mbar_expect_tx(&bar_q_full[st], stage_tx);
           uint8_t *dst = sStage + st * C::kDkvStageBytes;
-          const int qrow = bh * N + q_start + n * C::kStepRows;
+          const int qrow = (q_head0 + n / T) * N + q_start + (n % T) * C::kStepRows;
           for (int s = 0; s < C::kSlabs; ++s) {
             tma_load_2d(dst + s * C::kStepSlabBytes, &tmQ, &bar_q_full[st], s * 64, qrow);
             tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow);
@@ -592,7 +596,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);                       // K-major view of stage 0
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int T = tile_steps(lin / BH);
+      const int T = G * tile_steps(lin / BH);
       mbar_wait(&bar_res_full, ti & 1, ab, kDkvWaitKV);
       for (int n = 0; n < T; ++n, ++g) {
         const int st = g % S, b = g % NB;
@@ -626,7 +630,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     const SmemDesc dscQ0mn = make_smem_desc(smem_u32(sStage), C::kStepSlabBytes, 1024);    // MN-major view of stage 0
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int T = tile_steps(lin / BH);
+      const int T = G * tile_steps(lin / BH);
       if (ti > 0) mbar_wait(&bar_acc_free, (ti - 1) & 1, ab, kDkvWaitAccFree);   // the previous epilogue has read dV, dK
       for (int p = 0; p < T; ++p, ++g) {
         const int st = g % S, b = g % NB;
@@ -676,7 +680,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int kt = lin / BH, bh = lin % BH, T = tile_steps(kt);
+      const int kt = lin / BH, bh = lin % BH, Th = tile_steps(kt), T = G * Th;
       const int krow0 = bh * N + kt * 128;
 #ifdef GPROJ_TRACE
       const unsigned long long tile_t0 = global_ns();
@@ -687,7 +691,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         mbar_wait(&bar_sdp_full[wg], (g / NB) & 1, ab, kDkvWaitSdP);
         tc_fence_after();
         const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
-        if (CAUSAL && n < 2) dkv_step<true>(tS, tdP, nl, nl + 64, scale_log2, row - n * C::kStepRows);
+        if (CAUSAL && (n % Th) < 2) dkv_step<true>(tS, tdP, nl, nl + 64, scale_log2, row - (n % Th) * C::kStepRows);
         else                 dkv_step<false>(tS, tdP, nl, nl + 64, scale_log2, 0);
         tmem_wait_st();
         tc_fence_before();

@@ -48,7 +48,7 @@ template <int D, bool CAUSAL>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float *__restrict__ LSE, int N, int BH, int tiles_per_item, int total_items, float scale_log2, float alpha,
+                float *__restrict__ LSE, int N, int BH, int Hq, int G, int tiles_per_item, int total_items, float scale_log2, float alpha,
                 int *status) {
   using C = FwdCfg<D>;
   constexpr int S = C::kStages;
@@ -106,7 +106,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kFwdWaitKVEmpty);
           uint8_t *dK = sKV + st * 2 * C::kTileBytes, *dV = dK + C::kTileBytes;
-          const int krow = bh * N + j * C::kBlockN;
+          const int krow = kv_head_of(bh, Hq, G) * N + j * C::kBlockN;     // grouped-query: the group's shared K / V head
           mbar_expect_tx(&bar_k_full[st], C::kTileBytes);
           for (int s = 0; s < C::kSlabs; ++s) tma_load_2d(dK + s * C::kSlabBytes, &tmK, &bar_k_full[st], s * 64, krow);
           mbar_expect_tx(&bar_v_full[st], C::kTileBytes);

@@ -113,8 +113,15 @@ extern "C" {
 
 int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int N, int d,
                    float softmax_scale, int causal, void *stream) {
+  return gproj_attn_fwd_gqa(Q, K, V, O, LSE, B, H, H, N, d, softmax_scale, causal, stream);
+}
+
+int gproj_attn_fwd_gqa(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N,
+                       int d, float softmax_scale, int causal, void *stream) {
   if (!Q || !K || !V || !O || !LSE) return GPROJ_ERR_NULL;
   if (int rc = check_shape(B, H, N, d)) return rc;
+  if (Hkv <= 0 || H % Hkv != 0) return GPROJ_ERR_SHAPE;
+  const int G = H / Hkv;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || (reinterpret_cast<uintptr_t>(LSE) & 3u))
     return GPROJ_ERR_ALIGN;
   if (!std::isfinite(softmax_scale) || !(softmax_scale > 0.f)) return GPROJ_ERR_SCALE;
@@ -122,9 +129,9 @@ int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *
   if (int rc = device_state(&st)) return rc;
 
   const int BH = B * H;
-  const uint64_t rows = static_cast<uint64_t>(BH) * N;
+  const uint64_t rows = static_cast<uint64_t>(BH) * N, kv_rows = static_cast<uint64_t>(B) * Hkv * N;
   CUtensorMap mQ, mK, mV, mO;
-  if (!make_map(&mQ, Q, rows, d, 128) || !make_map(&mK, K, rows, d, 128) || !make_map(&mV, V, rows, d, 128) ||
+  if (!make_map(&mQ, Q, rows, d, 128) || !make_map(&mK, K, kv_rows, d, 128) || !make_map(&mV, V, kv_rows, d, 128) ||
       !make_map(&mO, O, rows, d, 128))
     return GPROJ_ERR_CUDA;
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
@@ -136,7 +143,7 @@ int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *
   const dim3 grid(static_cast<unsigned>(total_items < st->sm_count ? total_items : st->sm_count));   // persistent
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define GPROJ_LAUNCH_FWD(DD, CC)                                                                                    \
-  attn_fwd_kernel<DD, CC><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(mQ, mK, mV, mO, LSE, N, BH, tiles_per_item, total_items, \
+  attn_fwd_kernel<DD, CC><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(mQ, mK, mV, mO, LSE, N, BH, H, G, tiles_per_item, total_items, \
                                                                                       scale_log2, softmax_scale, st->status_ptr)
   if (d == 64) { if (causal) GPROJ_LAUNCH_FWD(64, true); else GPROJ_LAUNCH_FWD(64, false); }
   else         { if (causal) GPROJ_LAUNCH_FWD(128, true); else GPROJ_LAUNCH_FWD(128, false); }
@@ -155,8 +162,17 @@ size_t gproj_attn_bwd_workspace_bytes(int B, int H, int N, int d) {
 int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
                    void *dQ, void *dK, void *dV, int B, int H, int N, int d, float softmax_scale, int causal,
                    void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
+  return gproj_attn_bwd_gqa(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, H, N, d, softmax_scale, causal, workspace, workspace_bytes,
+                            flags, stream);
+}
+
+int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                       void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+                       void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
   if (!Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return GPROJ_ERR_NULL;
   if (int rc = check_shape(B, H, N, d)) return rc;
+  if (Hkv <= 0 || H % Hkv != 0) return GPROJ_ERR_SHAPE;
+  const int G = H / Hkv;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
       !aligned16(dK) || !aligned16(dV) || (reinterpret_cast<uintptr_t>(LSE) & 3u))
     return GPROJ_ERR_ALIGN;
@@ -171,33 +187,36 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
   DeviceState *st = nullptr;
   if (int rc = device_state(&st)) return rc;
 
-  const int BH = B * H;
-  const uint64_t rows = static_cast<uint64_t>(BH) * N;
+  const int BH = B * H, BHkv = B * Hkv;
+  const uint64_t rows = static_cast<uint64_t>(BH) * N, kv_rows = static_cast<uint64_t>(BHkv) * N;
   float *stats = static_cast<float *>(workspace);   // per 64-row block: 64 x {-LSE log2 e}, 64 x {-D}
   __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + align256(rows * sizeof(float2)));
 
   CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64, mdQst, mZst, mdKst, mdVst;
-  bool ok = make_map(&mQ128, Q, rows, d, 128) && make_map(&mdO128, dO, rows, d, 128) && make_map(&mK64, K, rows, d, 64) &&
-            make_map(&mV64, V, rows, d, 64) && make_map(&mK128, K, rows, d, 128) && make_map(&mV128, V, rows, d, 128) &&
+  bool ok = make_map(&mQ128, Q, rows, d, 128) && make_map(&mdO128, dO, rows, d, 128) && make_map(&mK64, K, kv_rows, d, 64) &&
+            make_map(&mV64, V, kv_rows, d, 64) && make_map(&mK128, K, kv_rows, d, 128) && make_map(&mV128, V, kv_rows, d, 128) &&
             make_map(&mQ64, Q, rows, d, 64) && make_map(&mdO64, dO, rows, d, 64) && make_map(&mZ64, Zneg, rows, d, 64) &&
-            make_map(&mdQst, dQ, rows, d, 128) && make_map(&mZst, Zneg, rows, d, 128) && make_map(&mdKst, dK, rows, d, 128) &&
-            make_map(&mdVst, dV, rows, d, 128);
+            make_map(&mdQst, dQ, rows, d, 128) && make_map(&mZst, Zneg, rows, d, 128) && make_map(&mdKst, dK, kv_rows, d, 128) &&
+            make_map(&mdVst, dV, kv_rows, d, 128);
   if (!ok) return GPROJ_ERR_CUDA;
 
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
-  const int total_tiles = BH * (N / 128);
+  const int total_tiles = BH * (N / 128), total_kv_tiles = BHkv * (N / 128);
   const dim3 grid(static_cast<unsigned>(total_tiles < st->sm_count ? total_tiles : st->sm_count));   // persistent: one CTA per SM
+  const dim3 grid_kv(static_cast<unsigned>(total_kv_tiles < st->sm_count ? total_kv_tiles : st->sm_count));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16 *Ob = static_cast<const __nv_bfloat16 *>(O), *dOb = static_cast<const __nv_bfloat16 *>(dO);
 #define GPROJ_LAUNCH_BWD(DD, CC)                                                                                        \
   do {                                                                                                                  \
     if (run_dq)                                                                                                         \
       bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                               \
-          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, N, BH, total_tiles, scale_log2, softmax_scale, flags, \
+          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, N, BH, H, G, total_tiles, scale_log2, softmax_scale,   \
+          flags,                                                                                                        \
           st->status_ptr);                                                                                              \
     if (run_dkv)                                                                                                        \
-      bwd_dkv_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
-          mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, N, BH, total_tiles, scale_log2, softmax_scale, flags,       \
+      bwd_dkv_kernel<DD, CC><<<grid_kv, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
+          mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,   \
+          flags,                                                                                                        \
           st->status_ptr);                                                                                              \
   } while (0)
   if (d == 64) { if (causal) GPROJ_LAUNCH_BWD(64, true); else GPROJ_LAUNCH_BWD(64, false); }

@@ -345,6 +345,10 @@ __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// Grouped-query layout: query head h of batch b (flat index b Hq + h) reads key / value head h / G of the same batch
+// (flat index b (Hq / G) + h / G).  G = 1 is ordinary multi-head attention.
+__device__ __forceinline__ int kv_head_of(int q_flat, int Hq, int G) { return (q_flat / Hq) * (Hq / G) + (q_flat % Hq) / G; }
+
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

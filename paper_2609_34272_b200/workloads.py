@@ -34,6 +34,11 @@ class Workload:
     q_offset: float = 0.0
     shared_offset: bool = False   # one offset vector for every head (workload 1)
     seed: int = BASE_SEED
+    Hkv: int = 0                  # key / value heads; 0 = same as H (no grouped queries)
+
+    @property
+    def kv_heads(self) -> int:
+        return self.Hkv if self.Hkv else self.H
 
     @property
     def softmax_scale(self) -> float:
@@ -55,6 +60,9 @@ WORKLOADS = {
     4: Workload("cfg4_noncausal_b4_h32_n8192_d128", 4, 32, 8192, 128, False, k_offset=16.0, q_offset=16.0,
                 seed=BASE_SEED + 4000),
     5: Workload("cfg5_causal_h8_n32768_d128", 1, 8, 32768, 128, True, k_offset=32.0, seed=BASE_SEED + 5000),
+    # Not one of the five benchmark configurations: the paper's own layout (16 query / 4 KV heads, d = 64, 4096 tokens,
+    # batch one; Appendix "Accuracy and Cost", "Captured inputs"), used by the grouped-query tests.
+    6: Workload("gqa_causal_h16_kv4_n4096_d64", 1, 16, 4096, 64, True, k_offset=16.0, seed=BASE_SEED + 6000, Hkv=4),
 }
 CFG3_OFFSET_NORMS = (0.0, 4.0, 16.0, 64.0)
 
@@ -74,16 +82,17 @@ def _offset(gen, B, H, d, norm, shared):
 
 
 def make_inputs(w: Workload):
-    """Returns dict of CPU torch.bfloat16 tensors Q, K, V, dO with shape [B,H,N,d]."""
+    """Returns dict of CPU torch.bfloat16 tensors Q, dO [B,H,N,d] and K, V [B,Hkv,N,d] (Hkv = H unless grouped)."""
     gen = torch.Generator(device="cpu")
     gen.manual_seed(w.seed)
     shape = (w.B, w.H, w.N, w.d)
+    kv_shape = (w.B, w.kv_heads, w.N, w.d)
     Q = torch.randn(shape, generator=gen, dtype=torch.float32)
-    K = torch.randn(shape, generator=gen, dtype=torch.float32)
-    V = torch.randn(shape, generator=gen, dtype=torch.float32)
+    K = torch.randn(kv_shape, generator=gen, dtype=torch.float32)
+    V = torch.randn(kv_shape, generator=gen, dtype=torch.float32)
     dO = torch.randn(shape, generator=gen, dtype=torch.float32)
     # Offset directions are always drawn (even for norm 0) so that variants share the base draw.
-    ck = _offset(gen, w.B, w.H, w.d, w.k_offset, w.shared_offset)
+    ck = _offset(gen, w.B, w.kv_heads, w.d, w.k_offset, w.shared_offset)
     cq = _offset(gen, w.B, w.H, w.d, w.q_offset, w.shared_offset)
     K = K + ck
     Q = Q + cq

@@ -174,6 +174,25 @@ def test_row_and_key_subsets_match_full():
     assert np.array_equal(dK, full["dK"][0, 0, rows]) and np.array_equal(dV, full["dV"][0, 0, rows])
 
 
+def test_grouped_queries_match_torch_autograd():
+    # Section 3.1: key and value contributions sum over the query heads that share a KV head.  Library reference:
+    # torch float64 autograd with the K / V heads repeated for their groups.
+    B, H, Hkv, N, d = 2, 6, 2, 33, 8
+    Q, dO = (randn_bf16((B, H, N, d), 300 + i) for i in range(2))
+    K, V = (randn_bf16((B, Hkv, N, d), 310 + i) for i in range(2))
+    alpha = 0.3
+    got = oracle.attn_fwd_bwd_f64(as_bits(Q), as_bits(K), as_bits(V), as_bits(dO), alpha, True)
+    q = Q.double().requires_grad_(True); k = K.double().requires_grad_(True); v = V.double().requires_grad_(True)
+    kk, vv = k.repeat_interleave(H // Hkv, dim=1), v.repeat_interleave(H // Hkv, dim=1)
+    s = alpha * q @ kk.transpose(-1, -2)
+    s = s.masked_fill(~torch.tril(torch.ones(N, N, dtype=torch.bool)), float("-inf"))
+    o = torch.softmax(s, dim=-1) @ vv
+    (o * dO.double()).sum().backward()
+    assert got["dK"].shape == (B, Hkv, N, d)
+    for name, ref in (("O", o.detach()), ("dQ", q.grad), ("dK", k.grad), ("dV", v.grad)):
+        assert np.abs(got[name] - ref.numpy()).max() <= 1e-12 * max(1.0, ref.abs().max().item()), name
+
+
 def test_rel_l2_metric():
     # 100 ||G^ - G|| / ||G||  (Appendix "Accuracy and Cost", "Reference and metric").
     g = np.array([3.0, 4.0]); gh = np.array([3.0, 4.5])

@@ -131,6 +131,14 @@ int gproj_attn_bwd_static_scratch(const void *Q, const void *K, const void *V, c
  */
 int gproj_last_device_status(void *stream, int *detail);
 
+/*
+ * Failure-detection self-test (no counterpart in the paper): enqueues a one-warp kernel whose only wait can never be
+ * satisfied.  The wait gives up after its budget (a fraction of a second), so a following gproj_last_device_status()
+ * returns GPROJ_ERR_TIMEOUT with detail 0x7e01, and clears it.  Nothing faults, traps or hangs; the context stays usable.
+ * Until the status is read and cleared, kernels launched by this library on the device return early without working.
+ */
+int gproj_selftest_wait_timeout(void *stream);
+
 /* Static, human-readable name of a status code. */
 const char *gproj_status_string(int status);
 

@@ -15,5 +15,6 @@ from .binding import (  # noqa: F401
     gproj_attn_fwd,
     gproj_last_device_status,
     gproj_last_launch_count,
+    gproj_selftest_wait_timeout,
     status_string,
 )

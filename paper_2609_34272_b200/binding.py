@@ -22,7 +22,7 @@ STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_fwd_gqa", "gproj_attn_bwd_gqa",
            "gproj_attn_bwd_static_scratch",
-           "gproj_last_device_status",
+           "gproj_last_device_status", "gproj_selftest_wait_timeout",
            "gproj_status_string", "gproj_last_launch_count")
 
 _lib = None
@@ -55,6 +55,8 @@ def load():
         lib.gproj_attn_bwd_gqa.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, sz, u, vp]
         lib.gproj_attn_bwd_static_scratch.restype = i
         lib.gproj_attn_bwd_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, u, vp]
+        lib.gproj_selftest_wait_timeout.restype = i
+        lib.gproj_selftest_wait_timeout.argtypes = [vp]
         lib.gproj_last_device_status.restype = i
         lib.gproj_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
         lib.gproj_status_string.restype = ctypes.c_char_p
@@ -181,6 +183,15 @@ def gproj_last_device_status(device=None):
     with torch.cuda.device(device):
         rc = load().gproj_last_device_status(_stream(device), ctypes.byref(detail))
     return rc, detail.value
+
+
+def gproj_selftest_wait_timeout(device=None):
+    """Enqueue the bounded-wait self-test kernel (its wait can never be satisfied; see the header)."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    with torch.cuda.device(device):
+        rc = load().gproj_selftest_wait_timeout(_stream(device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_selftest_wait_timeout")
 
 
 def gproj_last_launch_count() -> int:

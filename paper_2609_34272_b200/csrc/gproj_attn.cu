@@ -16,6 +16,18 @@ using namespace gproj;
 // Launch-status word: written by a kernel whose bounded wait gave up, read back on request.
 __device__ int g_device_status;
 
+// Self-test of the bounded-wait machinery: one warp waits on an mbarrier that nothing will ever arrive on.  The wait
+// gives up after its cycle budget, records its code in the status word and the kernel returns normally.
+__global__ void wait_timeout_selftest_kernel(int *status) {
+  __shared__ uint64_t bar;
+  __shared__ int cta_abort;
+  if (threadIdx.x == 0) { cta_abort = 0; mbar_init(&bar, 1); fence_mbar_init(); }
+  __syncthreads();
+  AbortState ab{status, &cta_abort};
+  mbar_wait(&bar, 0, ab, 0x7e);
+  __syncthreads();
+}
+
 constexpr int kMaxDevices = 64;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -268,6 +280,13 @@ int gproj_last_device_status(void *stream, int *detail) {
     return GPROJ_ERR_TIMEOUT;
   }
   return GPROJ_OK;
+}
+
+int gproj_selftest_wait_timeout(void *stream) {
+  DeviceState *st = nullptr;
+  if (int rc = device_state(&st)) return rc;
+  wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(st->status_ptr);
+  return cudaGetLastError() == cudaSuccess ? GPROJ_OK : GPROJ_ERR_CUDA;
 }
 
 const char *gproj_status_string(int status) {

@@ -101,6 +101,18 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
                        void *workspace, size_t workspace_bytes, unsigned flags, void *stream);
 
 /*
+ * Forward with options (fwd_flags = 0 is gproj_attn_fwd_gqa).  GPROJ_FWD_FLAG_FMA_SOFTMAX selects the native fused form
+ * of the softmax exponent, z = exp2(fma(x, a, -fl32(x_max a))) with a = softmax_scale * log2 e (Eq. "historical-fma",
+ * Appendix "The source of the saved-output error"): x a is not rounded on its own, so the largest score of a row need
+ * not map to exactly zero and a one-key row can return o_0 != v_0.  It exists to reproduce the paper's "FA3" forward
+ * next to the subtract-before-scale one on the same kernels; training code should leave it off.
+ */
+#define GPROJ_FWD_FLAG_FMA_SOFTMAX 1u
+int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, float *LSE,
+                      int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+                      unsigned fwd_flags, void *stream);
+
+/*
  * Backward for callers that must not allocate device memory (the paper has no counterpart: this is a
  * convenience of this library).  Some hosts of this code cannot call cudaMalloc at the point where they
  * need a gradient: a plugin running inside another framework's memory pool, a real-time or safety-audited

@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     FLAG_NO_Q_CORRECTION,
     FLAG_ONLY_DKV_PASS,
     FLAG_ONLY_DQ_PASS,
+    FWD_FLAG_FMA_SOFTMAX,
     GprojError,
     gproj_attn_bwd,
     gproj_attn_bwd_static_scratch,

@@ -17,10 +17,11 @@ FLAG_NO_Q_CORRECTION = 1
 FLAG_NO_K_CORRECTION = 2
 FLAG_ONLY_DQ_PASS = 4
 FLAG_ONLY_DKV_PASS = 8
+FWD_FLAG_FMA_SOFTMAX = 1
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
-EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_fwd_gqa", "gproj_attn_bwd_gqa",
+EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_fwd_gqa", "gproj_attn_bwd_gqa", "gproj_attn_fwd_ex",
            "gproj_attn_bwd_static_scratch",
            "gproj_last_device_status", "gproj_selftest_wait_timeout",
            "gproj_status_string", "gproj_last_launch_count")
@@ -51,6 +52,8 @@ def load():
         lib.gproj_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, sz, u, vp]
         lib.gproj_attn_fwd_gqa.restype = i
         lib.gproj_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+        lib.gproj_attn_fwd_ex.restype = i
+        lib.gproj_attn_fwd_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, i, u, vp]
         lib.gproj_attn_bwd_gqa.restype = i
         lib.gproj_attn_bwd_gqa.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, sz, u, vp]
         lib.gproj_attn_bwd_static_scratch.restype = i
@@ -93,7 +96,7 @@ def gproj_attn_bwd_workspace_bytes(B, H, N, d) -> int:
     return int(load().gproj_attn_bwd_workspace_bytes(B, H, N, d))
 
 
-def gproj_attn_fwd(Q, K, V, softmax_scale, causal, O=None, LSE=None):
+def gproj_attn_fwd(Q, K, V, softmax_scale, causal, O=None, LSE=None, fwd_flags=0):
     """O, LSE = attention forward.  Q: CUDA bfloat16 [B, H, N, d]; K, V: [B, Hkv, N, d] with H a multiple of Hkv
     (Hkv < H = grouped-query attention)."""
     _check_bf16("Q", Q)
@@ -106,7 +109,10 @@ def gproj_attn_fwd(Q, K, V, softmax_scale, causal, O=None, LSE=None):
         LSE = torch.empty((B, H, N), dtype=torch.float32, device=Q.device)
     _check_bf16("O", O, Q.shape)
     with torch.cuda.device(Q.device):
-        if Hkv == H:
+        if fwd_flags:
+            rc = load().gproj_attn_fwd_ex(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), B, H, Hkv, N, d,
+                                          float(softmax_scale), int(bool(causal)), int(fwd_flags), _stream(Q.device))
+        elif Hkv == H:
             rc = load().gproj_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
                                        B, H, N, d, float(softmax_scale), int(bool(causal)), _stream(Q.device))
         else:

@@ -10,7 +10,8 @@
 //                 so every row statistic is a private register.  While one warpgroup is in the ALUs the tensor
 //                 core works for the other one (the tensor-core queue is only 1-2 instructions deep, hence two
 //                 issuing warps: each one's barrier polls overlap the other's MMAs).
-// Softmax arithmetic: online softmax on the UNSCALED logits with the subtract-before-scale rounding of
+// Softmax arithmetic (FMA_SOFTMAX = false, the default): online softmax on the UNSCALED logits with the
+// subtract-before-scale rounding of
 // Eq. "gproj-forward": z = exp2(fl32[ fl32(x - x_max) * (alpha log2 e) ]); l accumulates the FP32 z, the value
 // product uses BF16(z); the accumulator is rescaled whenever the running maximum of any row of the warp moved.
 // The saved state is BF16 O (staged in the TMA layout over the consumed Q tile, written by a TMA store) and
@@ -44,7 +45,7 @@ enum FwdWaitCode {
   kFwdWaitPV = 0x17, kFwdWaitSFree = 0x18, kFwdWaitOFree = 0x19, kFwdWaitQFree = 0x1a
 };
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool FMA_SOFTMAX>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -256,6 +257,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(xr[c][i]));
         const float m_new = fmaxf(m_run, mx);
         const float corr = fast_exp2(__fmul_rn(__fsub_rn(m_run, m_new), scale_log2));
+        // FMA_SOFTMAX reproduces the native fused form of Eq. "historical-fma": z = exp2(fma(x, a, -fl32(x_max a))),
+        // in which x a is not rounded separately, so the largest score need not map to exactly zero.
+        const float m_scaled = __fmul_rn(m_new, scale_log2);
         // P~ of the previous key tile must have been consumed (and O_t updated) before either is touched
         if (j > 0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
         float rs = 0.f;
@@ -264,8 +268,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float z0 = fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i]), m_new), scale_log2));
-            const float z1 = fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i + 1]), m_new), scale_log2));
+            const float z0 = FMA_SOFTMAX ? fast_exp2(fmaf(__uint_as_float(xr[c][2 * i]), scale_log2, -m_scaled))
+                                         : fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i]), m_new), scale_log2));
+            const float z1 = FMA_SOFTMAX ? fast_exp2(fmaf(__uint_as_float(xr[c][2 * i + 1]), scale_log2, -m_scaled))
+                                         : fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i + 1]), m_new), scale_log2));
             rs += z0 + z1;
             pk[i] = pack_bf16x2(z0, z1);
           }

@@ -74,10 +74,14 @@ int device_state(DeviceState **out) {
       if (cudaGetSymbolAddress(reinterpret_cast<void **>(&st.status_ptr), g_device_status) != cudaSuccess)
         return GPROJ_ERR_CUDA;
       bool ok = true;
-      ok &= allow_smem(attn_fwd_kernel<64, true>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<64, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, true>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, true>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, true>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, false>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<128, true>, BwdCfg<128>::kDqSmemBytes) == cudaSuccess;
@@ -130,7 +134,14 @@ int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *
 
 int gproj_attn_fwd_gqa(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N,
                        int d, float softmax_scale, int causal, void *stream) {
+  return gproj_attn_fwd_ex(Q, K, V, O, LSE, B, H, Hkv, N, d, softmax_scale, causal, 0u, stream);
+}
+
+int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N,
+                      int d, float softmax_scale, int causal, unsigned fwd_flags, void *stream) {
   if (!Q || !K || !V || !O || !LSE) return GPROJ_ERR_NULL;
+  if (fwd_flags & ~GPROJ_FWD_FLAG_FMA_SOFTMAX) return GPROJ_ERR_FLAGS;
+  const bool fma = (fwd_flags & GPROJ_FWD_FLAG_FMA_SOFTMAX) != 0;
   if (int rc = check_shape(B, H, N, d)) return rc;
   if (Hkv <= 0 || H % Hkv != 0) return GPROJ_ERR_SHAPE;
   const int G = H / Hkv;
@@ -154,11 +165,14 @@ int gproj_attn_fwd_gqa(const void *Q, const void *K, const void *V, void *O, flo
   const int total_items = BH * ((n_qt + tiles_per_item - 1) / tiles_per_item);
   const dim3 grid(static_cast<unsigned>(total_items < st->sm_count ? total_items : st->sm_count));   // persistent
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define GPROJ_LAUNCH_FWD(DD, CC)                                                                                    \
-  attn_fwd_kernel<DD, CC><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(mQ, mK, mV, mO, LSE, N, BH, H, G, tiles_per_item, total_items, \
-                                                                                      scale_log2, softmax_scale, st->status_ptr)
-  if (d == 64) { if (causal) GPROJ_LAUNCH_FWD(64, true); else GPROJ_LAUNCH_FWD(64, false); }
-  else         { if (causal) GPROJ_LAUNCH_FWD(128, true); else GPROJ_LAUNCH_FWD(128, false); }
+#define GPROJ_LAUNCH_FWD(DD, CC, FF)                                                                                \
+  attn_fwd_kernel<DD, CC, FF><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(                             \
+      mQ, mK, mV, mO, LSE, N, BH, H, G, tiles_per_item, total_items, scale_log2, softmax_scale, st->status_ptr)
+#define GPROJ_LAUNCH_FWD_C(DD, FF)                                                                                  \
+  do { if (causal) GPROJ_LAUNCH_FWD(DD, true, FF); else GPROJ_LAUNCH_FWD(DD, false, FF); } while (0)
+  if (d == 64) { if (fma) GPROJ_LAUNCH_FWD_C(64, true); else GPROJ_LAUNCH_FWD_C(64, false); }
+  else         { if (fma) GPROJ_LAUNCH_FWD_C(128, true); else GPROJ_LAUNCH_FWD_C(128, false); }
+#undef GPROJ_LAUNCH_FWD_C
 #undef GPROJ_LAUNCH_FWD
   if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
   tl_launch_count = 1;

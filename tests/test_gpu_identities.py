@@ -171,3 +171,43 @@ def test_sharp_attention_far_keys_stress():
     print("stress: corrected", e_on, "uncorrected", e_off)
     assert all(v <= 1.0 for v in e_on.values()), e_on
     assert e_off["dQ"] > 20.0 and e_off["dQ"] > 50 * e_on["dQ"]
+
+
+def test_fma_softmax_breaks_the_one_key_identity_and_sbs_restores_it():
+    # Appendix "The source of the saved-output error" / "Prescribed FMA cases": all 64 query coordinates equal c 2^k, all
+    # key coordinates equal one, so every dot product is known exactly; the first causal row has a single key.  With the
+    # fused exponent r = fma(x, a, -fl32(x a)) the row's own score does not map to zero, z = 2^r != 1, and the output is
+    # v_0 BF16(z) / z instead of v_0.  Subtract-before-scale restores o_0 = v_0 in every case; GProj keeps dq_0 = 0.
+    N, d, alpha = 128, 64, 0.125
+    a32 = np.float32(np.float64(np.float32(alpha)) * 1.4426950408889634)
+    gen = torch.Generator().manual_seed(9)
+    V = torch.randn(1, 1, N, d, generator=gen).to(torch.bfloat16)
+    dO = torch.randn(1, 1, N, d, generator=gen).to(torch.bfloat16)
+    K = torch.ones(1, 1, N, d, dtype=torch.bfloat16)
+    violations = 0
+    for c in (3, 5, 7):
+        for k in range(16):
+            Q = torch.full((1, 1, N, d), float(c * 2 ** k), dtype=torch.bfloat16)
+            x = np.float64(64.0 * c * 2 ** k)                                   # exact logit of every (row, key) pair
+            r = np.float32(np.float64(x) * np.float64(a32) - np.float64(np.float32(np.float32(x) * a32)))   # fma residue
+            z = 2.0 ** np.float64(r)
+            Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+            O_sbs, LSE = g.gproj_attn_fwd(Qd, Kd, Vd, alpha, True)
+            O_fma, LSE_f = g.gproj_attn_fwd(Qd, Kd, Vd, alpha, True, fwd_flags=g.FWD_FLAG_FMA_SOFTMAX)
+            assert torch.equal(O_sbs[0, 0, 0].cpu(), V[0, 0, 0]), (c, k)       # identity holds with subtract-before-scale
+            v0 = V[0, 0, 0].double().numpy()
+            zb = float(torch.tensor(z, dtype=torch.float32).to(torch.bfloat16))
+            model = v0 * zb / z                                                # scalar model of the fused form
+            got = O_fma[0, 0, 0].double().cpu().numpy()
+            assert np.all(np.abs(got - model) <= 2.0 ** -7 * np.abs(model) + 1e-30), (c, k, r)
+            if r == 0.0:
+                assert torch.equal(O_fma[0, 0, 0].cpu(), V[0, 0, 0]), (c, k)
+            elif not torch.equal(O_fma[0, 0, 0].cpu(), V[0, 0, 0]):
+                violations += 1
+                # the backward on this saved state: exact dq_0 is zero; GProj returns exactly zero, the plain backward not
+                dQ, _, _ = g.gproj_attn_bwd(Qd, Kd, Vd, O_fma, LSE_f, dO.cuda(), alpha, True)
+                assert torch.all(dQ[0, 0, 0] == 0), (c, k)
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, hex(detail)
+    print("one-key violations with the fused exponent:", violations, "of 48")
+    assert violations >= 3

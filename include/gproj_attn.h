@@ -7,8 +7,9 @@
  *     layout [B][H][N][d] contiguous with d fastest; base addresses 16-byte aligned.
  *   - LSE is a DEVICE pointer to FP32 [B][H][N]: the natural-log sum-exp of the scaled scores
  *     s_ij = softmax_scale * q_i . k_j over the row's support.
- *   - Supported shapes: d in {64, 128}; N a positive multiple of 128; B, H >= 1; one H for
- *     queries and keys (no grouped heads); N_q = N_k = N; causal != 0 means row i attends to j <= i.
+ *   - Supported shapes: d in {64, 128}; any N >= 1 (tiles of 128 rows; a ragged last tile is zero-filled on load,
+ *     masked where it would enter a row statistic and clipped on store); B, H >= 1 with B*H*N < 2^31; N_q = N_k = N;
+ *     causal != 0 means row i attends to j <= i.  The *_gqa entry points take separate query / KV head counts.
  *   - The caller owns all memory.  The library never allocates, frees or synchronises; work is
  *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).
  *   - Return value: GPROJ_OK (0) or a negative gproj_status.  Nothing throws, aborts or traps.
@@ -29,7 +30,7 @@ extern "C" {
 typedef enum gproj_status {
   GPROJ_OK = 0,
   GPROJ_ERR_NULL = -1,      /* a required pointer is NULL */
-  GPROJ_ERR_SHAPE = -2,     /* unsupported d, N not a multiple of 128, non-positive dimension, size overflow */
+  GPROJ_ERR_SHAPE = -2,     /* unsupported d, non-positive dimension, H not a multiple of Hkv, size overflow */
   GPROJ_ERR_ALIGN = -3,     /* a tensor base address is not 16-byte aligned */
   GPROJ_ERR_WORKSPACE = -4, /* workspace NULL, misaligned or smaller than gproj_attn_bwd_workspace_bytes() */
   GPROJ_ERR_SCALE = -5,     /* softmax_scale not finite or not > 0 */

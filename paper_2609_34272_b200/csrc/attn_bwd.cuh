@@ -205,7 +205,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   __syncthreads();
   if (cta_skip != 0) return;   // an earlier wait gave up: drain the rest of the grid quickly
 
-  const int n_qt = N / 128;
+  // Ragged N: tiles and steps round up; rows past N load as zero (TMA fill) and are clipped on store.
+  const int n_qt = (N + 127) / 128, n64 = (N + C::kStepRows - 1) / C::kStepRows;
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
@@ -231,7 +232,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   TileSched sched(total_tiles);
   // tile decode: causal -> longest rows first
   auto tile_qt = [&](int lin) { return CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH); };
-  auto tile_steps = [&](int qt) { return CAUSAL ? 2 * (qt + 1) : N / C::kStepRows; };
+  auto tile_steps = [&](int qt) { return CAUSAL ? min(2 * (qt + 1), n64) : n64; };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (K, V) step tiles
@@ -244,10 +245,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kDqWaitKVEmpty);
           mbar_expect_tx(&bar_kv_full[st], C::kDqStageBytes);
           uint8_t *dst = sKV + st * C::kDqStageBytes;
-          const int krow = kv_head_of(bh, Hq, G) * N + n * C::kStepRows;   // grouped-query: the group's shared K / V head
+          const int kvh = kv_head_of(bh, Hq, G), krow = n * C::kStepRows;   // grouped-query: the group's shared K / V head
           for (int s = 0; s < C::kSlabs; ++s) {
-            tma_load_2d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow);
-            tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow);
+            tma_load_3d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow, kvh);
+            tma_load_3d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow, kvh);
           }
         }
       }
@@ -263,13 +264,13 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int rb = ti % R, row0 = (lin % BH) * N + tile_qt(lin) * 128;
+        const int rb = ti % R, bh = lin % BH, qrow0 = tile_qt(lin) * 128;
         if (ti >= R) mbar_wait(&bar_res_free[rb], ((ti / R) - 1) & 1, ab, kDqWaitResFree);
         mbar_expect_tx(&bar_res_full[rb], 2 * C::kBigTileBytes);
         uint8_t *dst = sRes + rb * 2 * C::kBigTileBytes;
         for (int s = 0; s < C::kSlabs; ++s) {
-          tma_load_2d(dst + s * C::kBigSlabBytes, &tmQ, &bar_res_full[rb], s * 64, row0);
-          tma_load_2d(dst + C::kBigTileBytes + s * C::kBigSlabBytes, &tmdO, &bar_res_full[rb], s * 64, row0);
+          tma_load_3d(dst + s * C::kBigSlabBytes, &tmQ, &bar_res_full[rb], s * 64, qrow0, bh);
+          tma_load_3d(dst + C::kBigTileBytes + s * C::kBigSlabBytes, &tmdO, &bar_res_full[rb], s * 64, qrow0, bh);
         }
       }
       if (cta_abort) {
@@ -353,8 +354,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const int qt = tile_qt(lin), bh = lin % BH, T = tile_steps(qt), rb = ti % R;
-      const int row0 = bh * N + qt * 128;
-      const size_t grow = static_cast<size_t>(row0 + row);
+      const size_t head_row0 = static_cast<size_t>(bh) * N;
+      const int qrow = qt * 128 + row;                 // this thread's query row within the head (may be >= N in a ragged tile)
 
       // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1).  Warpgroup 0 computes the
       // tile's 128 values with coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
@@ -364,8 +365,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 #pragma unroll 4
         for (int it = 0; it < 32 / RPI; ++it) {
           const int r = 32 * (warp & 3) + it * RPI + sub;
-          const uint4 a = __ldg(reinterpret_cast<const uint4 *>(Og + static_cast<size_t>(row0 + r) * D) + part);
-          const uint4 b = __ldg(reinterpret_cast<const uint4 *>(dOg + static_cast<size_t>(row0 + r) * D) + part);
+          uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+          if (qt * 128 + r < N) {
+            a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + qt * 128 + r) * D) + part);
+            b = __ldg(reinterpret_cast<const uint4 *>(dOg + (head_row0 + qt * 128 + r) * D) + part);
+          }
           const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
           float acc = 0.f;
 #pragma unroll
@@ -380,9 +384,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
       named_bar_sync(2, 128 * NB);
       const float Dv = s_D[row];
-      const float neg_lse2 = -LSE[grow] * 1.4426950408889634f;
-      if (wg == 0) {   // per 64-row block: 64 x {-LSE log2 e}, then 64 x {-D}
-        float *blk = stats + (grow >> 6) * 128 + (grow & 63);
+      const float neg_lse2 = (qrow < N) ? -LSE[head_row0 + qrow] * 1.4426950408889634f : 0.f;
+      // Per 64-row block of a head (n64 blocks, the last one padded with zeros): 64 x {-LSE log2 e}, then 64 x {-D}.
+      if (wg == 0 && qrow < n64 * C::kStepRows) {
+        float *blk = stats + (static_cast<size_t>(bh) * n64 + (qrow >> 6)) * 128 + (qrow & 63);
         blk[0] = neg_lse2;
         blk[64] = -Dv;
       }
@@ -391,8 +396,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       for (int n = (wg - g0 % NB + NB) % NB; n < T; n += NB) {
         mbar_wait(&bar_sdp_full[wg], ((g0 + n) / NB) & 1, ab, kDqWaitSdP);
         tc_fence_after();
-        if (CAUSAL && n >= T - 2) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho2, msum2);
-        else                      dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
+        // Probabilities are zeroed beyond the causal diagonal and, in the ragged last step, for the zero-filled keys
+        // past N (which would otherwise enter the row masses).  Rows of a causal tile never reach such keys.
+        if (CAUSAL && n >= 2 * qt)                  dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho2, msum2);
+        else if (!CAUSAL && (n + 1) * C::kStepRows > N) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, N - n * C::kStepRows - 1, rho2, msum2);
+        else                                        dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar_tr_ready[wg]);
@@ -463,8 +471,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       named_bar_sync(1, 128 * NB);
       if (threadIdx.x == 128) {
         for (int sl = 0; sl < C::kSlabs; ++sl) {
-          tma_store_2d(&tmdQ, stage_dq + sl * C::kBigSlabBytes, sl * 64, row0);
-          tma_store_2d(&tmZ, stage_z + sl * C::kBigSlabBytes, sl * 64, row0);
+          tma_store_3d(&tmdQ, stage_dq + sl * C::kBigSlabBytes, sl * 64, qt * 128, bh);
+          tma_store_3d(&tmZ, stage_z + sl * C::kBigSlabBytes, sl * 64, qt * 128, bh);
         }
         bulk_commit_group();
         if (!C::kSepStaging) bulk_wait_group_read0();     // staging shares the Q / dO buffer: reads must finish first
@@ -544,8 +552,11 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
 
   TileSched sched(total_tiles);
   // tile decode: causal -> key tile 0 has the most query steps and comes first
+  // Ragged N: query steps round up.  A zero-filled query column past N contributes exactly nothing (its dO, Q and Z rows
+  // are zero and its padded statistics are zero, so t = 0 and r multiplies zero rows); key rows past N are clipped on store.
+  const int n64 = (N + C::kStepRows - 1) / C::kStepRows;
   auto tile_q_start = [&](int kt) { return CAUSAL ? kt * 128 : 0; };
-  auto tile_steps = [&](int kt) { return (N - tile_q_start(kt)) / C::kStepRows; };
+  auto tile_steps = [&](int kt) { return n64 - tile_q_start(kt) / C::kStepRows; };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (Q, dO, Z, stats) step tiles
@@ -559,13 +570,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
           if (g >= S) mbar_wait(&bar_q_empty[st], ((g / S) - 1) & 1, ab, kDkvWaitQEmpty);
           mbar_expect_tx(&bar_q_full[st], stage_tx);
           uint8_t *dst = sStage + st * C::kDkvStageBytes;
-          const int qrow = (q_head0 + n / T) * N + q_start + (n % T) * C::kStepRows;
+          const int qh = q_head0 + n / T, qrow = q_start + (n % T) * C::kStepRows;
           for (int s = 0; s < C::kSlabs; ++s) {
-            tma_load_2d(dst + s * C::kStepSlabBytes, &tmQ, &bar_q_full[st], s * 64, qrow);
-            tma_load_2d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow);
-            if (use_z) tma_load_2d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow);
+            tma_load_3d(dst + s * C::kStepSlabBytes, &tmQ, &bar_q_full[st], s * 64, qrow, qh);
+            tma_load_3d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow, qh);
+            if (use_z) tma_load_3d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow, qh);
           }
-          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + 2 * static_cast<size_t>(qrow), 512, &bar_q_full[st]);
+          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + (static_cast<size_t>(qh) * n64 + (qrow >> 6)) * 128, 512, &bar_q_full[st]);
         }
       }
       if (cta_abort) {
@@ -578,12 +589,12 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int krow0 = (lin % BH) * N + (lin / BH) * 128;
+        const int bh = lin % BH, krow0 = (lin / BH) * 128;
         if (ti >= 1) mbar_wait(&bar_res_free, (ti - 1) & 1, ab, kDkvWaitResFree);
         mbar_expect_tx(&bar_res_full, 2 * C::kBigTileBytes);
         for (int s = 0; s < C::kSlabs; ++s) {
-          tma_load_2d(sK + s * C::kBigSlabBytes, &tmK, &bar_res_full, s * 64, krow0);
-          tma_load_2d(sV + s * C::kBigSlabBytes, &tmV, &bar_res_full, s * 64, krow0);
+          tma_load_3d(sK + s * C::kBigSlabBytes, &tmK, &bar_res_full, s * 64, krow0, bh);
+          tma_load_3d(sV + s * C::kBigSlabBytes, &tmV, &bar_res_full, s * 64, krow0, bh);
         }
       }
       if (cta_abort && ti > 0)
@@ -681,7 +692,6 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const int kt = lin / BH, bh = lin % BH, Th = tile_steps(kt), T = G * Th;
-      const int krow0 = bh * N + kt * 128;
 #ifdef GPROJ_TRACE
       const unsigned long long tile_t0 = global_ns();
 #endif
@@ -745,8 +755,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       named_bar_sync(1, 128 * NB);
       if (threadIdx.x == 128) {
         for (int sl = 0; sl < C::kSlabs; ++sl) {
-          tma_store_2d(&tmdV, stage_dv + sl * C::kBigSlabBytes, sl * 64, krow0);
-          tma_store_2d(&tmdK, stage_dk + sl * C::kBigSlabBytes, sl * 64, krow0);
+          tma_store_3d(&tmdV, stage_dv + sl * C::kBigSlabBytes, sl * 64, kt * 128, bh);
+          tma_store_3d(&tmdK, stage_dk + sl * C::kBigSlabBytes, sl * 64, kt * 128, bh);
         }
         bulk_commit_group();
         if (!C::kSepStaging) {             // staging shares the K / V tile: its reads must finish before the next load

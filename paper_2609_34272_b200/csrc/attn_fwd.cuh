@@ -68,7 +68,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __syncthreads();
   if (cta_skip != 0) return;   // an earlier wait gave up: drain the rest of the grid quickly
 
-  const int n_qt = N / C::kBlockM;
+  const int n_qt = (N + C::kBlockM - 1) / C::kBlockM;   // the last tile may be ragged: rows past N load as zero, stores clip
   const int TPI = tiles_per_item;                  // 2: a pair of query tiles per work item; 1: single tiles (small grids)
   const int n_pairs = (n_qt + TPI - 1) / TPI;
   AbortState ab{status, &cta_abort};
@@ -107,11 +107,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kFwdWaitKVEmpty);
           uint8_t *dK = sKV + st * 2 * C::kTileBytes, *dV = dK + C::kTileBytes;
-          const int krow = kv_head_of(bh, Hq, G) * N + j * C::kBlockN;     // grouped-query: the group's shared K / V head
+          const int kvh = kv_head_of(bh, Hq, G), krow = j * C::kBlockN;   // grouped-query: the group's shared K / V head
           mbar_expect_tx(&bar_k_full[st], C::kTileBytes);
-          for (int s = 0; s < C::kSlabs; ++s) tma_load_2d(dK + s * C::kSlabBytes, &tmK, &bar_k_full[st], s * 64, krow);
+          for (int s = 0; s < C::kSlabs; ++s) tma_load_3d(dK + s * C::kSlabBytes, &tmK, &bar_k_full[st], s * 64, krow, kvh);
           mbar_expect_tx(&bar_v_full[st], C::kTileBytes);
-          for (int s = 0; s < C::kSlabs; ++s) tma_load_2d(dV + s * C::kSlabBytes, &tmV, &bar_v_full[st], s * 64, krow);
+          for (int s = 0; s < C::kSlabs; ++s) tma_load_3d(dV + s * C::kSlabBytes, &tmV, &bar_v_full[st], s * 64, krow, kvh);
         }
       }
       // Every load is consumed by an MMA the epilogue waits for, so nothing is in flight at exit unless the
@@ -134,7 +134,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_expect_tx(&bar_q_full, tiles * C::kTileBytes);
         for (int t = 0; t < tiles; ++t)
           for (int s = 0; s < C::kSlabs; ++s)
-            tma_load_2d(sQ + t * C::kTileBytes + s * C::kSlabBytes, &tmQ, &bar_q_full, s * 64, bh * N + (TPI * pair + t) * C::kBlockM);
+            tma_load_3d(sQ + t * C::kTileBytes + s * C::kSlabBytes, &tmQ, &bar_q_full, s * 64, (TPI * pair + t) * C::kBlockM, bh);
       }
       if (cta_abort && ti > 0)
         for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full, (ti - 1) & 1); ++spin) {}
@@ -243,12 +243,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tS + 32 * c, xr[c]);
         tmem_wait_ld();
-        if (CAUSAL && j == qt) {
+        // Keys beyond the causal diagonal, and the zero-filled columns past the last key of a ragged tile, get -inf.
+        const bool diag = CAUSAL && j == qt, tail = (j == n_qt - 1) && (N % C::kBlockN != 0);
+        if (diag || tail) {
+          const int lim = min(diag ? row : C::kBlockN - 1, tail ? N - j * C::kBlockN - 1 : C::kBlockN - 1);
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (32 * c + i > row) xr[c][i] = 0xff800000u;   // -inf: key beyond the diagonal
+              if (32 * c + i > lim) xr[c][i] = 0xff800000u;
         }
         float mx = -INFINITY;
 #pragma unroll
@@ -317,12 +320,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       tc_fence_before();
       mbar_arrive(&bar_o_free[t]);                     // O_t may be overwritten by the next work item
-      const int grow = bh * N + qt * C::kBlockM;
-      LSE[grow + row] = fmaf(m_run, alpha, logf(l_run));
+      if (qt * C::kBlockM + row < N) LSE[static_cast<size_t>(bh) * N + qt * C::kBlockM + row] = fmaf(m_run, alpha, logf(l_run));
       fence_proxy_async_smem();
       named_bar_sync(1 + t, 128);
       if (row == 0) {
-        for (int sl = 0; sl < C::kSlabs; ++sl) tma_store_2d(&tmO, stage + sl * C::kSlabBytes, sl * 64, grow);
+        for (int sl = 0; sl < C::kSlabs; ++sl) tma_store_3d(&tmO, stage + sl * C::kSlabBytes, sl * 64, qt * C::kBlockM, bh);
         bulk_commit_group();
         bulk_wait_group_read0();
         mbar_arrive(&bar_q_free);                      // this tile's half of the Q buffer may be reloaded

@@ -98,13 +98,14 @@ int device_state(DeviceState **out) {
   return st.arch_ok ? GPROJ_OK : GPROJ_ERR_ARCH;
 }
 
-// [rows x d] BF16 row-major view, box = 64 columns (128 B, one swizzle atom) x box_rows.
-bool make_map(CUtensorMap *map, const void *base, uint64_t rows, int d, int box_rows) {
-  cuuint64_t dims[2] = {static_cast<cuuint64_t>(d), rows};
-  cuuint64_t strides[1] = {static_cast<cuuint64_t>(d) * 2};
-  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
-  cuuint32_t elem[2] = {1, 1};
-  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
+// [heads x N x d] BF16 row-major view, box = 64 columns (128 B, one swizzle atom) x box_rows of ONE head: a tile never
+// crosses into the next head, rows past N read as zero and are skipped by stores.
+bool make_map(CUtensorMap *map, const void *base, int heads, int N, int d, int box_rows) {
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(heads)};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(N) * d * 2};
+  cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
+  cuuint32_t elem[3] = {1, 1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, elem,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -114,14 +115,15 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int check_shape(int B, int H, int N, int d) {
   if (B <= 0 || H <= 0 || N <= 0) return GPROJ_ERR_SHAPE;
   if (d != 64 && d != 128) return GPROJ_ERR_SHAPE;
-  if (N % 128 != 0) return GPROJ_ERR_SHAPE;
   const long long rows = static_cast<long long>(B) * H * N;
-  if (rows >= (1LL << 31) || static_cast<long long>(B) * H >= (1LL << 20)) return GPROJ_ERR_SHAPE;
-  if (rows / 128 >= (1LL << 31)) return GPROJ_ERR_SHAPE;
+  if (rows >= (1LL << 31) || static_cast<long long>(B) * H >= (1LL << 20) || N > (1 << 24)) return GPROJ_ERR_SHAPE;
   return GPROJ_OK;
 }
 
 size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+// Row statistics {-LSE log2 e, -D}: per head ceil(N / 64) blocks of 64 rows (the last one zero-padded), 512 B each.
+size_t stats_bytes(int heads, int N) { return align256(static_cast<size_t>(heads) * ((N + 63) / 64) * 512); }
 
 }  // namespace
 
@@ -152,15 +154,15 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
   if (int rc = device_state(&st)) return rc;
 
   const int BH = B * H;
-  const uint64_t rows = static_cast<uint64_t>(BH) * N, kv_rows = static_cast<uint64_t>(B) * Hkv * N;
+  const int BHkv = B * Hkv;
   CUtensorMap mQ, mK, mV, mO;
-  if (!make_map(&mQ, Q, rows, d, 128) || !make_map(&mK, K, kv_rows, d, 128) || !make_map(&mV, V, kv_rows, d, 128) ||
-      !make_map(&mO, O, rows, d, 128))
+  if (!make_map(&mQ, Q, BH, N, d, 128) || !make_map(&mK, K, BHkv, N, d, 128) || !make_map(&mV, V, BHkv, N, d, 128) ||
+      !make_map(&mO, O, BH, N, d, 128))
     return GPROJ_ERR_CUDA;
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
   // One work item = a pair of query tiles of one head (two softmax warpgroups ping-pong on the tensor core); when
   // that leaves too few items to balance the SMs, items are single tiles.
-  const int n_qt = N / 128;
+  const int n_qt = (N + 127) / 128;
   const int tiles_per_item = (static_cast<long long>(BH) * ((n_qt + 1) / 2) * 2 >= 3LL * st->sm_count) ? 2 : 1;
   const int total_items = BH * ((n_qt + tiles_per_item - 1) / tiles_per_item);
   const dim3 grid(static_cast<unsigned>(total_items < st->sm_count ? total_items : st->sm_count));   // persistent
@@ -181,8 +183,7 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
 
 size_t gproj_attn_bwd_workspace_bytes(int B, int H, int N, int d) {
   if (check_shape(B, H, N, d) != GPROJ_OK) return 0;
-  const size_t rows = static_cast<size_t>(B) * H * N;
-  return align256(rows * sizeof(float2)) + align256(rows * static_cast<size_t>(d) * 2);
+  return stats_bytes(B * H, N) + align256(static_cast<size_t>(B) * H * N * static_cast<size_t>(d) * 2);
 }
 
 int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
@@ -214,20 +215,19 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
   if (int rc = device_state(&st)) return rc;
 
   const int BH = B * H, BHkv = B * Hkv;
-  const uint64_t rows = static_cast<uint64_t>(BH) * N, kv_rows = static_cast<uint64_t>(BHkv) * N;
   float *stats = static_cast<float *>(workspace);   // per 64-row block: 64 x {-LSE log2 e}, 64 x {-D}
-  __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + align256(rows * sizeof(float2)));
+  __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + stats_bytes(BH, N));
 
   CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64, mdQst, mZst, mdKst, mdVst;
-  bool ok = make_map(&mQ128, Q, rows, d, 128) && make_map(&mdO128, dO, rows, d, 128) && make_map(&mK64, K, kv_rows, d, 64) &&
-            make_map(&mV64, V, kv_rows, d, 64) && make_map(&mK128, K, kv_rows, d, 128) && make_map(&mV128, V, kv_rows, d, 128) &&
-            make_map(&mQ64, Q, rows, d, 64) && make_map(&mdO64, dO, rows, d, 64) && make_map(&mZ64, Zneg, rows, d, 64) &&
-            make_map(&mdQst, dQ, rows, d, 128) && make_map(&mZst, Zneg, rows, d, 128) && make_map(&mdKst, dK, kv_rows, d, 128) &&
-            make_map(&mdVst, dV, kv_rows, d, 128);
+  bool ok = make_map(&mQ128, Q, BH, N, d, 128) && make_map(&mdO128, dO, BH, N, d, 128) && make_map(&mK64, K, BHkv, N, d, 64) &&
+            make_map(&mV64, V, BHkv, N, d, 64) && make_map(&mK128, K, BHkv, N, d, 128) && make_map(&mV128, V, BHkv, N, d, 128) &&
+            make_map(&mQ64, Q, BH, N, d, 64) && make_map(&mdO64, dO, BH, N, d, 64) && make_map(&mZ64, Zneg, BH, N, d, 64) &&
+            make_map(&mdQst, dQ, BH, N, d, 128) && make_map(&mZst, Zneg, BH, N, d, 128) && make_map(&mdKst, dK, BHkv, N, d, 128) &&
+            make_map(&mdVst, dV, BHkv, N, d, 128);
   if (!ok) return GPROJ_ERR_CUDA;
 
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
-  const int total_tiles = BH * (N / 128), total_kv_tiles = BHkv * (N / 128);
+  const int n_qt = (N + 127) / 128, total_tiles = BH * n_qt, total_kv_tiles = BHkv * n_qt;
   const dim3 grid(static_cast<unsigned>(total_tiles < st->sm_count ? total_tiles : st->sm_count));   // persistent: one CTA per SM
   const dim3 grid_kv(static_cast<unsigned>(total_kv_tiles < st->sm_count ? total_kv_tiles : st->sm_count));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -307,7 +307,7 @@ const char *gproj_status_string(int status) {
   switch (status) {
     case GPROJ_OK: return "ok";
     case GPROJ_ERR_NULL: return "null pointer argument";
-    case GPROJ_ERR_SHAPE: return "unsupported shape (need d in {64,128}, N a positive multiple of 128)";
+    case GPROJ_ERR_SHAPE: return "unsupported shape (need d in {64,128}, B, H, N >= 1, H a multiple of the KV heads, B*H*N < 2^31)";
     case GPROJ_ERR_ALIGN: return "tensor base address not 16-byte aligned";
     case GPROJ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case GPROJ_ERR_SCALE: return "softmax_scale must be finite and positive";

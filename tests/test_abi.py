@@ -43,7 +43,9 @@ def test_workspace_bytes(lib):
     B, H, N, d = 2, 3, 256, 64
     rows = B * H * N
     assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, d) == rows * 8 + rows * d * 2
-    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 0
+    # ragged length: statistics are padded to whole 64-row blocks per head (2 blocks x 512 B), the query-shaped array is not
+    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 2 * 512 + 100 * 64 * 2
+    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 0, 64) == 0
     assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 128, 96) == 0
 
 
@@ -52,7 +54,7 @@ def test_argument_validation_without_gpu(lib):
     bad = ctypes.c_void_p(0x1008)
     fwd = lambda Q=p, LSE=p, B=1, H=1, N=128, d=64, scale=0.125: lib.gproj_attn_fwd(Q, p, p, p, LSE, B, H, N, d, scale, 1, None)
     assert fwd(Q=None) == -1
-    assert fwd(N=100) == -2 and fwd(d=96) == -2 and fwd(B=0) == -2 and fwd(N=0) == -2
+    assert fwd(N=-128) == -2 and fwd(d=96) == -2 and fwd(B=0) == -2 and fwd(N=0) == -2
     assert fwd(Q=bad) == -3
     assert fwd(scale=0.0) == -5 and fwd(scale=float("nan")) == -5 and fwd(scale=-1.0) == -5
     bwd = lambda ws=ctypes.c_void_p(0x1000), nbytes=1 << 30, flags=0, dQ=p: lib.gproj_attn_bwd(

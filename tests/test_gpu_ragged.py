@@ -1,0 +1,116 @@
+"""GPU parity on sequence lengths that are not a multiple of the 128-row tile (through the C ABI).
+
+The kernels round tiles and 64-row steps up; rows past N are zero-filled by the tensor-map loads and clipped by the
+tensor-map stores, and key columns past N are masked where they would enter a row statistic.  Every case is compared
+with the FP64 oracle on the full tensors (same bar as the tile-aligned parity tests), with more than one head so that
+a tile reaching into the next head's rows would show.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_34272_b200 as g
+from oracle import emulation as em
+from paper_2609_34272_b200.workloads import Workload, bits, from_bits, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "witness_minus24.txt")
+
+
+def to_np(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def run_gpu(inp, alpha, causal, flags=0):
+    dev = {k: v.cuda() for k, v in inp.items()}
+    O, LSE = g.gproj_attn_fwd(dev["Q"], dev["K"], dev["V"], alpha, causal)
+    dQ, dK, dV = g.gproj_attn_bwd(dev["Q"], dev["K"], dev["V"], O, LSE, dev["dO"], alpha, causal, flags=flags)
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, (g.status_string(rc), hex(detail))
+    return {"O": to_np(O), "LSE": LSE.cpu().numpy().astype(np.float64), "dQ": to_np(dQ), "dK": to_np(dK), "dV": to_np(dV)}
+
+
+def check(got, ex, bar=1.0):
+    errs = {}
+    for n in ("O", "dQ", "dK", "dV"):
+        assert got[n].shape == ex[n].shape
+        assert np.all(np.isfinite(got[n])), n
+        errs[n] = oracle.rel_l2_percent(got[n], ex[n])
+        assert errs[n] <= bar, (n, errs)
+        assert np.abs(got[n] - ex[n]).max() <= 0.03 * np.abs(ex[n]).max(), (n, "element-wise")
+    assert np.all(np.abs(got["LSE"] - ex["LSE"]) <= 1e-4 + 1e-5 * np.abs(ex["LSE"]))
+    return errs
+
+
+# N: below one 64-row step, on and around step and tile boundaries, several tiles with a ragged tail
+LENGTHS = [4, 63, 64, 65, 127, 129, 200, 320, 1000]
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("N", LENGTHS)
+def test_ragged_lengths(N, d, causal):
+    w = Workload("ragged", 2, 3, N, d, causal, k_offset=8.0, seed=5150 + 31 * N + d + (7 if causal else 0))
+    inp = make_inputs(w)
+    ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, causal)
+    check(run_gpu(inp, w.softmax_scale, causal), ex)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_ragged_grouped_queries(causal):
+    w = Workload("ragged_gqa", 2, 4, 200, 64, causal, k_offset=8.0, seed=6160, Hkv=2)
+    inp = make_inputs(w)
+    ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, causal)
+    check(run_gpu(inp, w.softmax_scale, causal), ex)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("d", [64, 128])
+def test_single_token(d, causal):
+    # N = 1: the row has one key, so O = v, LSE = alpha q.k, dV = dO, and the exact dQ and dK vanish.  With the
+    # projection dQ is exactly zero (t k - (t / 1) (1 k)); dK keeps only the rounding of BF16(lambda q).
+    w = Workload("one", 2, 2, 1, d, causal, k_offset=4.0, seed=77 + d)
+    inp = make_inputs(w)
+    got = run_gpu(inp, w.softmax_scale, causal)
+    assert np.array_equal(got["O"], to_np(inp["V"]))
+    assert np.array_equal(got["dV"], to_np(inp["dO"]))
+    assert np.all(got["dQ"] == 0.0)
+    assert np.abs(got["dK"]).max() <= 1e-4
+    lse = w.softmax_scale * (to_np(inp["Q"]) * to_np(inp["K"])).sum(-1)
+    assert np.all(np.abs(got["LSE"] - lse) <= 1e-4 + 1e-5 * np.abs(lse))
+
+
+def test_uncorrected_backward_on_ragged_length():
+    # the ablation flags take the same masked path
+    w = Workload("ragged_off", 1, 2, 333, 64, True, k_offset=4.0, seed=99)
+    inp = make_inputs(w)
+    ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, True)
+    check(run_gpu(inp, w.softmax_scale, True, flags=3), ex, bar=5.0)
+
+
+def test_minus24_witness_at_its_own_size():
+    # The four-key witness of Appendix A ("An exact -24 witness") as an N = 4 problem, columns zero-padded to d = 64:
+    # nothing but the four printed keys is in the row's support.
+    vals = {}
+    for line in open(GOLDEN):
+        line = line.split("#", 1)[0].strip()
+        if line:
+            key, *rest = line.split()
+            vals[key] = [float(x) for x in rest]
+    N, d = 4, 64
+    Q = np.zeros((N, d)); K = np.zeros((N, d)); V = np.zeros((N, d)); U = np.zeros((N, d))
+    for j in range(4):
+        K[j, :2] = vals[f"k{j + 1}"]
+        V[j, :2] = vals[f"v{j + 1}"]
+    U[:, :2] = vals["u"]
+    inp = {n: from_bits(em.f64_to_bf16_bits(x)).reshape(1, 1, N, d) for n, x in (("Q", Q), ("K", K), ("V", V), ("dO", U))}
+    alpha = vals["alpha"][0]
+    on = run_gpu(inp, alpha, False)
+    off = run_gpu(inp, alpha, False, flags=g.FLAG_NO_Q_CORRECTION)
+    assert np.all(on["O"][0, 0, :, 0] == vals["o"][0]) and np.all(on["O"][0, 0, :, 1] == vals["o"][1])
+    assert np.all(on["dQ"][0, 0, :, 0] == vals["dq0_gproj"][0])
+    assert np.all(off["dQ"][0, 0, :, 0] == vals["dq0_uncorrected"][0])

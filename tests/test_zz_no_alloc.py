@@ -49,5 +49,6 @@ def test_static_scratch_rejects_shapes_beyond_its_size():
     assert g.gproj_attn_bwd_workspace_bytes(4, 32, 8192, 128) > binding.STATIC_SCRATCH_BYTES
     rc = lib.gproj_attn_bwd_static_scratch(p, p, p, p, p, p, p, p, p, 4, 32, 8192, 128, 0.0884, 0, 0, None)
     assert rc == -4
-    rc = lib.gproj_attn_bwd_static_scratch(p, p, p, p, p, p, p, p, p, 1, 1, 100, 64, 0.125, 1, 0, None)
+    # an unsupported head dimension is rejected by the shape check, again before any pointer is used
+    rc = lib.gproj_attn_bwd_static_scratch(p, p, p, p, p, p, p, p, p, 1, 1, 128, 96, 0.125, 1, 0, None)
     assert rc == -2

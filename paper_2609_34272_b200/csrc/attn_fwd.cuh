@@ -59,7 +59,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t *sKV = sQ + 2 * C::kTileBytes;            // stage s: K tile, then V tile
 
   __shared__ uint64_t bar_q_full, bar_q_free, bar_k_full[S], bar_v_full[S], bar_kv_empty[S];
-  __shared__ uint64_t bar_s_full[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_drain[2];
+  __shared__ uint64_t bar_s_full[2], bar_s_free[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -79,7 +79,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int s = 0; s < S; ++s) { mbar_init(&bar_k_full[s], 1); mbar_init(&bar_v_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(&bar_drain[t], 1);
-      mbar_init(&bar_s_full[t], 1); mbar_init(&bar_p_ready[t], 128); mbar_init(&bar_pv_done[t], 1); mbar_init(&bar_o_free[t], 128);
+      mbar_init(&bar_s_full[t], 1); mbar_init(&bar_s_free[t], 128); mbar_init(&bar_p_ready[t], 128); mbar_init(&bar_pv_done[t], 1); mbar_init(&bar_o_free[t], 128);
     }
     fence_mbar_init();
   }
@@ -157,10 +157,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
           if (!active(pair, t, j)) continue;
-          // S_t may be overwritten once its previous contents are dead: read by the softmax (P~ elsewhere), or,
-          // when P~ lives in the same columns, consumed by the previous P~V product.
+          // S_t may be overwritten once its previous contents are dead: copied to registers by the softmax (P~ has its
+          // own columns), or, when P~ lives in the same columns, consumed by the previous P~V product.
           if (cnt[t] > 0) {
-            if (C::kSepP) mbar_wait(&bar_p_ready[t], (cnt[t] - 1) & 1, ab, kFwdWaitSFree);
+            if (C::kSepP) mbar_wait(&bar_s_free[t], (cnt[t] - 1) & 1, ab, kFwdWaitSFree);
             else          mbar_wait(&bar_pv_done[t], (cnt[t] - 1) & 1, ab, kFwdWaitSFree);
           }
           tc_fence_after();
@@ -243,6 +243,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tS + 32 * c, xr[c]);
         tmem_wait_ld();
+        if (C::kSepP) { tc_fence_before(); mbar_arrive(&bar_s_free[t]); }   // the next S_t may be issued while this one is in the ALUs
         // Keys beyond the causal diagonal, and the zero-filled columns past the last key of a ragged tile, get -inf.
         const bool diag = CAUSAL && j == qt, tail = (j == n_qt - 1) && (N % C::kBlockN != 0);
         if (diag || tail) {
@@ -253,34 +254,49 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int i = 0; i < 32; ++i)
               if (32 * c + i > lim) xr[c][i] = 0xff800000u;
         }
-        float mx = -INFINITY;
+        // Row maximum over eight independent chains (only two softmax warps share a scheduler, so a 128-long dependent
+        // chain would be pure latency).
+        float mxp[8];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int i = 0; i < 8; ++i) mxp[i] = __uint_as_float(xr[0][i]);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(xr[c][i]));
-        const float m_new = fmaxf(m_run, mx);
+        for (int e = 8; e < 128; ++e) mxp[e & 7] = fmaxf(mxp[e & 7], __uint_as_float(xr[e >> 5][e & 31]));
+        const float mx = fmaxf(fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])), fmaxf(fmaxf(mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7])));
+        // Lazy maximum: the running maximum is only raised when the tile's maximum exceeds it by more than 2^kLazyLog2
+        // in the exponent domain; otherwise the stale value stays (z <= 2^kLazyLog2, harmless in FP32 / BF16) and neither
+        // l nor the accumulator needs a rescale.  The first tile always sets it (m_run = -inf).
+        float m_new = fmaxf(m_run, mx);
+#ifndef GPROJ_FWD_EAGER_MAX
+        if (__fmul_rn(__fsub_rn(m_new, m_run), scale_log2) <= 8.0f) m_new = m_run;
+#endif
         const float corr = fast_exp2(__fmul_rn(__fsub_rn(m_run, m_new), scale_log2));
         // FMA_SOFTMAX reproduces the native fused form of Eq. "historical-fma": z = exp2(fma(x, a, -fl32(x_max a))),
         // in which x a is not rounded separately, so the largest score need not map to exactly zero.
         const float m_scaled = __fmul_rn(m_new, scale_log2);
         // P~ of the previous key tile must have been consumed (and O_t updated) before either is touched
         if (j > 0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
-        float rs = 0.f;
+        // Two columns per packed FP32 instruction: (x - x_max) and the scale keep their separate roundings
+        // (add.rn / mul.rn), the fused variant is one fma.rn; the row sum runs in four packed partial sums.
+        const uint64_t negm2 = f32x2(-m_new, -m_new), scale2 = f32x2(scale_log2, scale_log2), negms2 = f32x2(-m_scaled, -m_scaled);
+        uint64_t rs2[2] = {f32x2(0.f, 0.f), f32x2(0.f, 0.f)};
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float z0 = FMA_SOFTMAX ? fast_exp2(fmaf(__uint_as_float(xr[c][2 * i]), scale_log2, -m_scaled))
-                                         : fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i]), m_new), scale_log2));
-            const float z1 = FMA_SOFTMAX ? fast_exp2(fmaf(__uint_as_float(xr[c][2 * i + 1]), scale_log2, -m_scaled))
-                                         : fast_exp2(__fmul_rn(__fsub_rn(__uint_as_float(xr[c][2 * i + 1]), m_new), scale_log2));
-            rs += z0 + z1;
+            const uint64_t x2 = f32x2_bits(xr[c][2 * i], xr[c][2 * i + 1]);
+            float a0, a1;
+            f32x2_split(FMA_SOFTMAX ? fma2(x2, scale2, negms2) : mul2(add2(x2, negm2), scale2), a0, a1);
+            const float z0 = fast_exp2(a0), z1 = fast_exp2(a1);
+            rs2[i & 1] = add2(rs2[i & 1], f32x2(z0, z1));
             pk[i] = pack_bf16x2(z0, z1);
           }
           tmem_st16(tP + 16 * c, pk);
         }
-        l_run = l_run * corr + rs;
+        float rs0, rs1, rs2a, rs3;
+        f32x2_split(rs2[0], rs0, rs1);
+        f32x2_split(rs2[1], rs2a, rs3);
+        l_run = l_run * corr + ((rs0 + rs1) + (rs2a + rs3));
         if (j > 0 && __any_sync(0xffffffffu, m_new != m_run)) {
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {

@@ -42,10 +42,40 @@ struct FwdCfg {
 
 enum FwdWaitCode {
   kFwdWaitQ = 0x11, kFwdWaitK = 0x12, kFwdWaitV = 0x13, kFwdWaitKVEmpty = 0x14, kFwdWaitS = 0x15, kFwdWaitP = 0x16,
-  kFwdWaitPV = 0x17, kFwdWaitSFree = 0x18, kFwdWaitOFree = 0x19, kFwdWaitQFree = 0x1a
+  kFwdWaitPV = 0x17, kFwdWaitSFree = 0x18, kFwdWaitOFree = 0x19, kFwdWaitQFree = 0x1a, kFwdWaitTurn = 0x1b
 };
 
-template <int D, bool CAUSAL, bool FMA_SOFTMAX>
+
+// z = exp2(fl32[(x - x_max) (alpha log2 e)]) for the 128 columns of one row (two columns per packed FP32 instruction:
+// the subtraction and the scale keep their separate roundings, add.rn / mul.rn; the fused variant of
+// Eq. "historical-fma" is one fma.rn), BF16 pairs stored to TMEM at tP, returns the FP32 row sum of z (four packed
+// partial sums).
+template <bool FMA_SOFTMAX>
+__device__ __forceinline__ float softmax_exp_store(const uint32_t (&xr)[4][32], uint32_t tP, float m_new, float scale_log2, float m_scaled) {
+  const uint64_t negm2 = f32x2(-m_new, -m_new), scale2 = f32x2(scale_log2, scale_log2), negms2 = f32x2(-m_scaled, -m_scaled);
+  uint64_t rs2[2] = {f32x2(0.f, 0.f), f32x2(0.f, 0.f)};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint64_t x2 = f32x2_bits(xr[c][2 * i], xr[c][2 * i + 1]);
+      const uint64_t a2 = FMA_SOFTMAX ? fma2(x2, scale2, negms2) : mul2(add2(x2, negm2), scale2);
+      float a0, a1;
+      f32x2_split(a2, a0, a1);
+      const float z0 = fast_exp2(a0), z1 = fast_exp2(a1);
+      rs2[i & 1] = add2(rs2[i & 1], f32x2(z0, z1));
+      pk[i] = pack_bf16x2(z0, z1);
+    }
+    tmem_st16(tP + 16 * c, pk);
+  }
+  float r0, r1, r2, r3;
+  f32x2_split(rs2[0], r0, r1);
+  f32x2_split(rs2[1], r2, r3);
+  return (r0 + r1) + (r2 + r3);
+}
+
+template <int D, bool CAUSAL, bool FMA_SOFTMAX, bool TURNS>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -59,7 +89,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t *sKV = sQ + 2 * C::kTileBytes;            // stage s: K tile, then V tile
 
   __shared__ uint64_t bar_q_full, bar_q_free, bar_k_full[S], bar_v_full[S], bar_kv_empty[S];
-  __shared__ uint64_t bar_s_full[2], bar_s_free[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_drain[2];
+  __shared__ uint64_t bar_s_full[2], bar_s_free[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_turn[2], bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -79,7 +109,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int s = 0; s < S; ++s) { mbar_init(&bar_k_full[s], 1); mbar_init(&bar_v_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(&bar_drain[t], 1);
-      mbar_init(&bar_s_full[t], 1); mbar_init(&bar_s_free[t], 128); mbar_init(&bar_p_ready[t], 128); mbar_init(&bar_pv_done[t], 1); mbar_init(&bar_o_free[t], 128);
+      mbar_init(&bar_s_full[t], 1); mbar_init(&bar_s_free[t], 128); mbar_init(&bar_p_ready[t], 128); mbar_init(&bar_pv_done[t], 1); mbar_init(&bar_o_free[t], 128); mbar_init(&bar_turn[t], 128);
     }
     fence_mbar_init();
   }
@@ -220,7 +250,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tS = tmem_base + C::kColS + 128 * t + lane_addr;
     const uint32_t tO = tmem_base + C::kColO + D * t + lane_addr;
     const uint32_t tP = tmem_base + (C::kSepP ? C::kColP + 64 * t : C::kColS + 128 * t) + lane_addr;
-    int ti = 0, cnt = 0;
+    int ti = 0, cnt = 0, turn = 0;
     // With single-tile items the second warpgroup has nothing to do for the whole launch (and bar_q_free expects one
     // arrival per item only).
     for (int lin = (t < TPI) ? sched.next() : -1; lin >= 0; lin = sched.next(), ++ti) {
@@ -235,8 +265,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         continue;
       }
       float m_run = -INFINITY, l_run = 0.f;
+      // Both tiles of the pair exist: the warpgroups alternate in the exponential phase, step by step, tile 0 first.
+      const bool take_turns = TURNS && (TPI == 2) && (2 * pair + 1 < n_qt);
       for (int j = 0; j < T; ++j) {
-        if (!active(pair, t, j)) continue;
+        if (!active(pair, t, j)) {
+          // no work in this step (causal: the first tile of the pair ends one key tile earlier): pass the turn on
+          if (take_turns) {
+            if (t == 1 || turn > 0) mbar_wait(&bar_turn[t], (t == 1 ? turn : turn - 1) & 1, ab, kFwdWaitTurn);
+            mbar_arrive(&bar_turn[1 - t]);
+            ++turn;
+          }
+          continue;
+        }
         mbar_wait(&bar_s_full[t], cnt & 1, ab, kFwdWaitS);
         tc_fence_after();
         uint32_t xr[4][32];
@@ -254,13 +294,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int i = 0; i < 32; ++i)
               if (32 * c + i > lim) xr[c][i] = 0xff800000u;
         }
-        // Row maximum over eight independent chains (only two softmax warps share a scheduler, so a 128-long dependent
-        // chain would be pure latency).
+        // Row maximum over eight independent chains of three-input maxima (only two softmax warps share a scheduler, so a
+        // 128-long dependent chain would be pure latency).
         float mxp[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mxp[i] = __uint_as_float(xr[0][i]);
+        for (int i = 0; i < 8; ++i) mxp[i] = fmaxf(__uint_as_float(xr[0][i]), __uint_as_float(xr[0][8 + i]));
 #pragma unroll
-        for (int e = 8; e < 128; ++e) mxp[e & 7] = fmaxf(mxp[e & 7], __uint_as_float(xr[e >> 5][e & 31]));
+        for (int e = 16; e < 128; e += 16)
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            mxp[i] = fmax3(mxp[i], __uint_as_float(xr[(e + i) >> 5][(e + i) & 31]), __uint_as_float(xr[(e + 8 + i) >> 5][(e + 8 + i) & 31]));
         const float mx = fmaxf(fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])), fmaxf(fmaxf(mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7])));
         // Lazy maximum: the running maximum is only raised when the tile's maximum exceeds it by more than 2^kLazyLog2
         // in the exponent domain; otherwise the stale value stays (z <= 2^kLazyLog2, harmless in FP32 / BF16) and neither
@@ -275,28 +318,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const float m_scaled = __fmul_rn(m_new, scale_log2);
         // P~ of the previous key tile must have been consumed (and O_t updated) before either is touched
         if (j > 0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
-        // Two columns per packed FP32 instruction: (x - x_max) and the scale keep their separate roundings
-        // (add.rn / mul.rn), the fused variant is one fma.rn; the row sum runs in four packed partial sums.
-        const uint64_t negm2 = f32x2(-m_new, -m_new), scale2 = f32x2(scale_log2, scale_log2), negms2 = f32x2(-m_scaled, -m_scaled);
-        uint64_t rs2[2] = {f32x2(0.f, 0.f), f32x2(0.f, 0.f)};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const uint64_t x2 = f32x2_bits(xr[c][2 * i], xr[c][2 * i + 1]);
-            float a0, a1;
-            f32x2_split(FMA_SOFTMAX ? fma2(x2, scale2, negms2) : mul2(add2(x2, negm2), scale2), a0, a1);
-            const float z0 = fast_exp2(a0), z1 = fast_exp2(a1);
-            rs2[i & 1] = add2(rs2[i & 1], f32x2(z0, z1));
-            pk[i] = pack_bf16x2(z0, z1);
-          }
-          tmem_st16(tP + 16 * c, pk);
-        }
-        float rs0, rs1, rs2a, rs3;
-        f32x2_split(rs2[0], rs0, rs1);
-        f32x2_split(rs2[1], rs2a, rs3);
-        l_run = l_run * corr + ((rs0 + rs1) + (rs2a + rs3));
+        // The exponential phase is the only heavy user of the special-function unit (16 results per clock per SM, the
+        // forward's scarcest pipe).  With TURNS the two warpgroups alternate in it, so that one's exponentials run against
+        // the other's loads, maxima and barrier work instead of both phases colliding and then both leaving the unit idle
+        // (measured: +9 % at d = 128, -4 % at d = 64, so the host enables it for d = 128 with paired tiles only).
+        if (take_turns) { if (t == 1 || turn > 0) mbar_wait(&bar_turn[t], (t == 1 ? turn : turn - 1) & 1, ab, kFwdWaitTurn); }
+        const float rs = softmax_exp_store<FMA_SOFTMAX>(xr, tP, m_new, scale_log2, m_scaled);
+        if (take_turns) { mbar_arrive(&bar_turn[1 - t]); ++turn; }
+        l_run = l_run * corr + rs;
         if (j > 0 && __any_sync(0xffffffffu, m_new != m_run)) {
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {

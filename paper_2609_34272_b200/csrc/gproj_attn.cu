@@ -74,14 +74,16 @@ int device_state(DeviceState **out) {
       if (cudaGetSymbolAddress(reinterpret_cast<void **>(&st.status_ptr), g_device_status) != cudaSuccess)
         return GPROJ_ERR_CUDA;
       bool ok = true;
-      ok &= allow_smem(attn_fwd_kernel<64, true, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<64, false, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, true, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, false, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<64, true, true>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<64, false, true>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, true, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, false, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, false, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, false, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, false, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, false, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, false, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, false, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, true, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, true, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, true, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, true, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, true>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, false>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<128, true>, BwdCfg<128>::kDqSmemBytes) == cudaSuccess;
@@ -167,13 +169,17 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
   const int total_items = BH * ((n_qt + tiles_per_item - 1) / tiles_per_item);
   const dim3 grid(static_cast<unsigned>(total_items < st->sm_count ? total_items : st->sm_count));   // persistent
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define GPROJ_LAUNCH_FWD(DD, CC, FF)                                                                                \
-  attn_fwd_kernel<DD, CC, FF><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(                             \
+#define GPROJ_LAUNCH_FWD(DD, CC, FF, TT)                                                                            \
+  attn_fwd_kernel<DD, CC, FF, TT><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(                         \
       mQ, mK, mV, mO, LSE, N, BH, H, G, tiles_per_item, total_items, scale_log2, softmax_scale, st->status_ptr)
-#define GPROJ_LAUNCH_FWD_C(DD, FF)                                                                                  \
-  do { if (causal) GPROJ_LAUNCH_FWD(DD, true, FF); else GPROJ_LAUNCH_FWD(DD, false, FF); } while (0)
-  if (d == 64) { if (fma) GPROJ_LAUNCH_FWD_C(64, true); else GPROJ_LAUNCH_FWD_C(64, false); }
-  else         { if (fma) GPROJ_LAUNCH_FWD_C(128, true); else GPROJ_LAUNCH_FWD_C(128, false); }
+#define GPROJ_LAUNCH_FWD_C(DD, FF, TT)                                                                              \
+  do { if (causal) GPROJ_LAUNCH_FWD(DD, true, FF, TT); else GPROJ_LAUNCH_FWD(DD, false, FF, TT); } while (0)
+  // the softmax warpgroups alternate in the exponential phase where that was measured to pay: d = 128, paired tiles
+  const bool turns = (d == 128) && (tiles_per_item == 2) && !fma;
+  if (d == 64) { if (fma) GPROJ_LAUNCH_FWD_C(64, true, false); else GPROJ_LAUNCH_FWD_C(64, false, false); }
+  else if (fma) GPROJ_LAUNCH_FWD_C(128, true, false);
+  else if (turns) GPROJ_LAUNCH_FWD_C(128, false, true);
+  else GPROJ_LAUNCH_FWD_C(128, false, false);
 #undef GPROJ_LAUNCH_FWD_C
 #undef GPROJ_LAUNCH_FWD
   if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;

@@ -19,9 +19,12 @@
 //                   Epilogue: dK = BF16(alpha acc), dV = BF16(acc).
 //
 // Pipeline.  TMEM holds kNB score buffers (S and dP of one 64-wide step each) next to the two FP32
-// accumulators: 3 buffers at d = 64, 2 at d = 128 (512 columns either way).  Compute warpgroup w owns
-// buffer w and the steps n = w (mod kNB); it overwrites the consumed S / dP columns with the packed BF16
-// operands r / t.  The tensor-core queue is only one or two instructions deep, so an issuing warp is stalled
+// accumulators: 3 buffers at d = 64, 2 at d = 128 (512 columns either way).  Four compute warpgroups form two
+// groups; a group takes every second step and its two warpgroups split the step's 64 columns (thread <-> (row,
+// 32-column slice)).  A buffer is back with the tensor core after half the ALU time one warpgroup per step would
+// take -- that time bounds the loop  scores -> ALUs -> second-stage products -> buffer free  each buffer runs
+// through -- while the two groups, at different phases, hide each other's TMEM and barrier latencies.
+// The packed BF16 operands r / t overwrite the consumed S columns of their own 16-column chunk.  The tensor-core queue is only one or two instructions deep, so an issuing warp is stalled
 // for as long as its MMAs execute and anything else it does (barrier polls, commits) would idle the pipe.
 // Two warps therefore issue: warp 1 the score products of every step, warp 2 the second-stage products; each
 // one's bookkeeping overlaps the other's MMAs.  Reuse of a score buffer is ordered by an explicit barrier
@@ -49,8 +52,16 @@ struct BwdCfg {
   static constexpr int kStepRows = 64;                            // rows of a streamed tile
   static constexpr int kStepSlabBytes = kStepRows * 128;
   static constexpr int kStepTileBytes = kSlabs * kStepSlabBytes;
-  static constexpr int kNB = (D == 64) ? 3 : 2;                   // score buffers = compute warpgroups
-  static constexpr int kThreads = 128 + 128 * kNB;                // stage producer, 2 MMA warps, tile loader; kNB compute warpgroups
+  static constexpr int kNB = (D == 64) ? 3 : 2;                   // score buffers (steps in flight)
+  // Compute warpgroups: kGroups groups of kSlices warpgroups.  Group a takes the steps g = a (mod kGroups); inside it
+  // warpgroup h takes columns [kSliceCols h, kSliceCols (h + 1)) of the step.  Two groups keep two steps in the ALUs at
+  // different phases (one group's TMEM / barrier latencies hide behind the other's arithmetic); two slices halve the
+  // time a score buffer stays away from the tensor core.
+  static constexpr int kGroups = 2, kSlices = 2;
+  static constexpr int kWG = kGroups * kSlices;
+  static constexpr int kSliceCols = kStepRows / kSlices;
+  static constexpr int kCompute = 128 * kWG;                      // compute threads
+  static constexpr int kThreads = 128 + kCompute;                 // stage producer, 2 MMA warps, tile loader; compute warpgroups
   // Output staging for the TMA stores: its own buffer where shared memory allows (d = 64), else over the stationary tile.
   static constexpr bool kSepStaging = (D == 64);
   // TMEM columns: buffer b holds S at 128 b and dP at 128 b + 64; accumulators follow
@@ -107,68 +118,69 @@ __device__ __forceinline__ void score_pair(uint32_t x0, uint32_t x1, uint32_t dp
   t_packed = pack_bf16x2(t0, t1);
 }
 
-// One 64-column step of the dQ side for one query row.  `lim` = (row index) - (key index of column 0):
-// with MASKED, column c is beyond the causal diagonal when c > lim.  TMEM is read in 16-column chunks and the
-// next chunk's load is in flight while the current one is in the ALUs; the packed r / t overwrite columns
-// whose scores were consumed at least one chunk earlier.
+// One step of the dQ side for one query row and one slice (kSliceCols = 32 keys) of the step's 64 keys, in two 16-column
+// chunks: the second chunk's TMEM load is in flight while the first is in the ALUs.  tS / tdP address the slice's S and
+// dP columns; `lim` = (row index) - (key index of the slice's column 0): with MASKED, column c is beyond the causal
+// diagonal (or past the last key) when c > lim.  The packed BF16 operands overwrite the chunk's OWN score columns (r over
+// its first eight, t over its last eight: one K = 16 MMA slice each), so nobody writes over scores yet to be read.
 template <bool MASKED>
-__device__ __forceinline__ void dq_step(uint32_t tS, uint32_t tdP, float scale_log2, float neg_lse2, float Dv, int lim,
-                                        uint64_t &rho2, uint64_t &msum2) {
+__device__ __forceinline__ void dq_slice(uint32_t tS, uint32_t tdP, float scale_log2, float neg_lse2, float Dv, int lim,
+                                         uint64_t &rho2, uint64_t &msum2) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2), nl2 = f32x2(neg_lse2, neg_lse2), nd2 = f32x2(-Dv, -Dv);
   uint32_t xs[2][16], xp[2][16];
   tmem_ld16(tS, xs[0]);
   tmem_ld16(tdP, xp[0]);
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < 2; ++c) {
     tmem_wait_ld();
-    if (c < 3) {
-      tmem_ld16(tS + 16 * (c + 1), xs[(c + 1) & 1]);
-      tmem_ld16(tdP + 16 * (c + 1), xp[(c + 1) & 1]);
+    if (c == 0) {
+      tmem_ld16(tS + 16, xs[1]);
+      tmem_ld16(tdP + 16, xp[1]);
     }
     uint32_t pr[8], pt[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int col = 16 * c + 2 * i;
-      score_pair<MASKED>(xs[c & 1][2 * i], xs[c & 1][2 * i + 1], xp[c & 1][2 * i], xp[c & 1][2 * i + 1], scale2, nl2, nd2,
-                         col <= lim, col + 1 <= lim, pr[i], pt[i]);
+      score_pair<MASKED>(xs[c][2 * i], xs[c][2 * i + 1], xp[c][2 * i], xp[c][2 * i + 1], scale2, nl2, nd2, col <= lim, col + 1 <= lim,
+                         pr[i], pt[i]);
       // row masses of the operands AS ROUNDED (Eq. "gproj-row-mass"): re-expand the BF16 pairs and add in FP32
       msum2 = add2(msum2, f32x2_bits(pr[i] << 16, pr[i] & 0xffff0000u));
       rho2 = add2(rho2, f32x2_bits(pt[i] << 16, pt[i] & 0xffff0000u));
     }
-    tmem_st8(tS + 8 * c, pr);      // r over consumed S columns
-    tmem_st8(tdP + 8 * c, pt);     // t over consumed dP columns
+    tmem_st8(tS + 16 * c, pr);
+    tmem_st8(tS + 16 * c + 8, pt);
   }
 }
 
-// One 64-column step of the dK/dV side for one key row.  `lim` = (key row) - (query index of column 0):
-// with MASKED, column c is a query before this key when c < lim.  nl / nd: per-column -LSE log2 e and -D.
+// One step of the dK/dV side for one key row and one slice (32 queries) of the step's 64 queries, chunked as above.
+// `lim` = (key row) - (query index of the slice's column 0): with MASKED, column c is a query before this key when
+// c < lim.  nl / nd: the slice's per-column -LSE log2 e and -D (shared memory, same address for every lane: broadcast).
 template <bool MASKED>
-__device__ __forceinline__ void dkv_step(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim) {
+__device__ __forceinline__ void dkv_slice(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2);
   uint32_t xs[2][16], xp[2][16];
   tmem_ld16(tS, xs[0]);
   tmem_ld16(tdP, xp[0]);
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < 2; ++c) {
     tmem_wait_ld();
-    if (c < 3) {
-      tmem_ld16(tS + 16 * (c + 1), xs[(c + 1) & 1]);
-      tmem_ld16(tdP + 16 * (c + 1), xp[(c + 1) & 1]);
+    if (c == 0) {
+      tmem_ld16(tS + 16, xs[1]);
+      tmem_ld16(tdP + 16, xp[1]);
     }
     uint32_t pr[8], pt[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      // statistics of four columns per 16-byte shared-memory read (same address for every lane: broadcast)
       const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);
       const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
       const int col = 16 * c + 4 * i;
-      score_pair<MASKED>(xs[c & 1][4 * i], xs[c & 1][4 * i + 1], xp[c & 1][4 * i], xp[c & 1][4 * i + 1], scale2, l4.x, d4.x,
-                         col >= lim, col + 1 >= lim, pr[2 * i], pt[2 * i]);
-      score_pair<MASKED>(xs[c & 1][4 * i + 2], xs[c & 1][4 * i + 3], xp[c & 1][4 * i + 2], xp[c & 1][4 * i + 3], scale2, l4.y, d4.y,
-                         col + 2 >= lim, col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
+      score_pair<MASKED>(xs[c][4 * i], xs[c][4 * i + 1], xp[c][4 * i], xp[c][4 * i + 1], scale2, l4.x, d4.x, col >= lim, col + 1 >= lim,
+                         pr[2 * i], pt[2 * i]);
+      score_pair<MASKED>(xs[c][4 * i + 2], xs[c][4 * i + 3], xp[c][4 * i + 2], xp[c][4 * i + 3], scale2, l4.y, d4.y, col + 2 >= lim,
+                         col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
     }
-    tmem_st8(tS + 8 * c, pr);
-    tmem_st8(tdP + 8 * c, pt);
+    tmem_st8(tS + 16 * c, pr);
+    tmem_st8(tS + 16 * c + 8, pt);
   }
 }
 
@@ -198,7 +210,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
-  __shared__ float s_rho[NB - 1][128], s_m[NB - 1][128], s_lam[128], s_D[128];
+  __shared__ float s_rho[C::kWG - 1][128], s_m[C::kWG - 1][128], s_lam[128], s_D[128];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
@@ -212,9 +224,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     cta_abort = 0;
     for (int r = 0; r < R; ++r) { mbar_init(&bar_res_full[r], 1); mbar_init(&bar_res_free[r], 2); }
     for (int s = 0; s < S; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
-    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
+    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128 * C::kSlices); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
-    mbar_init(&bar_acc_free, 128 * NB);
+    mbar_init(&bar_acc_free, C::kCompute);
     mbar_init(&bar_drain[0], 1);
     mbar_init(&bar_drain[1], 1);
     fence_mbar_init();
@@ -328,15 +340,16 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         mbar_wait(&bar_tr_ready[b], (g / NB) & 1, ab, kDqWaitTR);
         tc_fence_after();
         const SmemDesc dscK = dscK0mn.advanced(st * C::kDqStageBytes);
-        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;     // packed BF16 r / t over the S / dP columns
+        // packed BF16 operands of key slice k (16 keys): r over columns 16 k .. 16 k + 7 of the buffer, t over the next eight
+        const uint32_t tR = tmem_base + 128 * b, tT = tR + 8;
         const uint32_t acc = (p > 0) ? 1u : 0u;
         if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)
-            umma_ts(tmem_base + C::kColAcc0, tT + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+            umma_ts(tmem_base + C::kColAcc0, tT + 16 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)
-            umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+            umma_ts(tmem_base + C::kColAcc1, tR + 16 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
           umma_commit(&bar_buf_free[b]);
           umma_commit(&bar_kv_empty[st]);
           if (p == T - 1) umma_commit(&bar_acc_done);
@@ -346,25 +359,25 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     }
     drain_mmas_if_aborted(&bar_drain[1], ab);
   } else {
-    // ---------------------------------------------------------------- compute: thread <-> query row
-    const int wg = (warp - 4) >> 2;
+    // ---------------------------------------------------------------- compute: thread <-> (query row, key slice of every kGroups-th step)
+    const int wg = (warp - 4) >> 2, grp = wg / C::kSlices, slice = wg % C::kSlices;
     const int row = 32 * (warp & 3) + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
-    const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
+    const uint32_t slice_addr = tmem_base + lane_addr + C::kSliceCols * slice;
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const int qt = tile_qt(lin), bh = lin % BH, T = tile_steps(qt), rb = ti % R;
       const size_t head_row0 = static_cast<size_t>(bh) * N;
       const int qrow = qt * 128 + row;                 // this thread's query row within the head (may be >= N in a ragged tile)
 
-      // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1).  Warpgroup 0 computes the
-      // tile's 128 values with coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
-      if (wg == 0) {
+      // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1): each of the 16 compute warps
+      // takes eight rows, coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
+      {
         constexpr int L = D / 8, RPI = 32 / L;           // lanes per row, rows per warp-wide load
         const int sub = lane / L, part = lane % L;
-#pragma unroll 4
-        for (int it = 0; it < 32 / RPI; ++it) {
-          const int r = 32 * (warp & 3) + it * RPI + sub;
+#pragma unroll
+        for (int it = 0; it < 8 / RPI; ++it) {
+          const int r = 8 * (warp - 4) + it * RPI + sub;
           uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
           if (qt * 128 + r < N) {
             a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + qt * 128 + r) * D) + part);
@@ -382,7 +395,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
           if (part == 0) s_D[r] = acc;
         }
       }
-      named_bar_sync(2, 128 * NB);
+      named_bar_sync(2, C::kCompute);
       const float Dv = s_D[row];
       const float neg_lse2 = (qrow < N) ? -LSE[head_row0 + qrow] * 1.4426950408889634f : 0.f;
       // Per 64-row block of a head (n64 blocks, the last one padded with zeros): 64 x {-LSE log2 e}, then 64 x {-D}.
@@ -393,17 +406,20 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
 
       uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);
-      for (int n = (wg - g0 % NB + NB) % NB; n < T; n += NB) {
-        mbar_wait(&bar_sdp_full[wg], ((g0 + n) / NB) & 1, ab, kDqWaitSdP);
+      for (int n = (grp - g0 % C::kGroups + C::kGroups) % C::kGroups; n < T; n += C::kGroups) {
+        const int g = g0 + n, b = g % NB;
+        mbar_wait(&bar_sdp_full[b], (g / NB) & 1, ab, kDqWaitSdP);
         tc_fence_after();
+        const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
         // Probabilities are zeroed beyond the causal diagonal and, in the ragged last step, for the zero-filled keys
         // past N (which would otherwise enter the row masses).  Rows of a causal tile never reach such keys.
-        if (CAUSAL && n >= 2 * qt)                  dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, row - (n * C::kStepRows - qt * 128), rho2, msum2);
-        else if (!CAUSAL && (n + 1) * C::kStepRows > N) dq_step<true>(tS, tdP, scale_log2, neg_lse2, Dv, N - n * C::kStepRows - 1, rho2, msum2);
-        else                                        dq_step<false>(tS, tdP, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
+        const int key0 = n * C::kStepRows + C::kSliceCols * slice;   // key index of the slice's column 0
+        if (CAUSAL && n >= 2 * qt)                       dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, qrow - key0, rho2, msum2);
+        else if (!CAUSAL && (n + 1) * C::kStepRows > N)  dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, N - 1 - key0, rho2, msum2);
+        else                                             dq_slice<false>(tS16, tdP16, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&bar_tr_ready[wg]);
+        mbar_arrive(&bar_tr_ready[b]);
       }
 
       // ---- row statistics of all warpgroups (fixed order), lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
@@ -413,44 +429,41 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       float rho_t = rho_lo + rho_hi, m_t = m_lo + m_hi;
       if (wg > 0) { s_rho[wg - 1][row] = rho_t; s_m[wg - 1][row] = m_t; }
       if (C::kSepStaging && threadIdx.x == 128) bulk_wait_group_read0();   // the previous tile's stores have left the staging buffer
-      named_bar_sync(1, 128 * NB);
+      named_bar_sync(1, C::kCompute);
       if (wg == 0) {
 #pragma unroll
-        for (int w = 0; w < NB - 1; ++w) { rho_t += s_rho[w][row]; m_t += s_m[w][row]; }
+        for (int w = 0; w < C::kWG - 1; ++w) { rho_t += s_rho[w][row]; m_t += s_m[w][row]; }
         s_lam[row] = (m_t != 0.f) ? __fdiv_rn(rho_t, m_t) : 0.f;
       }
-      named_bar_sync(1, 128 * NB);
+      named_bar_sync(1, C::kCompute);
       const float lam = s_lam[row];
       const float lam_q = (flags & kFlagNoQCorrection) ? 0.f : lam;
       const float lam_k = (flags & kFlagNoKCorrection) ? 0.f : lam;
 
       mbar_wait(&bar_acc_done, ti & 1, ab, kDqWaitAcc);
       tc_fence_after();
-      // The 32-column chunks of the epilogue are dealt round-robin to the warpgroups.  Results are staged in the
+      // The 16-column chunks of the epilogue are dealt round-robin to the warpgroups.  Results are staged in the
       // TMA (128-byte swizzled) layout and written out by TMA stores: Z = -BF16(lambda q), dQ.
       uint8_t *sQt = sRes + rb * 2 * C::kBigTileBytes, *sdOt = sQt + C::kBigTileBytes;
       uint8_t *stage_dq = C::kSepStaging ? sOut : sdOt, *stage_z = C::kSepStaging ? sOut + C::kBigTileBytes : sQt;
-      constexpr int kMaxCh = (D / 32 + NB - 1) / NB;       // epilogue chunks per warpgroup
-      uint32_t a[kMaxCh][32], b[kMaxCh][32];
+      constexpr int kCh = D / (16 * C::kWG);               // 16-column epilogue chunks per warpgroup
+      uint32_t a[kCh][16], b[kCh][16];
 #pragma unroll
-      for (int nch = 0; nch < kMaxCh; ++nch) {
-        const int cc = wg + nch * NB;
-        if (cc < D / 32) {
-          tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + 32 * cc, a[nch]);
-          tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + 32 * cc, b[nch]);
-        }
+      for (int nch = 0; nch < kCh; ++nch) {
+        const int cc = wg + nch * C::kWG;
+        tmem_ld16(tmem_base + C::kColAcc0 + lane_addr + 16 * cc, a[nch]);
+        tmem_ld16(tmem_base + C::kColAcc1 + lane_addr + 16 * cc, b[nch]);
       }
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&bar_acc_free);          // the accumulators may be overwritten by the next tile
 #pragma unroll
-      for (int nch = 0; nch < kMaxCh; ++nch) {
-        const int cc = wg + nch * NB;
-        if (cc >= D / 32) break;
-        const uint32_t slab = (cc >> 1) * C::kBigSlabBytes;
+      for (int nch = 0; nch < kCh; ++nch) {
+        const int cc = wg + nch * C::kWG;
+        const uint32_t slab = (cc >> 2) * C::kBigSlabBytes;
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const uint32_t off = slab + swz128_offset(row, 4 * (cc & 1) + v);
+        for (int v = 0; v < 2; ++v) {
+          const uint32_t off = slab + swz128_offset(row, 2 * (cc & 3) + v);
           const uint4 qv = *reinterpret_cast<const uint4 *>(sQt + off);
           const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
           uint32_t dqw[4], zw[4];
@@ -468,7 +481,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         }
       }
       fence_proxy_async_smem();
-      named_bar_sync(1, 128 * NB);
+      named_bar_sync(1, C::kCompute);
       if (threadIdx.x == 128) {
         for (int sl = 0; sl < C::kSlabs; ++sl) {
           tma_store_3d(&tmdQ, stage_dq + sl * C::kBigSlabBytes, sl * 64, qt * 128, bh);
@@ -533,9 +546,9 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     mbar_init(&bar_res_full, 1);
     mbar_init(&bar_res_free, 2);
     for (int s = 0; s < S; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
-    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128); mbar_init(&bar_buf_free[b], 1); }
+    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128 * C::kSlices); mbar_init(&bar_buf_free[b], 1); }
     mbar_init(&bar_acc_done, 1);
-    mbar_init(&bar_acc_free, 128 * NB);
+    mbar_init(&bar_acc_free, C::kCompute);
     mbar_init(&bar_drain[0], 1);
     mbar_init(&bar_drain[1], 1);
     fence_mbar_init();
@@ -649,7 +662,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         tc_fence_after();
         const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes),
                        dscZ = dscdO.advanced(C::kStepTileBytes);
-        const uint32_t tR = tmem_base + 128 * b, tT = tR + 64;
+        // packed BF16 operands of query slice k (16 queries): r^T over columns 16 k .. 16 k + 7 of the buffer, t^T over the next eight
+        const uint32_t tR = tmem_base + 128 * b, tT = tR + 8;
         const uint32_t acc = (p > 0) ? 1u : 0u;
         if (elect_one_sync()) {
           if (D == 64 && use_z) {
@@ -658,21 +672,21 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
             // (an N = 64 instruction costs as much as 0.7 of an N = 128 one).  dK gets its main term t^T Q afterwards.
 #pragma unroll
             for (int k = 0; k < C::kStepRows / 16; ++k)    // [dV | dK] += r^T [dO | -BF16(lambda Q)]
-              umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_fused, k > 0 ? 1u : acc);
+              umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_fused, k > 0 ? 1u : acc);
 #pragma unroll
             for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += t^T Q
-              umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, 1u);
+              umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, 1u);
           } else {
 #pragma unroll
             for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
-              umma_ts(tmem_base + C::kColAcc0, tR + 8 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+              umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
 #pragma unroll
             for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
-              umma_ts(tmem_base + C::kColAcc1, tT + 8 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+              umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
             if (use_z) {
 #pragma unroll
               for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
-                umma_ts(tmem_base + C::kColAcc1, tR + 8 * k, dscZ.at(k * 2048), idesc_a, 1u);
+                umma_ts(tmem_base + C::kColAcc1, tR + 16 * k, dscZ.at(k * 2048), idesc_a, 1u);
             }
           }
           umma_commit(&bar_buf_free[b]);
@@ -684,42 +698,43 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     }
     drain_mmas_if_aborted(&bar_drain[1], ab);
   } else {
-    // ---------------------------------------------------------------- compute: thread <-> key row
-    const int wg = (warp - 4) >> 2;
+    // ---------------------------------------------------------------- compute: thread <-> (key row, query slice of every kGroups-th step)
+    const int wg = (warp - 4) >> 2, grp = wg / C::kSlices, slice = wg % C::kSlices;
     const int row = 32 * (warp & 3) + lane;                  // key row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
-    const uint32_t tS = tmem_base + 128 * wg + lane_addr, tdP = tS + 64;
+    const uint32_t slice_addr = tmem_base + lane_addr + C::kSliceCols * slice;
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const int kt = lin / BH, bh = lin % BH, Th = tile_steps(kt), T = G * Th;
 #ifdef GPROJ_TRACE
       const unsigned long long tile_t0 = global_ns();
 #endif
-      for (int n = (wg - g0 % NB + NB) % NB; n < T; n += NB) {
-        const int g = g0 + n, st = g % S;
-        mbar_wait(&bar_q_full[st], (g / S) & 1, ab, kDkvWaitQ);      // row statistics of this step landed
-        mbar_wait(&bar_sdp_full[wg], (g / NB) & 1, ab, kDkvWaitSdP);
+      for (int n = (grp - g0 % C::kGroups + C::kGroups) % C::kGroups; n < T; n += C::kGroups) {
+        const int g = g0 + n, st = g % S, b = g % NB;
+        // The scores of this step were issued after its stage (and with it the row statistics) had landed in shared
+        // memory, so their completion covers both.
+        mbar_wait(&bar_sdp_full[b], (g / NB) & 1, ab, kDkvWaitSdP);
         tc_fence_after();
-        const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes);
-        if (CAUSAL && (n % Th) < 2) dkv_step<true>(tS, tdP, nl, nl + 64, scale_log2, row - (n % Th) * C::kStepRows);
-        else                 dkv_step<false>(tS, tdP, nl, nl + 64, scale_log2, 0);
+        const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
+        const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes) + C::kSliceCols * slice;
+        const int nh = n % Th;                                      // step within the current query head
+        if (CAUSAL && nh < 2) dkv_slice<true>(tS16, tdP16, nl, nl + 64, scale_log2, row - nh * C::kStepRows - C::kSliceCols * slice);
+        else                  dkv_slice<false>(tS16, tdP16, nl, nl + 64, scale_log2, 0);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&bar_tr_ready[wg]);
+        mbar_arrive(&bar_tr_ready[b]);
       }
 
       mbar_wait(&bar_acc_done, ti & 1, ab, kDkvWaitAcc);
       tc_fence_after();
       uint8_t *stage_dk = C::kSepStaging ? sOut : sK, *stage_dv = C::kSepStaging ? sOut + C::kBigTileBytes : sV;
-      constexpr int kMaxCh = (D / 32 + NB - 1) / NB;       // epilogue chunks per warpgroup
-      uint32_t a[kMaxCh][32], b[kMaxCh][32];
+      constexpr int kCh = D / (16 * C::kWG);               // 16-column epilogue chunks per warpgroup
+      uint32_t a[kCh][16], b[kCh][16];
 #pragma unroll
-      for (int nch = 0; nch < kMaxCh; ++nch) {
-        const int cc = wg + nch * NB;
-        if (cc < D / 32) {
-          tmem_ld32(tmem_base + C::kColAcc0 + lane_addr + 32 * cc, a[nch]);
-          tmem_ld32(tmem_base + C::kColAcc1 + lane_addr + 32 * cc, b[nch]);
-        }
+      for (int nch = 0; nch < kCh; ++nch) {
+        const int cc = wg + nch * C::kWG;
+        tmem_ld16(tmem_base + C::kColAcc0 + lane_addr + 16 * cc, a[nch]);
+        tmem_ld16(tmem_base + C::kColAcc1 + lane_addr + 16 * cc, b[nch]);
       }
       tmem_wait_ld();
       tc_fence_before();
@@ -729,17 +744,16 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
           mbar_arrive(&bar_res_free);      // second arrival: with its own staging buffer the epilogue never touches K / V
           bulk_wait_group_read0();         // the previous tile's stores have left the staging buffer
         }
-        named_bar_sync(1, 128 * NB);
+        named_bar_sync(1, C::kCompute);
       }
       // staged in the TMA (128-byte swizzled) layout, then stored by TMA
 #pragma unroll
-      for (int nch = 0; nch < kMaxCh; ++nch) {
-        const int cc = wg + nch * NB;
-        if (cc >= D / 32) break;
-        const uint32_t slab = (cc >> 1) * C::kBigSlabBytes;
+      for (int nch = 0; nch < kCh; ++nch) {
+        const int cc = wg + nch * C::kWG;
+        const uint32_t slab = (cc >> 2) * C::kBigSlabBytes;
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const uint32_t off = slab + swz128_offset(row, 4 * (cc & 1) + v);
+        for (int v = 0; v < 2; ++v) {
+          const uint32_t off = slab + swz128_offset(row, 2 * (cc & 3) + v);
           uint32_t vw[4], kw[4];
 #pragma unroll
           for (int w = 0; w < 4; ++w) {
@@ -752,7 +766,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         }
       }
       fence_proxy_async_smem();
-      named_bar_sync(1, 128 * NB);
+      named_bar_sync(1, C::kCompute);
       if (threadIdx.x == 128) {
         for (int sl = 0; sl < C::kSlabs; ++sl) {
           tma_store_3d(&tmdV, stage_dv + sl * C::kBigSlabBytes, sl * 64, kt * 128, bh);

@@ -114,6 +114,35 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
                       unsigned fwd_flags, void *stream);
 
 /*
+ * Packed (variable-length) sequences.  The paper's synthetic suite exercises "packed segments" and "unequal lengths"
+ * (Appendix "Synthetic Numerical Suite"); its training layout packs documents into one row axis.  Here the tensors are
+ * [H][T][d] (queries, O, dO, dQ) and [Hkv][T][d] (keys, values, dK, dV) with T = cu_seqlens[num_seqs] rows per head; sequence
+ * s owns rows cu_seqlens[s] .. cu_seqlens[s+1]-1 of EVERY head, and a query attends only to keys of its own sequence
+ * (Eq. "row-attention" with the support L restricted to the sequence; causal: keys at or before it inside the sequence).
+ * LSE is [H][T].  Query and key lengths of a sequence are equal, so no row has an empty support.  Empty sequences
+ * (two equal offsets) are allowed and skipped.
+ *   - cu_seqlens is a HOST array of num_seqs + 1 non-decreasing ints starting at 0 (read during the call, not kept).
+ *   - The kernels need a tile list in DEVICE memory.  gproj_attn_varlen_plan() writes it into a HOST buffer of
+ *     gproj_attn_varlen_plan_bytes() bytes; the caller copies that buffer to 16-byte aligned device memory (any way it
+ *     likes) and passes the device pointer.  The plan depends on cu_seqlens and on `causal` (tiles are ordered by
+ *     decreasing work), not on H, d or the data; it can be reused for every layer and step with the same packing.
+ *   - Arithmetic, flags, status codes and workspace rules are those of gproj_attn_fwd_ex / gproj_attn_bwd_gqa; the
+ *     workspace size comes from gproj_attn_bwd_varlen_workspace_bytes().  Errors: GPROJ_ERR_SHAPE for a malformed
+ *     cu_seqlens (or H*T >= 2^31), GPROJ_ERR_NULL / GPROJ_ERR_ALIGN for the plan pointer, GPROJ_ERR_WORKSPACE for a plan
+ *     buffer or workspace that is too small.
+ */
+size_t gproj_attn_varlen_plan_bytes(const int *cu_seqlens, int num_seqs);
+int gproj_attn_varlen_plan(const int *cu_seqlens, int num_seqs, int causal, void *plan_host, size_t plan_bytes);
+int gproj_attn_fwd_varlen(const void *Q, const void *K, const void *V, void *O, float *LSE, const int *cu_seqlens,
+                          int num_seqs, const void *plan_device, int H, int Hkv, int d, float softmax_scale, int causal,
+                          unsigned fwd_flags, void *stream);
+size_t gproj_attn_bwd_varlen_workspace_bytes(const int *cu_seqlens, int num_seqs, int H, int d);
+int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                          void *dQ, void *dK, void *dV, const int *cu_seqlens, int num_seqs, const void *plan_device,
+                          int H, int Hkv, int d, float softmax_scale, int causal, void *workspace, size_t workspace_bytes,
+                          unsigned flags, void *stream);
+
+/*
  * Backward for callers that must not allocate device memory (the paper has no counterpart: this is a
  * convenience of this library).  Some hosts of this code cannot call cudaMalloc at the point where they
  * need a gradient: a plugin running inside another framework's memory pool, a real-time or safety-audited

@@ -10,10 +10,13 @@ from .binding import (  # noqa: F401
     FLAG_ONLY_DQ_PASS,
     FWD_FLAG_FMA_SOFTMAX,
     GprojError,
+    VarlenPlan,
     gproj_attn_bwd,
     gproj_attn_bwd_static_scratch,
+    gproj_attn_bwd_varlen,
     gproj_attn_bwd_workspace_bytes,
     gproj_attn_fwd,
+    gproj_attn_fwd_varlen,
     gproj_last_device_status,
     gproj_last_launch_count,
     gproj_selftest_wait_timeout,

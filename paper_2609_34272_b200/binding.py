@@ -23,6 +23,8 @@ STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_fwd_gqa", "gproj_attn_bwd_gqa", "gproj_attn_fwd_ex",
            "gproj_attn_bwd_static_scratch",
+           "gproj_attn_varlen_plan_bytes", "gproj_attn_varlen_plan", "gproj_attn_fwd_varlen",
+           "gproj_attn_bwd_varlen_workspace_bytes", "gproj_attn_bwd_varlen",
            "gproj_last_device_status", "gproj_selftest_wait_timeout",
            "gproj_status_string", "gproj_last_launch_count")
 
@@ -58,6 +60,17 @@ def load():
         lib.gproj_attn_bwd_gqa.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, sz, u, vp]
         lib.gproj_attn_bwd_static_scratch.restype = i
         lib.gproj_attn_bwd_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, u, vp]
+        ip = ctypes.POINTER(ctypes.c_int)
+        lib.gproj_attn_varlen_plan_bytes.restype = ctypes.c_size_t
+        lib.gproj_attn_varlen_plan_bytes.argtypes = [ip, i]
+        lib.gproj_attn_varlen_plan.restype = i
+        lib.gproj_attn_varlen_plan.argtypes = [ip, i, i, vp, ctypes.c_size_t]
+        lib.gproj_attn_fwd_varlen.restype = i
+        lib.gproj_attn_fwd_varlen.argtypes = [vp, vp, vp, vp, vp, ip, i, vp, i, i, i, f, i, u, vp]
+        lib.gproj_attn_bwd_varlen_workspace_bytes.restype = ctypes.c_size_t
+        lib.gproj_attn_bwd_varlen_workspace_bytes.argtypes = [ip, i, i, i]
+        lib.gproj_attn_bwd_varlen.restype = i
+        lib.gproj_attn_bwd_varlen.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ip, i, vp, i, i, i, f, i, vp, ctypes.c_size_t, u, vp]
         lib.gproj_selftest_wait_timeout.restype = i
         lib.gproj_selftest_wait_timeout.argtypes = [vp]
         lib.gproj_last_device_status.restype = i
@@ -202,3 +215,64 @@ def gproj_selftest_wait_timeout(device=None):
 
 def gproj_last_launch_count() -> int:
     return int(load().gproj_last_launch_count())
+
+
+class VarlenPlan:
+    """Packed-sequence description: host cu_seqlens plus the device tile list the kernels walk (built once per packing)."""
+
+    def __init__(self, cu_seqlens, causal, device="cuda"):
+        cu = [int(x) for x in cu_seqlens]
+        self.num_seqs = len(cu) - 1
+        self.cu = (ctypes.c_int * len(cu))(*cu)
+        self.causal = bool(causal)
+        self.total = cu[-1]
+        nbytes = int(load().gproj_attn_varlen_plan_bytes(self.cu, self.num_seqs))
+        if nbytes == 0 and self.total <= 0:
+            raise GprojError(-2, "gproj_attn_varlen_plan_bytes")
+        host = torch.empty(max(nbytes, 16), dtype=torch.uint8)
+        rc = load().gproj_attn_varlen_plan(self.cu, self.num_seqs, int(self.causal), ctypes.c_void_p(host.data_ptr()), nbytes)
+        if rc != GPROJ_OK:
+            raise GprojError(rc, "gproj_attn_varlen_plan")
+        self.host = host
+        self.device = host.to(device)
+
+
+def gproj_attn_fwd_varlen(Q, K, V, plan, softmax_scale, fwd_flags=0):
+    """O, LSE = forward over packed sequences.  Q: CUDA bfloat16 [H, T, d]; K, V: [Hkv, T, d]; plan: VarlenPlan."""
+    _check_bf16("Q", Q)
+    H, T, d = Q.shape
+    _check_bf16("K", K); _check_bf16("V", V, K.shape)
+    if K.dim() != 3 or K.shape[1] != T or K.shape[2] != d or H % K.shape[0] != 0 or T != plan.total:
+        raise ValueError("packed K/V must be [Hkv, T, d] with T = cu_seqlens[-1] and H a multiple of Hkv")
+    O = torch.empty_like(Q)
+    LSE = torch.empty((H, T), dtype=torch.float32, device=Q.device)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_fwd_varlen(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), plan.cu,
+                                          plan.num_seqs, plan.device.data_ptr(), H, K.shape[0], d, float(softmax_scale),
+                                          int(plan.causal), int(fwd_flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_fwd_varlen")
+    return O, LSE
+
+
+def gproj_attn_bwd_varlen(Q, K, V, O, LSE, dO, plan, softmax_scale, flags=0, workspace=None):
+    """dQ, dK, dV = backward over packed sequences (same layout as gproj_attn_fwd_varlen)."""
+    _check_bf16("Q", Q)
+    H, T, d = Q.shape
+    for name, t in (("O", O), ("dO", dO)):
+        _check_bf16(name, t, Q.shape)
+    _check_bf16("K", K); _check_bf16("V", V, K.shape)
+    if not (LSE.is_cuda and LSE.dtype == torch.float32 and LSE.is_contiguous() and tuple(LSE.shape) == (H, T)):
+        raise TypeError("LSE must be a contiguous CUDA float32 tensor [H, T]")
+    need = int(load().gproj_attn_bwd_varlen_workspace_bytes(plan.cu, plan.num_seqs, H, d))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_bwd_varlen(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
+                                          dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), plan.cu, plan.num_seqs,
+                                          plan.device.data_ptr(), H, K.shape[0], d, float(softmax_scale), int(plan.causal),
+                                          workspace.data_ptr(), workspace.numel(), int(flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_bwd_varlen")
+    return dQ, dK, dV

@@ -93,6 +93,31 @@ struct TileSched {
   }
 };
 
+// One 128-row tile of one sequence.  Rows are counted inside a head ([heads][rows][d] tensors): dense calls have one
+// sequence [0, N) per head; packed (variable-length) calls have several, listed tile by tile in a plan the host
+// prepared: {row0, seq0, seq_end, blk0} with blk0 the sequence's first 64-row block of row statistics.
+struct TileInfo { int row0, seq0, seq_end, blk0; };
+__device__ __forceinline__ TileInfo tile_info(const int4 *plan, int idx, int dense_tile, int N) {
+  if (plan != nullptr) {
+    const int4 e = __ldg(plan + idx);
+    return TileInfo{e.x, e.y, e.z, e.w};
+  }
+  return TileInfo{128 * dense_tile, 0, N, 0};
+}
+// Rows [row0, row0 + 128) may be written by a TMA store (which clips at the tensor's end N) unless the tile is the
+// ragged tail of a sequence that is followed by another one.
+__device__ __forceinline__ bool tile_store_by_tma(const TileInfo &t, int N) { return t.row0 + 128 <= t.seq_end || t.seq_end == N; }
+// Plain row-wise copy of a staged [128 x D] BF16 tile (128-byte swizzled slabs) to global memory, rows < rows_valid only.
+template <int D>
+__device__ __forceinline__ void store_rows_clipped(const uint8_t *stage, int slab_bytes, __nv_bfloat16 *dst_row0, int row, int rows_valid) {
+  if (row < rows_valid) {
+    uint4 *dst = reinterpret_cast<uint4 *>(dst_row0 + static_cast<size_t>(row) * D);
+#pragma unroll
+    for (int ch = 0; ch < D / 8; ++ch)
+      dst[ch] = *reinterpret_cast<const uint4 *>(stage + (ch >> 3) * slab_bytes + swz128_offset(row, ch & 7));
+  }
+}
+
 enum BwdWaitCode {
   kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26, kDqWaitBuf = 0x27, kDqWaitResFree = 0x28, kDqWaitAccFree = 0x29,
   kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36, kDkvWaitBuf = 0x37, kDkvWaitResFree = 0x38, kDkvWaitAccFree = 0x39
@@ -154,9 +179,10 @@ __device__ __forceinline__ void dq_slice(uint32_t tS, uint32_t tdP, float scale_
 
 // One step of the dK/dV side for one key row and one slice (32 queries) of the step's 64 queries, chunked as above.
 // `lim` = (key row) - (query index of the slice's column 0): with MASKED, column c is a query before this key when
-// c < lim.  nl / nd: the slice's per-column -LSE log2 e and -D (shared memory, same address for every lane: broadcast).
+// c < lim; `hi` = (last query of the sequence) - (query index of column 0): a column c > hi belongs to the next packed
+// sequence (or is zero fill).  nl / nd: the slice's per-column -LSE log2 e and -D (shared memory, same address for every lane: broadcast).
 template <bool MASKED>
-__device__ __forceinline__ void dkv_slice(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim) {
+__device__ __forceinline__ void dkv_slice(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim, int hi) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2);
   uint32_t xs[2][16], xp[2][16];
   tmem_ld16(tS, xs[0]);
@@ -174,10 +200,10 @@ __device__ __forceinline__ void dkv_slice(uint32_t tS, uint32_t tdP, const float
       const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);
       const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
       const int col = 16 * c + 4 * i;
-      score_pair<MASKED>(xs[c][4 * i], xs[c][4 * i + 1], xp[c][4 * i], xp[c][4 * i + 1], scale2, l4.x, d4.x, col >= lim, col + 1 >= lim,
-                         pr[2 * i], pt[2 * i]);
-      score_pair<MASKED>(xs[c][4 * i + 2], xs[c][4 * i + 3], xp[c][4 * i + 2], xp[c][4 * i + 3], scale2, l4.y, d4.y, col + 2 >= lim,
-                         col + 3 >= lim, pr[2 * i + 1], pt[2 * i + 1]);
+      score_pair<MASKED>(xs[c][4 * i], xs[c][4 * i + 1], xp[c][4 * i], xp[c][4 * i + 1], scale2, l4.x, d4.x, col >= lim && col <= hi,
+                         col + 1 >= lim && col + 1 <= hi, pr[2 * i], pt[2 * i]);
+      score_pair<MASKED>(xs[c][4 * i + 2], xs[c][4 * i + 3], xp[c][4 * i + 2], xp[c][4 * i + 3], scale2, l4.y, d4.y,
+                         col + 2 >= lim && col + 2 <= hi, col + 3 >= lim && col + 3 <= hi, pr[2 * i + 1], pt[2 * i + 1]);
     }
     tmem_st8(tS + 16 * c, pr);
     tmem_st8(tS + 16 * c + 8, pt);
@@ -197,6 +223,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const __grid_constant__ CUtensorMap tmZ,    // store, box 64 x 128 rows
               const __nv_bfloat16 *__restrict__ Og, const __nv_bfloat16 *__restrict__ dOg,
               const float *__restrict__ LSE, float *__restrict__ stats,
+              __nv_bfloat16 *__restrict__ dQg, __nv_bfloat16 *__restrict__ Zg,   // plain-store targets of clipped tiles
+              const int4 *__restrict__ plan, int nblk,                          // packed sequences: tile list; 64-row statistic blocks per head
               int N, int BH, int Hq, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
   using C = BwdCfg<D>;
   constexpr int NB = C::kNB, R = C::kDqResBufs, S = C::kDqStages;
@@ -218,7 +246,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   if (cta_skip != 0) return;   // an earlier wait gave up: drain the rest of the grid quickly
 
   // Ragged N: tiles and steps round up; rows past N load as zero (TMA fill) and are clipped on store.
-  const int n_qt = (N + 127) / 128, n64 = (N + C::kStepRows - 1) / C::kStepRows;
+  const int n_qt = (N + 127) / 128;
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
@@ -243,21 +271,26 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 
   TileSched sched(total_tiles);
   // tile decode: causal -> longest rows first
-  auto tile_qt = [&](int lin) { return CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH); };
-  auto tile_steps = [&](int qt) { return CAUSAL ? min(2 * (qt + 1), n64) : n64; };
+  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH), N); };
+  // 64-key steps of a query tile: its sequence's keys up to the tile's last row (causal) or all of them
+  auto steps_of = [&](const TileInfo &t) {
+    const int kend = CAUSAL ? min(t.row0 + 128, t.seq_end) : t.seq_end;
+    return (kend - t.seq0 + C::kStepRows - 1) / C::kStepRows;
+  };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (K, V) step tiles
     if (lane == 0) {
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
-        const int qt = tile_qt(lin), bh = lin % BH, T = tile_steps(qt);
+        const TileInfo tl = tile_of(lin);
+        const int bh = lin % BH, T = steps_of(tl);
         for (int n = 0; n < T; ++n, ++g) {
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kDqWaitKVEmpty);
           mbar_expect_tx(&bar_kv_full[st], C::kDqStageBytes);
           uint8_t *dst = sKV + st * C::kDqStageBytes;
-          const int kvh = kv_head_of(bh, Hq, G), krow = n * C::kStepRows;   // grouped-query: the group's shared K / V head
+          const int kvh = kv_head_of(bh, Hq, G), krow = tl.seq0 + n * C::kStepRows;   // grouped-query: the group's shared K / V head
           for (int s = 0; s < C::kSlabs; ++s) {
             tma_load_3d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow, kvh);
             tma_load_3d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow, kvh);
@@ -276,7 +309,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int rb = ti % R, bh = lin % BH, qrow0 = tile_qt(lin) * 128;
+        const int rb = ti % R, bh = lin % BH, qrow0 = tile_of(lin).row0;
         if (ti >= R) mbar_wait(&bar_res_free[rb], ((ti / R) - 1) & 1, ab, kDqWaitResFree);
         mbar_expect_tx(&bar_res_full[rb], 2 * C::kBigTileBytes);
         uint8_t *dst = sRes + rb * 2 * C::kBigTileBytes;
@@ -299,7 +332,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     const SmemDesc dscK0 = make_smem_desc(smem_u32(sKV), 16, 1024);                          // K-major view of stage 0
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int T = tile_steps(tile_qt(lin)), rb = ti % R;
+      const int T = steps_of(tile_of(lin)), rb = ti % R;
       mbar_wait(&bar_res_full[rb], (ti / R) & 1, ab, kDqWaitQ);
       const SmemDesc dscQ = dscRes0.advanced(rb * 2 * C::kBigTileBytes), dscdO = dscQ.advanced(C::kBigTileBytes);
       for (int n = 0; n < T; ++n, ++g) {
@@ -333,7 +366,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     const SmemDesc dscK0mn = make_smem_desc(smem_u32(sKV), C::kStepSlabBytes, 1024);       // MN-major view of stage 0
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int T = tile_steps(tile_qt(lin));
+      const int T = steps_of(tile_of(lin));
       if (ti > 0) mbar_wait(&bar_acc_free, (ti - 1) & 1, ab, kDqWaitAccFree);   // the previous epilogue has read A, B
       for (int p = 0; p < T; ++p, ++g) {
         const int st = g % S, b = g % NB;
@@ -366,9 +399,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     const uint32_t slice_addr = tmem_base + lane_addr + C::kSliceCols * slice;
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int qt = tile_qt(lin), bh = lin % BH, T = tile_steps(qt), rb = ti % R;
+      const TileInfo tl = tile_of(lin);
+      const int bh = lin % BH, T = steps_of(tl), rb = ti % R;
       const size_t head_row0 = static_cast<size_t>(bh) * N;
-      const int qrow = qt * 128 + row;                 // this thread's query row within the head (may be >= N in a ragged tile)
+      const int qrow = tl.row0 + row;                  // this thread's query row within the head (past seq_end in a ragged tile)
 
       // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1): each of the 16 compute warps
       // takes eight rows, coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
@@ -379,9 +413,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         for (int it = 0; it < 8 / RPI; ++it) {
           const int r = 8 * (warp - 4) + it * RPI + sub;
           uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-          if (qt * 128 + r < N) {
-            a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + qt * 128 + r) * D) + part);
-            b = __ldg(reinterpret_cast<const uint4 *>(dOg + (head_row0 + qt * 128 + r) * D) + part);
+          if (tl.row0 + r < tl.seq_end) {
+            a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + tl.row0 + r) * D) + part);
+            b = __ldg(reinterpret_cast<const uint4 *>(dOg + (head_row0 + tl.row0 + r) * D) + part);
           }
           const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
           float acc = 0.f;
@@ -397,10 +431,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
       named_bar_sync(2, C::kCompute);
       const float Dv = s_D[row];
-      const float neg_lse2 = (qrow < N) ? -LSE[head_row0 + qrow] * 1.4426950408889634f : 0.f;
-      // Per 64-row block of a head (n64 blocks, the last one padded with zeros): 64 x {-LSE log2 e}, then 64 x {-D}.
-      if (wg == 0 && qrow < n64 * C::kStepRows) {
-        float *blk = stats + (static_cast<size_t>(bh) * n64 + (qrow >> 6)) * 128 + (qrow & 63);
+      const float neg_lse2 = (qrow < tl.seq_end) ? -LSE[head_row0 + qrow] * 1.4426950408889634f : 0.f;
+      // Per 64-row block of a sequence (the last one padded with zeros): 64 x {-LSE log2 e}, then 64 x {-D}.
+      const int rel = qrow - tl.seq0;                  // row inside the sequence
+      if (wg == 0 && rel < ((tl.seq_end - tl.seq0 + C::kStepRows - 1) / C::kStepRows) * C::kStepRows) {
+        float *blk = stats + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * 128 + (rel & 63);
         blk[0] = neg_lse2;
         blk[64] = -Dv;
       }
@@ -413,9 +448,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
         // Probabilities are zeroed beyond the causal diagonal and, in the ragged last step, for the zero-filled keys
         // past N (which would otherwise enter the row masses).  Rows of a causal tile never reach such keys.
-        const int key0 = n * C::kStepRows + C::kSliceCols * slice;   // key index of the slice's column 0
-        if (CAUSAL && n >= 2 * qt)                       dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, qrow - key0, rho2, msum2);
-        else if (!CAUSAL && (n + 1) * C::kStepRows > N)  dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, N - 1 - key0, rho2, msum2);
+        const int key0 = tl.seq0 + n * C::kStepRows + C::kSliceCols * slice;   // row (inside the head) of the slice's column 0
+        if (CAUSAL && (n + 1) * C::kStepRows > tl.row0 - tl.seq0)              dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, qrow - key0, rho2, msum2);
+        else if (!CAUSAL && tl.seq0 + (n + 1) * C::kStepRows > tl.seq_end)     dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, tl.seq_end - 1 - key0, rho2, msum2);
         else                                             dq_slice<false>(tS16, tdP16, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
         tmem_wait_st();
         tc_fence_before();
@@ -482,14 +517,22 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
       fence_proxy_async_smem();
       named_bar_sync(1, C::kCompute);
-      if (threadIdx.x == 128) {
-        for (int sl = 0; sl < C::kSlabs; ++sl) {
-          tma_store_3d(&tmdQ, stage_dq + sl * C::kBigSlabBytes, sl * 64, qt * 128, bh);
-          tma_store_3d(&tmZ, stage_z + sl * C::kBigSlabBytes, sl * 64, qt * 128, bh);
+      if (tile_store_by_tma(tl, N)) {
+        if (threadIdx.x == 128) {
+          for (int sl = 0; sl < C::kSlabs; ++sl) {
+            tma_store_3d(&tmdQ, stage_dq + sl * C::kBigSlabBytes, sl * 64, tl.row0, bh);
+            tma_store_3d(&tmZ, stage_z + sl * C::kBigSlabBytes, sl * 64, tl.row0, bh);
+          }
+          bulk_commit_group();
+          if (!C::kSepStaging) bulk_wait_group_read0();   // staging shares the Q / dO buffer: reads must finish first
+          mbar_arrive(&bar_res_free[rb]);                 // second arrival: the epilogue no longer needs this buffer
         }
-        bulk_commit_group();
-        if (!C::kSepStaging) bulk_wait_group_read0();     // staging shares the Q / dO buffer: reads must finish first
-        mbar_arrive(&bar_res_free[rb]);                   // second arrival: the epilogue no longer needs this buffer
+      } else {
+        // ragged last tile of a packed sequence that another sequence follows: rows past its end are not ours to write
+        if (wg < 2) store_rows_clipped<D>(wg == 0 ? stage_dq : stage_z, C::kBigSlabBytes,
+                                         (wg == 0 ? dQg : Zg) + (head_row0 + tl.row0) * D, row, tl.seq_end - tl.row0);
+        named_bar_sync(1, C::kCompute);
+        if (threadIdx.x == 128) mbar_arrive(&bar_res_free[rb]);
       }
       g0 += T;
     }
@@ -514,6 +557,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmdK,   // store, box 64 x 128 rows
                const __grid_constant__ CUtensorMap tmdV,   // store, box 64 x 128 rows
                const float *__restrict__ stats,
+               __nv_bfloat16 *__restrict__ dKg, __nv_bfloat16 *__restrict__ dVg,   // plain-store targets of clipped tiles
+               const int4 *__restrict__ plan, int nblk,                           // packed sequences: tile list; statistic blocks per head
                int N, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
   // BH counts (batch, KV head) pairs here.  With grouped queries (G > 1) one work item walks the query steps of all G
   // query heads of its KV head, so their contributions are summed in the FP32 accumulators (Section 3.1: key and value
@@ -567,16 +612,18 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   // tile decode: causal -> key tile 0 has the most query steps and comes first
   // Ragged N: query steps round up.  A zero-filled query column past N contributes exactly nothing (its dO, Q and Z rows
   // are zero and its padded statistics are zero, so t = 0 and r multiplies zero rows); key rows past N are clipped on store.
-  const int n64 = (N + C::kStepRows - 1) / C::kStepRows;
-  auto tile_q_start = [&](int kt) { return CAUSAL ? kt * 128 : 0; };
-  auto tile_steps = [&](int kt) { return n64 - tile_q_start(kt) / C::kStepRows; };
+  // In a packed layout the query columns past the end of the sequence are the next sequence's rows and are masked.
+  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, lin / BH, N); };
+  auto q_start_of = [&](const TileInfo &t) { return CAUSAL ? t.row0 : t.seq0; };          // first query row that sees this key tile
+  auto steps_of = [&](const TileInfo &t) { return (t.seq_end - q_start_of(t) + C::kStepRows - 1) / C::kStepRows; };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (Q, dO, Z, stats) step tiles
     if (lane == 0) {
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
-        const int kt = lin / BH, bh = lin % BH, T = tile_steps(kt), q_start = tile_q_start(kt);
+        const TileInfo tl = tile_of(lin);
+        const int bh = lin % BH, T = steps_of(tl), q_start = q_start_of(tl);
         const int q_head0 = (bh / Hkv) * (Hkv * G) + (bh % Hkv) * G;     // first query head of the group (flat index)
         for (int n = 0; n < G * T; ++n, ++g) {
           const int st = g % S;
@@ -589,7 +636,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
             tma_load_3d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow, qh);
             if (use_z) tma_load_3d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow, qh);
           }
-          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + (static_cast<size_t>(qh) * n64 + (qrow >> 6)) * 128, 512, &bar_q_full[st]);
+          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + (static_cast<size_t>(qh) * nblk + tl.blk0 + ((qrow - tl.seq0) >> 6)) * 128, 512, &bar_q_full[st]);
         }
       }
       if (cta_abort) {
@@ -602,7 +649,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int bh = lin % BH, krow0 = (lin / BH) * 128;
+        const int bh = lin % BH, krow0 = tile_of(lin).row0;
         if (ti >= 1) mbar_wait(&bar_res_free, (ti - 1) & 1, ab, kDkvWaitResFree);
         mbar_expect_tx(&bar_res_full, 2 * C::kBigTileBytes);
         for (int s = 0; s < C::kSlabs; ++s) {
@@ -620,7 +667,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);                       // K-major view of stage 0
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int T = G * tile_steps(lin / BH);
+      const int T = G * steps_of(tile_of(lin));
       mbar_wait(&bar_res_full, ti & 1, ab, kDkvWaitKV);
       for (int n = 0; n < T; ++n, ++g) {
         const int st = g % S, b = g % NB;
@@ -654,7 +701,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     const SmemDesc dscQ0mn = make_smem_desc(smem_u32(sStage), C::kStepSlabBytes, 1024);    // MN-major view of stage 0
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int T = G * tile_steps(lin / BH);
+      const int T = G * steps_of(tile_of(lin));
       if (ti > 0) mbar_wait(&bar_acc_free, (ti - 1) & 1, ab, kDkvWaitAccFree);   // the previous epilogue has read dV, dK
       for (int p = 0; p < T; ++p, ++g) {
         const int st = g % S, b = g % NB;
@@ -705,7 +752,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     const uint32_t slice_addr = tmem_base + lane_addr + C::kSliceCols * slice;
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int kt = lin / BH, bh = lin % BH, Th = tile_steps(kt), T = G * Th;
+      const TileInfo tl = tile_of(lin);
+      const int bh = lin % BH, Th = steps_of(tl), T = G * Th, q_start = q_start_of(tl);
 #ifdef GPROJ_TRACE
       const unsigned long long tile_t0 = global_ns();
 #endif
@@ -718,8 +766,11 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
         const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes) + C::kSliceCols * slice;
         const int nh = n % Th;                                      // step within the current query head
-        if (CAUSAL && nh < 2) dkv_slice<true>(tS16, tdP16, nl, nl + 64, scale_log2, row - nh * C::kStepRows - C::kSliceCols * slice);
-        else                  dkv_slice<false>(tS16, tdP16, nl, nl + 64, scale_log2, 0);
+        const int q0 = q_start + nh * C::kStepRows + C::kSliceCols * slice;   // query row (inside the head) of the slice's column 0
+        if ((CAUSAL && nh < 2) || q_start + (nh + 1) * C::kStepRows > tl.seq_end)
+          dkv_slice<true>(tS16, tdP16, nl, nl + 64, scale_log2, CAUSAL ? tl.row0 + row - q0 : 0, tl.seq_end - 1 - q0);
+        else
+          dkv_slice<false>(tS16, tdP16, nl, nl + 64, scale_log2, 0, 0);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar_tr_ready[b]);
@@ -767,19 +818,27 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       }
       fence_proxy_async_smem();
       named_bar_sync(1, C::kCompute);
-      if (threadIdx.x == 128) {
-        for (int sl = 0; sl < C::kSlabs; ++sl) {
-          tma_store_3d(&tmdV, stage_dv + sl * C::kBigSlabBytes, sl * 64, kt * 128, bh);
-          tma_store_3d(&tmdK, stage_dk + sl * C::kBigSlabBytes, sl * 64, kt * 128, bh);
-        }
-        bulk_commit_group();
-        if (!C::kSepStaging) {             // staging shares the K / V tile: its reads must finish before the next load
-          bulk_wait_group_read0();
-          mbar_arrive(&bar_res_free);
-        }
+      if (tile_store_by_tma(tl, N)) {
+        if (threadIdx.x == 128) {
+          for (int sl = 0; sl < C::kSlabs; ++sl) {
+            tma_store_3d(&tmdV, stage_dv + sl * C::kBigSlabBytes, sl * 64, tl.row0, bh);
+            tma_store_3d(&tmdK, stage_dk + sl * C::kBigSlabBytes, sl * 64, tl.row0, bh);
+          }
+          bulk_commit_group();
+          if (!C::kSepStaging) {           // staging shares the K / V tile: its reads must finish before the next load
+            bulk_wait_group_read0();
+            mbar_arrive(&bar_res_free);
+          }
 #ifdef GPROJ_TRACE
-        tile_trace(lin, tile_t0, global_ns());
+          tile_trace(lin, tile_t0, global_ns());
 #endif
+        }
+      } else {
+        // ragged last tile of a packed sequence that another sequence follows: rows past its end are not ours to write
+        if (wg < 2) store_rows_clipped<D>(wg == 0 ? stage_dk : stage_dv, C::kBigSlabBytes,
+                                         (wg == 0 ? dKg : dVg) + (static_cast<size_t>(bh) * N + tl.row0) * D, row, tl.seq_end - tl.row0);
+        named_bar_sync(1, C::kCompute);
+        if (!C::kSepStaging && threadIdx.x == 128) mbar_arrive(&bar_res_free);
       }
       g0 += T;
     }

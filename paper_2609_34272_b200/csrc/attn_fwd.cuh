@@ -79,7 +79,7 @@ template <int D, bool CAUSAL, bool FMA_SOFTMAX, bool TURNS>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float *__restrict__ LSE, int N, int BH, int Hq, int G, int tiles_per_item, int total_items, float scale_log2, float alpha,
+                __nv_bfloat16 *__restrict__ Og, const int4 *__restrict__ plan, float *__restrict__ LSE, int N, int BH, int Hq, int G, int tiles_per_item, int total_items, float scale_log2, float alpha,
                 int *status) {
   using C = FwdCfg<D>;
   constexpr int S = C::kStages;
@@ -120,24 +120,37 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);   // the shuffle marks it warp-uniform
 
-  // Work items ordered by decreasing work (causal: last pair first).  Item -> (pair index, head).
+  // Work items ordered by decreasing work (causal: last pair first).  Item -> (sequence, first query tile, tiles) and head.
+  // Dense calls: one sequence [0, N) per head, items are pairs (or single tiles); packed calls: single tiles from the plan.
+  struct Item { int seq0, len, qt0, nq, n_kt; };   // qt0: index of the first query tile inside its sequence; nq: query tiles; n_kt: key tiles walked
   TileSched sched(total_items);
-  auto item_pair = [&](int lin) { return CAUSAL ? (n_pairs - 1 - lin / BH) : (lin / BH); };
-  auto n_steps = [&](int pair) { return CAUSAL ? min(TPI * pair + TPI, n_qt) : n_qt; };   // key tiles walked by the item
+  auto decode = [&](int lin) {
+    Item it;
+    if (plan != nullptr) {
+      const TileInfo ti = tile_info(plan, lin / BH, 0, N);
+      it.seq0 = ti.seq0; it.len = ti.seq_end - ti.seq0; it.qt0 = (ti.row0 - ti.seq0) / C::kBlockM; it.nq = 1;
+    } else {
+      const int pair = CAUSAL ? (n_pairs - 1 - lin / BH) : (lin / BH);
+      it.seq0 = 0; it.len = N; it.qt0 = TPI * pair; it.nq = min(TPI, n_qt - it.qt0);
+    }
+    it.n_kt = CAUSAL ? it.qt0 + it.nq : (it.len + C::kBlockN - 1) / C::kBlockN;
+    return it;
+  };
   // query tile t of the item takes part in key step j?
-  auto active = [&](int pair, int t, int j) { return t < TPI && (TPI * pair + t < n_qt) && (!CAUSAL || j <= TPI * pair + t); };
+  auto active = [&](const Item &it, int t, int j) { return t < it.nq && (!CAUSAL || j <= it.qt0 + t); };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of K_j, V_j
     if (lane == 0) {
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
-        const int pair = item_pair(lin), bh = lin % BH, T = n_steps(pair);
+        const Item it = decode(lin);
+        const int bh = lin % BH, T = it.n_kt;
         for (int j = 0; j < T; ++j, ++g) {
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kFwdWaitKVEmpty);
           uint8_t *dK = sKV + st * 2 * C::kTileBytes, *dV = dK + C::kTileBytes;
-          const int kvh = kv_head_of(bh, Hq, G), krow = j * C::kBlockN;   // grouped-query: the group's shared K / V head
+          const int kvh = kv_head_of(bh, Hq, G), krow = it.seq0 + j * C::kBlockN;   // grouped-query: the group's shared K / V head
           mbar_expect_tx(&bar_k_full[st], C::kTileBytes);
           for (int s = 0; s < C::kSlabs; ++s) tma_load_3d(dK + s * C::kSlabBytes, &tmK, &bar_k_full[st], s * 64, krow, kvh);
           mbar_expect_tx(&bar_v_full[st], C::kTileBytes);
@@ -158,13 +171,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int pair = item_pair(lin), bh = lin % BH;
-        const int tiles = (TPI == 2 && 2 * pair + 1 < n_qt) ? 2 : 1;
+        const Item it = decode(lin);
+        const int bh = lin % BH, tiles = it.nq;
         if (ti >= 1) mbar_wait(&bar_q_free, (ti - 1) & 1, ab, kFwdWaitQFree);
         mbar_expect_tx(&bar_q_full, tiles * C::kTileBytes);
         for (int t = 0; t < tiles; ++t)
           for (int s = 0; s < C::kSlabs; ++s)
-            tma_load_3d(sQ + t * C::kTileBytes + s * C::kSlabBytes, &tmQ, &bar_q_full, s * 64, (TPI * pair + t) * C::kBlockM, bh);
+            tma_load_3d(sQ + t * C::kTileBytes + s * C::kSlabBytes, &tmQ, &bar_q_full, s * 64, it.seq0 + (it.qt0 + t) * C::kBlockM, bh);
       }
       if (cta_abort && ti > 0)
         for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full, (ti - 1) & 1); ++spin) {}
@@ -178,7 +191,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const SmemDesc dscK0 = make_smem_desc(smem_u32(sKV), 16, 1024);
     int g = 0, ti = 0, cnt[2] = {0, 0};
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int pair = item_pair(lin), T = n_steps(pair);
+      const Item it = decode(lin);
+      const int T = it.n_kt;
       mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
       for (int j = 0; j < T; ++j, ++g) {
         const int st = g % S;
@@ -186,7 +200,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const SmemDesc dscK = dscK0.advanced(st * 2 * C::kTileBytes);
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-          if (!active(pair, t, j)) continue;
+          if (!active(it, t, j)) continue;
           // S_t may be overwritten once its previous contents are dead: copied to registers by the softmax (P~ has its
           // own columns), or, when P~ lives in the same columns, consumed by the previous P~V product.
           if (cnt[t] > 0) {
@@ -215,14 +229,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const SmemDesc dscV0 = make_smem_desc(smem_u32(sKV + C::kTileBytes), C::kSlabBytes, 1024);
     int g = 0, ti = 0, cnt[2] = {0, 0};
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const int pair = item_pair(lin), T = n_steps(pair);
+      const Item it = decode(lin);
+      const int T = it.n_kt;
       for (int j = 0; j < T; ++j, ++g) {
         const int st = g % S;
         mbar_wait(&bar_v_full[st], (g / S) & 1, ab, kFwdWaitV);
         const SmemDesc dscV = dscV0.advanced(st * 2 * C::kTileBytes);
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-          if (!active(pair, t, j)) continue;
+          if (!active(it, t, j)) continue;
           if (j == 0 && ti > 0) mbar_wait(&bar_o_free[t], (ti - 1) & 1, ab, kFwdWaitOFree);   // previous epilogue has read O_t
           mbar_wait(&bar_p_ready[t], cnt[t] & 1, ab, kFwdWaitP);
           tc_fence_after();
@@ -254,9 +269,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // With single-tile items the second warpgroup has nothing to do for the whole launch (and bar_q_free expects one
     // arrival per item only).
     for (int lin = (t < TPI) ? sched.next() : -1; lin >= 0; lin = sched.next(), ++ti) {
-      const int pair = item_pair(lin), bh = lin % BH, T = n_steps(pair);
-      const int qt = TPI * pair + t;
-      if (qt >= n_qt) {
+      const Item it = decode(lin);
+      const int bh = lin % BH, T = it.n_kt;
+      const int qt = it.qt0 + t;                      // this warpgroup's query tile inside the sequence
+      if (t >= it.nq) {
         // Odd number of query tiles: the last pair has no second tile.  Stay in step with the item (its Q has landed)
         // before handing back this slot, so that no barrier runs ahead of the roles that wait on it.
         mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
@@ -266,9 +282,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       float m_run = -INFINITY, l_run = 0.f;
       // Both tiles of the pair exist: the warpgroups alternate in the exponential phase, step by step, tile 0 first.
-      const bool take_turns = TURNS && (TPI == 2) && (2 * pair + 1 < n_qt);
+      const bool take_turns = TURNS && it.nq == 2;
       for (int j = 0; j < T; ++j) {
-        if (!active(pair, t, j)) {
+        if (!active(it, t, j)) {
           // no work in this step (causal: the first tile of the pair ends one key tile earlier): pass the turn on
           if (take_turns) {
             if (t == 1 || turn > 0) mbar_wait(&bar_turn[t], (t == 1 ? turn : turn - 1) & 1, ab, kFwdWaitTurn);
@@ -285,9 +301,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tmem_wait_ld();
         if (C::kSepP) { tc_fence_before(); mbar_arrive(&bar_s_free[t]); }   // the next S_t may be issued while this one is in the ALUs
         // Keys beyond the causal diagonal, and the zero-filled columns past the last key of a ragged tile, get -inf.
-        const bool diag = CAUSAL && j == qt, tail = (j == n_qt - 1) && (N % C::kBlockN != 0);
+        const bool diag = CAUSAL && j == qt, tail = (j + 1) * C::kBlockN > it.len;
         if (diag || tail) {
-          const int lim = min(diag ? row : C::kBlockN - 1, tail ? N - j * C::kBlockN - 1 : C::kBlockN - 1);
+          const int lim = min(diag ? row : C::kBlockN - 1, tail ? it.len - j * C::kBlockN - 1 : C::kBlockN - 1);
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
@@ -365,14 +381,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       tc_fence_before();
       mbar_arrive(&bar_o_free[t]);                     // O_t may be overwritten by the next work item
-      if (qt * C::kBlockM + row < N) LSE[static_cast<size_t>(bh) * N + qt * C::kBlockM + row] = fmaf(m_run, alpha, logf(l_run));
+      const int qrow0 = it.seq0 + qt * C::kBlockM;      // first row of the tile inside the head
+      if (qt * C::kBlockM + row < it.len) LSE[static_cast<size_t>(bh) * N + qrow0 + row] = fmaf(m_run, alpha, logf(l_run));
       fence_proxy_async_smem();
       named_bar_sync(1 + t, 128);
-      if (row == 0) {
-        for (int sl = 0; sl < C::kSlabs; ++sl) tma_store_3d(&tmO, stage + sl * C::kSlabBytes, sl * 64, qt * C::kBlockM, bh);
-        bulk_commit_group();
-        bulk_wait_group_read0();
-        mbar_arrive(&bar_q_free);                      // this tile's half of the Q buffer may be reloaded
+      const TileInfo tinfo{qrow0, it.seq0, it.seq0 + it.len, 0};
+      if (tile_store_by_tma(tinfo, N)) {
+        if (row == 0) {
+          for (int sl = 0; sl < C::kSlabs; ++sl) tma_store_3d(&tmO, stage + sl * C::kSlabBytes, sl * 64, qrow0, bh);
+          bulk_commit_group();
+          bulk_wait_group_read0();
+          mbar_arrive(&bar_q_free);                    // this tile's half of the Q buffer may be reloaded
+        }
+      } else {
+        // ragged last tile of a packed sequence that another sequence follows: rows past its end are not ours to write
+        store_rows_clipped<D>(stage, C::kSlabBytes, Og + (static_cast<size_t>(bh) * N + qrow0) * D, row, it.len - qt * C::kBlockM);
+        named_bar_sync(1 + t, 128);
+        if (row == 0) mbar_arrive(&bar_q_free);
       }
     }
   }

@@ -4,7 +4,9 @@
 
 #include <cmath>
 #include <cstdint>
+#include <algorithm>
 #include <mutex>
+#include <vector>
 
 #include "attn_bwd.cuh"
 #include "attn_fwd.cuh"
@@ -124,6 +126,13 @@ int check_shape(int B, int H, int N, int d) {
 
 size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
+int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N, int d,
+               float softmax_scale, int causal, unsigned fwd_flags, const int4 *plan, int n_plan_tiles, void *stream);
+int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+               void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+               void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
+               int n_plan_tiles, int nblk, void *stream);
+
 // Row statistics {-LSE log2 e, -D}: per head ceil(N / 64) blocks of 64 rows (the last one zero-padded), 512 B each.
 size_t stats_bytes(int heads, int N) { return align256(static_cast<size_t>(heads) * ((N + 63) / 64) * 512); }
 
@@ -143,6 +152,17 @@ int gproj_attn_fwd_gqa(const void *Q, const void *K, const void *V, void *O, flo
 
 int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N,
                       int d, float softmax_scale, int causal, unsigned fwd_flags, void *stream) {
+  return launch_fwd(Q, K, V, O, LSE, B, H, Hkv, N, d, softmax_scale, causal, fwd_flags, nullptr, 0, stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+// Dense call: plan == nullptr, one sequence [0, N) per head.  Packed call: B = 1, N = total tokens, plan = device tile
+// list (query order) with n_plan_tiles entries.
+int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N, int d,
+               float softmax_scale, int causal, unsigned fwd_flags, const int4 *plan, int n_plan_tiles, void *stream) {
   if (!Q || !K || !V || !O || !LSE) return GPROJ_ERR_NULL;
   if (fwd_flags & ~GPROJ_FWD_FLAG_FMA_SOFTMAX) return GPROJ_ERR_FLAGS;
   const bool fma = (fwd_flags & GPROJ_FWD_FLAG_FMA_SOFTMAX) != 0;
@@ -164,14 +184,16 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
   // One work item = a pair of query tiles of one head (two softmax warpgroups ping-pong on the tensor core); when
   // that leaves too few items to balance the SMs, items are single tiles.
-  const int n_qt = (N + 127) / 128;
-  const int tiles_per_item = (static_cast<long long>(BH) * ((n_qt + 1) / 2) * 2 >= 3LL * st->sm_count) ? 2 : 1;
+  const int n_qt = plan ? n_plan_tiles : (N + 127) / 128;
+  const int tiles_per_item = (!plan && static_cast<long long>(BH) * ((n_qt + 1) / 2) * 2 >= 3LL * st->sm_count) ? 2 : 1;
   const int total_items = BH * ((n_qt + tiles_per_item - 1) / tiles_per_item);
+  if (total_items <= 0) return GPROJ_OK;   // nothing but empty sequences
   const dim3 grid(static_cast<unsigned>(total_items < st->sm_count ? total_items : st->sm_count));   // persistent
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define GPROJ_LAUNCH_FWD(DD, CC, FF, TT)                                                                            \
   attn_fwd_kernel<DD, CC, FF, TT><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(                         \
-      mQ, mK, mV, mO, LSE, N, BH, H, G, tiles_per_item, total_items, scale_log2, softmax_scale, st->status_ptr)
+      mQ, mK, mV, mO, static_cast<__nv_bfloat16 *>(O), plan, LSE, N, BH, H, G, tiles_per_item, total_items, scale_log2,      \
+      softmax_scale, st->status_ptr)
 #define GPROJ_LAUNCH_FWD_C(DD, FF, TT)                                                                              \
   do { if (causal) GPROJ_LAUNCH_FWD(DD, true, FF, TT); else GPROJ_LAUNCH_FWD(DD, false, FF, TT); } while (0)
   // the softmax warpgroups alternate in the exponential phase where that was measured to pay: d = 128, paired tiles
@@ -186,6 +208,10 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
   tl_launch_count = 1;
   return GPROJ_OK;
 }
+
+}  // namespace
+
+extern "C" {
 
 size_t gproj_attn_bwd_workspace_bytes(int B, int H, int N, int d) {
   if (check_shape(B, H, N, d) != GPROJ_OK) return 0;
@@ -202,6 +228,20 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
 int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
                        void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
                        void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
+  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, Hkv, N, d, softmax_scale, causal, workspace, workspace_bytes, flags,
+                    nullptr, nullptr, 0, (N + 63) / 64, stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+// Dense call: plans == nullptr.  Packed call: B = 1, N = total tokens, plan_q / plan_kv = device tile lists in the order
+// of the dQ-side and the dK/dV-side kernel, nblk = 64-row statistic blocks per head.
+int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+               void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+               void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
+               int n_plan_tiles, int nblk, void *stream) {
   if (!Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return GPROJ_ERR_NULL;
   if (int rc = check_shape(B, H, N, d)) return rc;
   if (Hkv <= 0 || H % Hkv != 0) return GPROJ_ERR_SHAPE;
@@ -214,15 +254,16 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
     return GPROJ_ERR_FLAGS;
   const bool run_dq = !(flags & GPROJ_FLAG_ONLY_DKV_PASS), run_dkv = !(flags & GPROJ_FLAG_ONLY_DQ_PASS);
   if (!run_dq && !run_dkv) return GPROJ_ERR_FLAGS;
+  const size_t stats_sz = align256(static_cast<size_t>(B) * H * nblk * 512);
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-      workspace_bytes < gproj_attn_bwd_workspace_bytes(B, H, N, d))
+      workspace_bytes < stats_sz + align256(static_cast<size_t>(B) * H * N * static_cast<size_t>(d) * 2))
     return GPROJ_ERR_WORKSPACE;
   DeviceState *st = nullptr;
   if (int rc = device_state(&st)) return rc;
 
   const int BH = B * H, BHkv = B * Hkv;
   float *stats = static_cast<float *>(workspace);   // per 64-row block: 64 x {-LSE log2 e}, 64 x {-D}
-  __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + stats_bytes(BH, N));
+  __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + stats_sz);
 
   CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64, mdQst, mZst, mdKst, mdVst;
   bool ok = make_map(&mQ128, Q, BH, N, d, 128) && make_map(&mdO128, dO, BH, N, d, 128) && make_map(&mK64, K, BHkv, N, d, 64) &&
@@ -233,7 +274,8 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
   if (!ok) return GPROJ_ERR_CUDA;
 
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
-  const int n_qt = (N + 127) / 128, total_tiles = BH * n_qt, total_kv_tiles = BHkv * n_qt;
+  const int n_qt = plan_q ? n_plan_tiles : (N + 127) / 128, total_tiles = BH * n_qt, total_kv_tiles = BHkv * n_qt;
+  if (total_tiles <= 0) return GPROJ_OK;   // nothing but empty sequences
   const dim3 grid(static_cast<unsigned>(total_tiles < st->sm_count ? total_tiles : st->sm_count));   // persistent: one CTA per SM
   const dim3 grid_kv(static_cast<unsigned>(total_kv_tiles < st->sm_count ? total_kv_tiles : st->sm_count));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -242,12 +284,14 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
   do {                                                                                                                  \
     if (run_dq)                                                                                                         \
       bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                               \
-          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, N, BH, H, G, total_tiles, scale_log2, softmax_scale,   \
+          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, static_cast<__nv_bfloat16 *>(dQ), Zneg, plan_q, nblk,   \
+          N, BH, H, G, total_tiles, scale_log2, softmax_scale,                                                        \
           flags,                                                                                                        \
           st->status_ptr);                                                                                              \
     if (run_dkv)                                                                                                        \
       bwd_dkv_kernel<DD, CC><<<grid_kv, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
-          mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,   \
+          mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, static_cast<__nv_bfloat16 *>(dK),                        \
+          static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,     \
           flags,                                                                                                        \
           st->status_ptr);                                                                                              \
   } while (0)
@@ -257,6 +301,104 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
   if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
   tl_launch_count = (run_dq ? 1 : 0) + (run_dkv ? 1 : 0);
   return GPROJ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---- packed (variable-length) sequences ------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+
+struct PackedShape { int total, n_tiles, nblk; };
+
+// cu_seqlens: num_seqs + 1 non-decreasing row offsets, the first one 0.  Empty sequences are allowed and skipped.
+bool packed_shape(const int *cu, int num_seqs, PackedShape *out) {
+  if (!cu || num_seqs <= 0 || cu[0] != 0) return false;
+  long long tiles = 0, blocks = 0;
+  for (int s = 0; s < num_seqs; ++s) {
+    const long long len = static_cast<long long>(cu[s + 1]) - cu[s];
+    if (len < 0) return false;
+    tiles += (len + 127) / 128;
+    blocks += (len + 63) / 64;
+  }
+  if (cu[num_seqs] <= 0 || tiles >= (1LL << 24)) return false;
+  out->total = cu[num_seqs];
+  out->n_tiles = static_cast<int>(tiles);
+  out->nblk = static_cast<int>(blocks);
+  return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t gproj_attn_varlen_plan_bytes(const int *cu_seqlens, int num_seqs) {
+  PackedShape ps;
+  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return 0;
+  return 2 * static_cast<size_t>(ps.n_tiles) * sizeof(int4);
+}
+
+int gproj_attn_varlen_plan(const int *cu_seqlens, int num_seqs, int causal, void *plan_host, size_t plan_bytes) {
+  PackedShape ps;
+  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
+  if (!plan_host) return GPROJ_ERR_NULL;
+  if (plan_bytes < 2 * static_cast<size_t>(ps.n_tiles) * sizeof(int4)) return GPROJ_ERR_WORKSPACE;
+  struct Entry { int4 e; long long work_q, work_kv; };
+  std::vector<Entry> v;
+  v.reserve(static_cast<size_t>(ps.n_tiles));
+  int blk0 = 0;
+  for (int s = 0; s < num_seqs; ++s) {
+    const int seq0 = cu_seqlens[s], seq_end = cu_seqlens[s + 1], len = seq_end - seq0;
+    for (int t = 0; t * 128 < len; ++t) {
+      Entry en;
+      en.e = make_int4(seq0 + 128 * t, seq0, seq_end, blk0);
+      const int upto = (t + 1) * 128 < len ? (t + 1) * 128 : len;
+      en.work_q = causal ? upto : len;            // keys a query tile walks
+      en.work_kv = causal ? len - 128 * t : len;  // queries a key tile walks
+      v.push_back(en);
+    }
+    blk0 += (len + 63) / 64;
+  }
+  int4 *out = static_cast<int4 *>(plan_host);
+  // the persistent kernels deal tiles in this order: longest first (stable, so equal tiles keep their memory order)
+  std::stable_sort(v.begin(), v.end(), [](const Entry &a, const Entry &b) { return a.work_q > b.work_q; });
+  for (size_t i = 0; i < v.size(); ++i) out[i] = v[i].e;
+  std::stable_sort(v.begin(), v.end(), [](const Entry &a, const Entry &b) { return a.work_kv > b.work_kv; });
+  for (size_t i = 0; i < v.size(); ++i) out[v.size() + i] = v[i].e;
+  return GPROJ_OK;
+}
+
+int gproj_attn_fwd_varlen(const void *Q, const void *K, const void *V, void *O, float *LSE, const int *cu_seqlens,
+                          int num_seqs, const void *plan_device, int H, int Hkv, int d, float softmax_scale, int causal,
+                          unsigned fwd_flags, void *stream) {
+  PackedShape ps;
+  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
+  if (!plan_device) return GPROJ_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
+  return launch_fwd(Q, K, V, O, LSE, 1, H, Hkv, ps.total, d, softmax_scale, causal, fwd_flags,
+                    static_cast<const int4 *>(plan_device), ps.n_tiles, stream);
+}
+
+size_t gproj_attn_bwd_varlen_workspace_bytes(const int *cu_seqlens, int num_seqs, int H, int d) {
+  PackedShape ps;
+  if (!packed_shape(cu_seqlens, num_seqs, &ps) || check_shape(1, H, ps.total, d) != GPROJ_OK) return 0;
+  return align256(static_cast<size_t>(H) * ps.nblk * 512) + align256(static_cast<size_t>(H) * ps.total * static_cast<size_t>(d) * 2);
+}
+
+int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                          void *dQ, void *dK, void *dV, const int *cu_seqlens, int num_seqs, const void *plan_device, int H,
+                          int Hkv, int d, float softmax_scale, int causal, void *workspace, size_t workspace_bytes,
+                          unsigned flags, void *stream) {
+  PackedShape ps;
+  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
+  if (!plan_device) return GPROJ_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
+  const int4 *plan = static_cast<const int4 *>(plan_device);
+  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, 1, H, Hkv, ps.total, d, softmax_scale, causal, workspace, workspace_bytes,
+                    flags, plan, plan + ps.n_tiles, ps.n_tiles, ps.nblk, stream);
 }
 
 // ---- backward without a caller-supplied workspace -------------------------------------------------

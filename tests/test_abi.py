@@ -69,3 +69,35 @@ def test_python_binding_refuses_cpu_tensors():
     x = torch.zeros(1, 1, 128, 64, dtype=torch.bfloat16)
     with pytest.raises(TypeError):
         binding.gproj_attn_fwd(x, x, x, 0.125, True)
+
+
+def test_varlen_plan_on_host(lib):
+    # the plan is host arithmetic: every 128-row tile of every non-empty sequence exactly once in each of the two orders,
+    # longest work first, statistic blocks numbered sequence after sequence
+    import numpy as np
+    cu = [0, 1, 6, 70, 70, 470, 598]
+    arr = (ctypes.c_int * len(cu))(*cu)
+    S = len(cu) - 1
+    lens = np.diff(cu)
+    n_tiles = int(sum((l + 127) // 128 for l in lens))
+    nbytes = lib.gproj_attn_varlen_plan_bytes(arr, S)
+    assert nbytes == 2 * n_tiles * 16
+    for causal in (0, 1):
+        buf = np.zeros(2 * n_tiles * 4, dtype=np.int32)
+        assert lib.gproj_attn_varlen_plan(arr, S, causal, buf.ctypes.data_as(ctypes.c_void_p), nbytes) == 0
+        plan = buf.reshape(2, n_tiles, 4)
+        expect = set()
+        blk = 0
+        for s in range(S):
+            for t in range((lens[s] + 127) // 128):
+                expect.add((cu[s] + 128 * t, cu[s], cu[s + 1], blk))
+            blk += (lens[s] + 63) // 64
+        for order in range(2):
+            assert set(map(tuple, plan[order].tolist())) == expect and len(plan[order]) == len(expect)
+        work_q = [min(r0 + 128, e) - s0 if causal else e - s0 for r0, s0, e, _ in plan[0]]
+        work_kv = [e - r0 if causal else e - s0 for r0, s0, e, _ in plan[1]]
+        assert work_q == sorted(work_q, reverse=True) and work_kv == sorted(work_kv, reverse=True)
+    assert lib.gproj_attn_varlen_plan(arr, S, 1, None, nbytes) == -1
+    assert lib.gproj_attn_varlen_plan(arr, S, 1, ctypes.c_void_p(0x1000), 16) == -4
+    bad = (ctypes.c_int * 3)(0, 5, 3)
+    assert lib.gproj_attn_varlen_plan_bytes(bad, 2) == 0 and lib.gproj_attn_varlen_plan(bad, 2, 1, None, 0) == -2

@@ -42,7 +42,7 @@ struct FwdCfg {
 
 enum FwdWaitCode {
   kFwdWaitQ = 0x11, kFwdWaitK = 0x12, kFwdWaitV = 0x13, kFwdWaitKVEmpty = 0x14, kFwdWaitS = 0x15, kFwdWaitP = 0x16,
-  kFwdWaitPV = 0x17, kFwdWaitSFree = 0x18, kFwdWaitOFree = 0x19, kFwdWaitQFree = 0x1a, kFwdWaitTurn = 0x1b
+  kFwdWaitPV = 0x17, kFwdWaitSFree = 0x18, kFwdWaitOFree = 0x19, kFwdWaitQFree = 0x1a, kFwdWaitTurn = 0x1b, kFwdWaitMerge = 0x1c
 };
 
 
@@ -75,7 +75,9 @@ __device__ __forceinline__ float softmax_exp_store(const uint32_t (&xr)[4][32], 
   return (r0 + r1) + (r2 + r3);
 }
 
-template <int D, bool CAUSAL, bool FMA_SOFTMAX, bool TURNS>
+// MODE: 0 = pairs of query tiles, 1 = pairs whose warpgroups take turns in the exponential phase, 2 = single tiles with
+// the key range split between the warpgroups.
+template <int D, bool CAUSAL, bool FMA_SOFTMAX, int MODE>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -89,7 +91,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t *sKV = sQ + 2 * C::kTileBytes;            // stage s: K tile, then V tile
 
   __shared__ uint64_t bar_q_full, bar_q_free, bar_k_full[S], bar_v_full[S], bar_kv_empty[S];
-  __shared__ uint64_t bar_s_full[2], bar_s_free[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_turn[2], bar_drain[2];
+  __shared__ uint64_t bar_s_full[2], bar_s_free[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_turn[2], bar_merge, bar_drain[2];
+  __shared__ float s_m1[2][128], s_l1[2][128];   // split mode: running maximum and normaliser of the second warpgroup
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -99,12 +102,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (cta_skip != 0) return;   // an earlier wait gave up: drain the rest of the grid quickly
 
   const int n_qt = (N + C::kBlockM - 1) / C::kBlockM;   // the last tile may be ragged: rows past N load as zero, stores clip
-  const int TPI = tiles_per_item;                  // 2: a pair of query tiles per work item; 1: single tiles (small grids)
+  const int TPI = tiles_per_item;                  // 2: a pair of query tiles per work item; 1: single tiles, key range split
+  constexpr bool split = (MODE == 2);              // one query tile; warpgroup t takes the key tiles j = t (mod 2), merged at the end
+  constexpr bool TURNS = (MODE == 1);
   const int n_pairs = (n_qt + TPI - 1) / TPI;
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
     mbar_init(&bar_q_full, 1);
+    mbar_init(&bar_merge, 128);
     mbar_init(&bar_q_free, tiles_per_item);         // one arrival per query tile slot: its O store has left shared memory
     for (int s = 0; s < S; ++s) { mbar_init(&bar_k_full[s], 1); mbar_init(&bar_v_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
@@ -200,7 +206,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const SmemDesc dscK = dscK0.advanced(st * 2 * C::kTileBytes);
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-          if (!active(it, t, j)) continue;
+          if (split ? ((j & 1) != t) : !active(it, t, j)) continue;
           // S_t may be overwritten once its previous contents are dead: copied to registers by the softmax (P~ has its
           // own columns), or, when P~ lives in the same columns, consumed by the previous P~V product.
           if (cnt[t] > 0) {
@@ -208,7 +214,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             else          mbar_wait(&bar_pv_done[t], (cnt[t] - 1) & 1, ab, kFwdWaitSFree);
           }
           tc_fence_after();
-          const SmemDesc dscQ = dscQ0.advanced(t * C::kTileBytes);
+          const SmemDesc dscQ = dscQ0.advanced(split ? 0 : t * C::kTileBytes);
           if (elect_one_sync()) {
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
@@ -237,12 +243,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const SmemDesc dscV = dscV0.advanced(st * 2 * C::kTileBytes);
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-          if (!active(it, t, j)) continue;
-          if (j == 0 && ti > 0) mbar_wait(&bar_o_free[t], (ti - 1) & 1, ab, kFwdWaitOFree);   // previous epilogue has read O_t
+          if (split ? ((j & 1) != t) : !active(it, t, j)) continue;
+          const bool first = split ? (j < 2) : (j == 0);     // first product into O_t in this work item
+          if (first && ti > 0) mbar_wait(&bar_o_free[t], (ti - 1) & 1, ab, kFwdWaitOFree);   // previous epilogue has read O_t
           mbar_wait(&bar_p_ready[t], cnt[t] & 1, ab, kFwdWaitP);
           tc_fence_after();
           const uint32_t tP = tmem_base + (C::kSepP ? C::kColP + 64 * t : C::kColS + 128 * t);
-          const uint32_t acc = (j > 0) ? 1u : 0u;
+          const uint32_t acc = first ? 0u : 1u;
           if (elect_one_sync()) {
 #pragma unroll
             for (int k = 0; k < C::kBlockN / 16; ++k)
@@ -266,13 +273,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tO = tmem_base + C::kColO + D * t + lane_addr;
     const uint32_t tP = tmem_base + (C::kSepP ? C::kColP + 64 * t : C::kColS + 128 * t) + lane_addr;
     int ti = 0, cnt = 0, turn = 0;
-    // With single-tile items the second warpgroup has nothing to do for the whole launch (and bar_q_free expects one
-    // arrival per item only).
-    for (int lin = (t < TPI) ? sched.next() : -1; lin >= 0; lin = sched.next(), ++ti) {
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const Item it = decode(lin);
       const int bh = lin % BH, T = it.n_kt;
-      const int qt = it.qt0 + t;                      // this warpgroup's query tile inside the sequence
-      if (t >= it.nq) {
+      const int qt = it.qt0 + (split ? 0 : t);        // this warpgroup's query tile inside the sequence
+      // Split mode: stay in step with the item (its Q has landed), so that a warpgroup without key tiles cannot run ahead.
+      if (split) mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
+      if (!split && t >= it.nq) {
         // Odd number of query tiles: the last pair has no second tile.  Stay in step with the item (its Q has landed)
         // before handing back this slot, so that no barrier runs ahead of the roles that wait on it.
         mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
@@ -283,8 +290,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       float m_run = -INFINITY, l_run = 0.f;
       // Both tiles of the pair exist: the warpgroups alternate in the exponential phase, step by step, tile 0 first.
       const bool take_turns = TURNS && it.nq == 2;
-      for (int j = 0; j < T; ++j) {
-        if (!active(it, t, j)) {
+      const int cnt_item0 = cnt;
+      for (int j = split ? t : 0; j < T; j += split ? 2 : 1) {
+        const bool first = split ? (j < 2) : (j == 0);     // this warpgroup's first key tile of the item
+        if (!split && !active(it, t, j)) {
           // no work in this step (causal: the first tile of the pair ends one key tile earlier): pass the turn on
           if (take_turns) {
             if (t == 1 || turn > 0) mbar_wait(&bar_turn[t], (t == 1 ? turn : turn - 1) & 1, ab, kFwdWaitTurn);
@@ -333,7 +342,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // in which x a is not rounded separately, so the largest score need not map to exactly zero.
         const float m_scaled = __fmul_rn(m_new, scale_log2);
         // P~ of the previous key tile must have been consumed (and O_t updated) before either is touched
-        if (j > 0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
+        if (!first) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
         // The exponential phase is the only heavy user of the special-function unit (16 results per clock per SM, the
         // forward's scarcest pipe).  With TURNS the two warpgroups alternate in it, so that one's exponentials run against
         // the other's loads, maxima and barrier work instead of both phases colliding and then both leaving the unit idle
@@ -342,7 +351,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const float rs = softmax_exp_store<FMA_SOFTMAX>(xr, tP, m_new, scale_log2, m_scaled);
         if (take_turns) { mbar_arrive(&bar_turn[1 - t]); ++turn; }
         l_run = l_run * corr + rs;
-        if (j > 0 && __any_sync(0xffffffffu, m_new != m_run)) {
+        if (!first && __any_sync(0xffffffffu, m_new != m_run)) {
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
@@ -360,14 +369,45 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ++cnt;
       }
       // ---- epilogue: O = BF16(acc / l) staged in the TMA layout over this tile's Q, LSE = alpha x_max + ln l
-      mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV);
-      tc_fence_after();
-      const float inv_l = 1.0f / l_run;
+      if (cnt > cnt_item0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
+      if (split && t == 1) {
+        // hand this half's statistics to warpgroup 0, which merges the two accumulators (l = 0: no key tiles here)
+        s_m1[ti & 1][row] = m_run;
+        s_l1[ti & 1][row] = l_run;
+        tc_fence_before();
+        mbar_arrive(&bar_merge);
+        continue;
+      }
+      // Split mode: O = (O_0 s_0 + O_1 s_1) / (l_0 s_0 + l_1 s_1) with s_t = exp2((m_t - max(m_0, m_1)) alpha log2 e).
+      const bool has1 = split && T >= 2;               // the second warpgroup had at least one key tile
+      float a0 = 1.0f / l_run, a1 = 0.f;
+      if (split) {
+        mbar_wait(&bar_merge, ti & 1, ab, kFwdWaitMerge);
+        tc_fence_after();
+        if (has1) {
+          const float m1 = s_m1[ti & 1][row], l1 = s_l1[ti & 1][row];
+          const float m = fmaxf(m_run, m1);
+          const float s0 = fast_exp2(__fmul_rn(__fsub_rn(m_run, m), scale_log2)), s1 = fast_exp2(__fmul_rn(__fsub_rn(m1, m), scale_log2));
+          l_run = fmaf(l_run, s0, l1 * s1);
+          m_run = m;
+          const float inv = 1.0f / l_run;
+          a0 = s0 * inv;
+          a1 = s1 * inv;
+        }
+      }
+      const float inv_l = has1 ? 1.0f : a0;            // with two halves the weights a_0, a_1 already carry 1 / l
       uint8_t *stage = sQ + t * C::kTileBytes;         // no MMA reads this Q tile any more
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t o[32];
         tmem_ld32(tO + 32 * c, o);
+        if (has1) {
+          uint32_t o1[32];
+          tmem_ld32(tO + D + 32 * c, o1);              // O_1 sits D columns after O_0, same lanes
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(fmaf(__uint_as_float(o1[i]), a1, __uint_as_float(o[i]) * a0));
+        }
         tmem_wait_ld();
         const uint32_t slab = (c >> 1) * C::kSlabBytes;
 #pragma unroll
@@ -381,6 +421,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       tc_fence_before();
       mbar_arrive(&bar_o_free[t]);                     // O_t may be overwritten by the next work item
+      if (split) mbar_arrive(&bar_o_free[1]);          // warpgroup 0 has read both accumulators
       const int qrow0 = it.seq0 + qt * C::kBlockM;      // first row of the tile inside the head
       if (qt * C::kBlockM + row < it.len) LSE[static_cast<size_t>(bh) * N + qrow0 + row] = fmaf(m_run, alpha, logf(l_run));
       fence_proxy_async_smem();

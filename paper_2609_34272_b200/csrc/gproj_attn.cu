@@ -76,16 +76,24 @@ int device_state(DeviceState **out) {
       if (cudaGetSymbolAddress(reinterpret_cast<void **>(&st.status_ptr), g_device_status) != cudaSuccess)
         return GPROJ_ERR_CUDA;
       bool ok = true;
-      ok &= allow_smem(attn_fwd_kernel<64, true, false, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<64, false, false, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, true, false, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, true, false, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, false, false, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, false, false, true>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<64, true, true, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<64, false, true, false>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, true, true, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
-      ok &= allow_smem(attn_fwd_kernel<128, false, true, false>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, false, 0>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, false, 2>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, true, 0>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, true, true, 2>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, false, 0>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, false, 2>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, true, 0>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<64, false, true, 2>, FwdCfg<64>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, false, 0>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, false, 1>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, false, 2>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, true, 0>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, true, true, 2>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, false, 0>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, false, 1>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, false, 2>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, true, 0>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(attn_fwd_kernel<128, false, true, 2>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, true>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, false>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<128, true>, BwdCfg<128>::kDqSmemBytes) == cudaSuccess;
@@ -190,18 +198,22 @@ int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE,
   if (total_items <= 0) return GPROJ_OK;   // nothing but empty sequences
   const dim3 grid(static_cast<unsigned>(total_items < st->sm_count ? total_items : st->sm_count));   // persistent
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define GPROJ_LAUNCH_FWD(DD, CC, FF, TT)                                                                            \
-  attn_fwd_kernel<DD, CC, FF, TT><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(                         \
+#define GPROJ_LAUNCH_FWD(DD, CC, FF, MM)                                                                            \
+  attn_fwd_kernel<DD, CC, FF, MM><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(                         \
       mQ, mK, mV, mO, static_cast<__nv_bfloat16 *>(O), plan, LSE, N, BH, H, G, tiles_per_item, total_items, scale_log2,      \
       softmax_scale, st->status_ptr)
-#define GPROJ_LAUNCH_FWD_C(DD, FF, TT)                                                                              \
-  do { if (causal) GPROJ_LAUNCH_FWD(DD, true, FF, TT); else GPROJ_LAUNCH_FWD(DD, false, FF, TT); } while (0)
-  // the softmax warpgroups alternate in the exponential phase where that was measured to pay: d = 128, paired tiles
-  const bool turns = (d == 128) && (tiles_per_item == 2) && !fma;
-  if (d == 64) { if (fma) GPROJ_LAUNCH_FWD_C(64, true, false); else GPROJ_LAUNCH_FWD_C(64, false, false); }
-  else if (fma) GPROJ_LAUNCH_FWD_C(128, true, false);
-  else if (turns) GPROJ_LAUNCH_FWD_C(128, false, true);
-  else GPROJ_LAUNCH_FWD_C(128, false, false);
+#define GPROJ_LAUNCH_FWD_C(DD, FF, MM)                                                                              \
+  do { if (causal) GPROJ_LAUNCH_FWD(DD, true, FF, MM); else GPROJ_LAUNCH_FWD(DD, false, FF, MM); } while (0)
+#define GPROJ_LAUNCH_FWD_F(DD, MM)                                                                                  \
+  do { if (fma) GPROJ_LAUNCH_FWD_C(DD, true, MM); else GPROJ_LAUNCH_FWD_C(DD, false, MM); } while (0)
+  // Single tiles: the two softmax warpgroups split the key range of the tile.  Pairs: one tile each, and at d = 128
+  // they alternate in the exponential phase (measured to pay there only).
+  const bool split = (tiles_per_item == 1), turns = (d == 128) && !split && !fma;
+  if (d == 64) { if (split) GPROJ_LAUNCH_FWD_F(64, 2); else GPROJ_LAUNCH_FWD_F(64, 0); }
+  else if (split) GPROJ_LAUNCH_FWD_F(128, 2);
+  else if (turns) GPROJ_LAUNCH_FWD_C(128, false, 1);
+  else GPROJ_LAUNCH_FWD_F(128, 0);
+#undef GPROJ_LAUNCH_FWD_F
 #undef GPROJ_LAUNCH_FWD_C
 #undef GPROJ_LAUNCH_FWD
   if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;

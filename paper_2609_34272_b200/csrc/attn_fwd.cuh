@@ -1,24 +1,29 @@
 // Fused attention forward for sm_100a: O = softmax(alpha Q K^T) V and the row log-sum-exp.
 //
-// A persistent CTA (one per SM) walks a static list of work items; one item = a PAIR of 128-row query tiles of
-// one (batch, head), processed against the key tiles they attend to.  Roles (384 threads):
+// A persistent CTA (one per SM) walks a static list of work items.  Roles (384 threads):
 //   warp 0        TMA producer of the streamed K_j / V_j tiles (separate barriers: S needs only K, P~V only V)
-//   warp 1        tensor-core issuer 1: S_t = Q_t K_j^T for both query tiles (N = 128, FP32 in TMEM); owns TMEM
+//   warp 1        tensor-core issuer 1: S_t = Q K_j^T (N = 128, FP32 in TMEM); owns TMEM
 //   warp 2        tensor-core issuer 2: O_t += P~_t V_j with the BF16 probabilities read straight from TMEM
-//   warp 3        TMA loader of the stationary Q pair
-//   warps 4..7    softmax warpgroup of query tile 0, warps 8..11 of query tile 1: thread <-> query row (TMEM lane),
-//                 so every row statistic is a private register.  While one warpgroup is in the ALUs the tensor
-//                 core works for the other one (the tensor-core queue is only 1-2 instructions deep, hence two
-//                 issuing warps: each one's barrier polls overlap the other's MMAs).
+//   warp 3        TMA loader of the stationary Q tile(s)
+//   warps 4..7    softmax warpgroup 0, warps 8..11 softmax warpgroup 1: thread <-> query row (TMEM lane), so every
+//                 row statistic is a private register.  While one warpgroup is in the ALUs the tensor core works for
+//                 the other one (the tensor-core queue is only 1-2 instructions deep, hence two issuing warps: each
+//                 one's barrier polls overlap the other's MMAs).
+// Work items (template parameter MODE):
+//   pairs (0, 1)  one item = two 128-row query tiles of one (batch, head), warpgroup t <-> tile t, every K / V tile
+//                 serves both; with MODE 1 the warpgroups also take turns in the exponential phase.
+//   split (2)     one item = one query tile; warpgroup t takes the key tiles j = t (mod 2) with its own running
+//                 maximum, normaliser and accumulator, and warpgroup 0 merges the two halves at the end.  Used when
+//                 pairs would leave SMs idle and for packed sequences.
 // Softmax arithmetic (FMA_SOFTMAX = false, the default): online softmax on the UNSCALED logits with the
 // subtract-before-scale rounding of
 // Eq. "gproj-forward": z = exp2(fl32[ fl32(x - x_max) * (alpha log2 e) ]); l accumulates the FP32 z, the value
-// product uses BF16(z); the accumulator is rescaled whenever the running maximum of any row of the warp moved.
+// product uses BF16(z); the running maximum is raised lazily and the accumulator rescaled only then.
 // The saved state is BF16 O (staged in the TMA layout over the consumed Q tile, written by a TMA store) and
 // FP32 LSE = alpha x_max + ln l  (Algorithm 1, "Input").
 // TMEM: S_0, S_1 (128 columns each), O_0, O_1 (d each); at d = 64 the packed P~_t have their own 64 columns, so
-// S_t of the next key tile can be issued as soon as the softmax has read the current one; at d = 128 TMEM is full
-// and P~_t overwrites the first half of S_t.
+// S_t of the next key tile can be issued as soon as the softmax has copied the current one to registers; at d = 128
+// TMEM is full and P~_t overwrites the first half of S_t.
 #pragma once
 #include "attn_bwd.cuh"   // TileSched
 #include "sm100_primitives.cuh"

@@ -143,6 +143,23 @@ int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const voi
                           unsigned flags, void *stream);
 
 /*
+ * Forward and backward in one call from HOST buffers (a convenience around the entry points above; the paper's
+ * Algorithm 1 starts from tensors already on the device).  Q, K, V, dO are copied to the device, the forward
+ * (Eq. "gproj-forward") and the backward (Algorithm 1) run, and dQ, dK, dV (and O, LSE when those pointers are not NULL)
+ * are copied back, all enqueued in order on `stream`.
+ *   - Q, K, V, dO, O, LSE, dQ, dK, dV are HOST pointers with the layouts of gproj_attn_fwd_gqa / gproj_attn_bwd_gqa.  Page-locked
+ *     memory makes the call asynchronous; pageable memory works but serialises in the CUDA runtime.  The buffers must stay
+ *     valid until the stream has reached the end of the call's work.
+ *   - `staging` is DEVICE memory owned by the caller, 256-byte aligned, at least gproj_attn_host_staging_bytes() bytes (copies
+ *     of the eight tensors, LSE and the backward workspace); GPROJ_ERR_WORKSPACE otherwise.  Nothing is allocated.
+ *   - flags: those of gproj_attn_bwd without the ONLY_* bits.
+ */
+size_t gproj_attn_host_staging_bytes(int B, int H, int Hkv, int N, int d);
+int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const void *dO, void *O, float *LSE,
+                            void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale,
+                            int causal, void *staging, size_t staging_bytes, unsigned flags, void *stream);
+
+/*
  * Backward for callers that must not allocate device memory (the paper has no counterpart: this is a
  * convenience of this library).  Some hosts of this code cannot call cudaMalloc at the point where they
  * need a gradient: a plugin running inside another framework's memory pool, a real-time or safety-audited

@@ -25,6 +25,7 @@ EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd",
            "gproj_attn_bwd_static_scratch",
            "gproj_attn_varlen_plan_bytes", "gproj_attn_varlen_plan", "gproj_attn_fwd_varlen",
            "gproj_attn_bwd_varlen_workspace_bytes", "gproj_attn_bwd_varlen",
+           "gproj_attn_host_staging_bytes", "gproj_attn_fwd_bwd_host",
            "gproj_last_device_status", "gproj_selftest_wait_timeout",
            "gproj_status_string", "gproj_last_launch_count")
 
@@ -71,6 +72,10 @@ def load():
         lib.gproj_attn_bwd_varlen_workspace_bytes.argtypes = [ip, i, i, i]
         lib.gproj_attn_bwd_varlen.restype = i
         lib.gproj_attn_bwd_varlen.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ip, i, vp, i, i, i, f, i, vp, ctypes.c_size_t, u, vp]
+        lib.gproj_attn_host_staging_bytes.restype = ctypes.c_size_t
+        lib.gproj_attn_host_staging_bytes.argtypes = [i, i, i, i, i]
+        lib.gproj_attn_fwd_bwd_host.restype = i
+        lib.gproj_attn_fwd_bwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, ctypes.c_size_t, u, vp]
         lib.gproj_selftest_wait_timeout.restype = i
         lib.gproj_selftest_wait_timeout.argtypes = [vp]
         lib.gproj_last_device_status.restype = i
@@ -276,3 +281,26 @@ def gproj_attn_bwd_varlen(Q, K, V, O, LSE, dO, plan, softmax_scale, flags=0, wor
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_bwd_varlen")
     return dQ, dK, dV
+
+
+def gproj_attn_host_staging_bytes(B, H, Hkv, N, d) -> int:
+    return int(load().gproj_attn_host_staging_bytes(B, H, Hkv, N, d))
+
+
+def gproj_attn_fwd_bwd_host(Q, K, V, dO, dQ, dK, dV, softmax_scale, causal, staging, O=None, LSE=None, flags=0):
+    """Forward + backward from HOST bfloat16 tensors (pinned for an asynchronous call) into HOST dQ, dK, dV (and O, LSE if
+    given); `staging` is a CUDA uint8 tensor of gproj_attn_host_staging_bytes() bytes.  Work is enqueued on the current stream."""
+    for name, t in (("Q", Q), ("K", K), ("V", V), ("dO", dO), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+        if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
+            raise TypeError(f"{name} must be a contiguous CPU bfloat16 tensor")
+    B, H, N, d = Q.shape
+    Hkv = K.shape[1]
+    if not (staging.is_cuda and staging.dtype == torch.uint8 and staging.is_contiguous()):
+        raise TypeError("staging must be a contiguous CUDA uint8 tensor")
+    ptr = lambda t: ctypes.c_void_p(t.data_ptr()) if t is not None else None
+    with torch.cuda.device(staging.device):
+        rc = load().gproj_attn_fwd_bwd_host(ptr(Q), ptr(K), ptr(V), ptr(dO), ptr(O), ptr(LSE), ptr(dQ), ptr(dK), ptr(dV), B, H, Hkv, N, d,
+                                            float(softmax_scale), int(bool(causal)), ptr(staging), staging.numel(), int(flags),
+                                            _stream(staging.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_fwd_bwd_host")

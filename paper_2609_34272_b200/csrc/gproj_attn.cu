@@ -413,6 +413,49 @@ int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const voi
                     flags, plan, plan + ps.n_tiles, ps.n_tiles, ps.nblk, stream);
 }
 
+// ---- forward + backward from host buffers ----------------------------------------------------------
+size_t gproj_attn_host_staging_bytes(int B, int H, int Hkv, int N, int d) {
+  if (check_shape(B, H, N, d) != GPROJ_OK || Hkv <= 0 || H % Hkv != 0) return 0;
+  const size_t q = align256(static_cast<size_t>(B) * H * N * d * 2), kv = align256(static_cast<size_t>(B) * Hkv * N * d * 2);
+  return 4 * q + 4 * kv + align256(static_cast<size_t>(B) * H * N * sizeof(float)) + gproj_attn_bwd_workspace_bytes(B, H, N, d);
+}
+
+int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const void *dO, void *O, float *LSE, void *dQ,
+                            void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+                            void *staging, size_t staging_bytes, unsigned flags, void *stream) {
+  if (!Q || !K || !V || !dO || !dQ || !dK || !dV) return GPROJ_ERR_NULL;
+  const size_t need = gproj_attn_host_staging_bytes(B, H, Hkv, N, d);
+  if (need == 0) return GPROJ_ERR_SHAPE;
+  if (!staging || (reinterpret_cast<uintptr_t>(staging) & 255u) || staging_bytes < need) return GPROJ_ERR_WORKSPACE;
+  const size_t qb = static_cast<size_t>(B) * H * N * d * 2, kvb = static_cast<size_t>(B) * Hkv * N * d * 2;
+  const size_t lb = static_cast<size_t>(B) * H * N * sizeof(float);
+  uint8_t *p = static_cast<uint8_t *>(staging);
+  auto take = [&](size_t bytes) { uint8_t *r = p; p += align256(bytes); return r; };
+  uint8_t *dQin = take(qb), *dOin = take(qb), *dOout = take(qb), *dQout = take(qb);
+  uint8_t *dKin = take(kvb), *dVin = take(kvb), *dKout = take(kvb), *dVout = take(kvb);
+  float *dLSE = reinterpret_cast<float *>(take(lb));
+  uint8_t *ws = p;
+  const size_t ws_bytes = gproj_attn_bwd_workspace_bytes(B, H, N, d);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  bool ok = cudaMemcpyAsync(dQin, Q, qb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+            cudaMemcpyAsync(dKin, K, kvb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+            cudaMemcpyAsync(dVin, V, kvb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+            cudaMemcpyAsync(dOin, dO, qb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+  if (int rc = gproj_attn_fwd_gqa(dQin, dKin, dVin, dOout, dLSE, B, H, Hkv, N, d, softmax_scale, causal, stream)) return rc;
+  if (int rc = gproj_attn_bwd_gqa(dQin, dKin, dVin, dOout, dLSE, dOin, dQout, dKout, dVout, B, H, Hkv, N, d, softmax_scale,
+                                  causal, ws, ws_bytes, flags, stream))
+    return rc;
+  ok = cudaMemcpyAsync(dQ, dQout, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaMemcpyAsync(dK, dKout, kvb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaMemcpyAsync(dV, dVout, kvb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (ok && O) ok = cudaMemcpyAsync(O, dOout, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (ok && LSE) ok = cudaMemcpyAsync(LSE, dLSE, lb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+  tl_launch_count = 3;
+  return GPROJ_OK;
+}
+
 // ---- backward without a caller-supplied workspace -------------------------------------------------
 // The scratch is a file-scope device array.  In host code the array's name is only a handle: the
 // address a kernel or a TMA descriptor can use must be looked up per device with cudaGetSymbolAddress.

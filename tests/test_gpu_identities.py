@@ -211,3 +211,23 @@ def test_fma_softmax_breaks_the_one_key_identity_and_sbs_restores_it():
     assert rc == 0, hex(detail)
     print("one-key violations with the fused exponent:", violations, "of 48")
     assert violations >= 3
+
+
+def test_host_buffer_entry_point_matches_device_calls():
+    # forward + backward from pinned host tensors: same kernels, so bit for bit the results of the device-pointer calls
+    w = Workload("host", 2, 4, 320, 64, True, k_offset=4.0, seed=31, Hkv=2)
+    inp = make_inputs(w)
+    O, LSE, dQ, dK, dV = fwd_bwd(inp["Q"], inp["K"], inp["V"], inp["dO"], w.softmax_scale, True)
+    host = {k: v.pin_memory() for k, v in inp.items()}
+    hO = torch.empty_like(host["Q"]).pin_memory(); hL = torch.empty(w.B, w.H, w.N, dtype=torch.float32).pin_memory()
+    hdQ = torch.empty_like(host["Q"]).pin_memory(); hdK = torch.empty_like(host["K"]).pin_memory(); hdV = torch.empty_like(host["K"]).pin_memory()
+    staging = torch.empty(g.gproj_attn_host_staging_bytes(w.B, w.H, w.kv_heads, w.N, w.d), dtype=torch.uint8, device="cuda")
+    g.gproj_attn_fwd_bwd_host(host["Q"], host["K"], host["V"], host["dO"], hdQ, hdK, hdV, w.softmax_scale, True, staging, O=hO, LSE=hL)
+    rc, detail = g.gproj_last_device_status()      # synchronises the stream
+    assert rc == 0, hex(detail)
+    assert torch.equal(hO, O.cpu()) and torch.equal(hL, LSE.cpu())
+    assert torch.equal(hdQ, dQ.cpu()) and torch.equal(hdK, dK.cpu()) and torch.equal(hdV, dV.cpu())
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(g.GprojError) as e:
+        g.gproj_attn_fwd_bwd_host(host["Q"], host["K"], host["V"], host["dO"], hdQ, hdK, hdV, w.softmax_scale, True, small)
+    assert e.value.status == -4

@@ -177,35 +177,67 @@ __device__ __forceinline__ void dq_slice(uint32_t tS, uint32_t tdP, float scale_
   }
 }
 
-// One step of the dK/dV side for one key row and one slice (32 queries) of the step's 64 queries, chunked as above.
-// `lim` = (key row) - (query index of the slice's column 0): with MASKED, column c is a query before this key when
-// c < lim; `hi` = (last query of the sequence) - (query index of column 0): a column c > hi belongs to the next packed
-// sequence (or is zero fill).  nl / nd: the slice's per-column -LSE log2 e and -D (shared memory, same address for every lane: broadcast).
+// The dK/dV side does the arithmetic of a step in two phases, so that the tensor core can start on the products that need
+// only r^T while the ALUs are still busy with t^T (measured: -15 % on that kernel at d = 128; the dQ side did not gain):
+//   phase 1 (needs S^T):   p = exp2(x * (alpha log2 e) - LSE log2 e), r = BF16(p); p is kept in FP32 registers
+//   phase 2 (needs dP^T):  t = BF16(fl32[p * fl32(dP - D)])
+// Each thread owns one key row and one slice (32 query columns) of the step, handled in two 16-column chunks whose TMEM
+// loads are software-pipelined; the packed operands overwrite the chunk's own consumed S columns (r the first eight, t
+// the last eight).
+
+// Phase 1 of the dK/dV side (thread <-> key row, columns = queries).  `lim` = (key row) - (query index of the slice's
+// column 0): with MASKED, column c is a query before this key when c < lim; `hi` = (last query of the sequence) - (query
+// index of column 0): a column c > hi belongs to the next packed sequence (or is zero fill).  nl: the slice's per-column
+// -LSE log2 e (shared memory, same address for every lane: broadcast reads).
 template <bool MASKED>
-__device__ __forceinline__ void dkv_slice(uint32_t tS, uint32_t tdP, const float *nl, const float *nd, float scale_log2, int lim, int hi) {
+__device__ __forceinline__ void dkv_phase1(uint32_t tS, const float *nl, float scale_log2, int lim, int hi, float (&p)[32]) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2);
-  uint32_t xs[2][16], xp[2][16];
+  uint32_t xs[2][16];
   tmem_ld16(tS, xs[0]);
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    tmem_wait_ld();
+    if (c == 0) tmem_ld16(tS + 16, xs[1]);
+    uint32_t pr[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);   // four columns per 16-byte read
+      const int col = 16 * c + 4 * i;
+      float a[4];
+      f32x2_split(fma2(f32x2_bits(xs[c][4 * i], xs[c][4 * i + 1]), scale2, l4.x), a[0], a[1]);
+      f32x2_split(fma2(f32x2_bits(xs[c][4 * i + 2], xs[c][4 * i + 3]), scale2, l4.y), a[2], a[3]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float pe = fast_exp2(a[e]);
+        if (MASKED && (col + e < lim || col + e > hi)) pe = 0.f;
+        p[col + e] = pe;
+      }
+      pr[2 * i] = pack_bf16x2(p[col], p[col + 1]);
+      pr[2 * i + 1] = pack_bf16x2(p[col + 2], p[col + 3]);
+    }
+    tmem_st8(tS + 16 * c, pr);
+  }
+}
+
+// Phase 2 of the dK/dV side.  nd: the slice's per-column -D.
+__device__ __forceinline__ void dkv_phase2(uint32_t tS, uint32_t tdP, const float *nd, const float (&p)[32]) {
+  uint32_t xp[2][16];
   tmem_ld16(tdP, xp[0]);
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
     tmem_wait_ld();
-    if (c == 0) {
-      tmem_ld16(tS + 16, xs[1]);
-      tmem_ld16(tdP + 16, xp[1]);
-    }
-    uint32_t pr[8], pt[8];
+    if (c == 0) tmem_ld16(tdP + 16, xp[1]);
+    uint32_t pt[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);
       const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
       const int col = 16 * c + 4 * i;
-      score_pair<MASKED>(xs[c][4 * i], xs[c][4 * i + 1], xp[c][4 * i], xp[c][4 * i + 1], scale2, l4.x, d4.x, col >= lim && col <= hi,
-                         col + 1 >= lim && col + 1 <= hi, pr[2 * i], pt[2 * i]);
-      score_pair<MASKED>(xs[c][4 * i + 2], xs[c][4 * i + 3], xp[c][4 * i + 2], xp[c][4 * i + 3], scale2, l4.y, d4.y,
-                         col + 2 >= lim && col + 2 <= hi, col + 3 >= lim && col + 3 <= hi, pr[2 * i + 1], pt[2 * i + 1]);
+      float t0, t1, t2, t3;
+      f32x2_split(mul2(f32x2(p[col], p[col + 1]), add2(f32x2_bits(xp[c][4 * i], xp[c][4 * i + 1]), d4.x)), t0, t1);
+      f32x2_split(mul2(f32x2(p[col + 2], p[col + 3]), add2(f32x2_bits(xp[c][4 * i + 2], xp[c][4 * i + 3]), d4.y)), t2, t3);
+      pt[2 * i] = pack_bf16x2(t0, t1);
+      pt[2 * i + 1] = pack_bf16x2(t2, t3);
     }
-    tmem_st8(tS + 16 * c, pr);
     tmem_st8(tS + 16 * c + 8, pt);
   }
 }
@@ -573,7 +605,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   uint8_t *sOut = sStage + S * C::kDkvStageBytes;   // staging (dK tile, then dV tile) when separate
 
   __shared__ uint64_t bar_res_full, bar_res_free, bar_q_full[S], bar_q_empty[S];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
+  __shared__ uint64_t bar_s_full[NB], bar_dp_full[NB], bar_r_ready[NB], bar_t_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -591,7 +623,10 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     mbar_init(&bar_res_full, 1);
     mbar_init(&bar_res_free, 2);
     for (int s = 0; s < S; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
-    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128 * C::kSlices); mbar_init(&bar_buf_free[b], 1); }
+    for (int b = 0; b < NB; ++b) {
+      mbar_init(&bar_s_full[b], 1); mbar_init(&bar_dp_full[b], 1); mbar_init(&bar_buf_free[b], 1);
+      mbar_init(&bar_r_ready[b], 128 * C::kSlices); mbar_init(&bar_t_ready[b], 128 * C::kSlices);
+    }
     mbar_init(&bar_acc_done, 1);
     mbar_init(&bar_acc_free, C::kCompute);
     mbar_init(&bar_drain[0], 1);
@@ -682,12 +717,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
             umma_ss(tS, dscK.at(oa), dscQ.at(ob), idesc_s, k > 0);
           }
+          umma_commit(&bar_s_full[b]);                      // phase 1 of the ALUs needs only S^T
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
             umma_ss(tdP, dscV.at(oa), dscdO.at(ob), idesc_s, k > 0);
           }
-          umma_commit(&bar_sdp_full[b]);
+          umma_commit(&bar_dp_full[b]);
           if (n == T - 1) umma_commit(&bar_res_free);   // no MMA reads this K / V tile any more
         }
         __syncwarp();
@@ -705,37 +741,40 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       if (ti > 0) mbar_wait(&bar_acc_free, (ti - 1) & 1, ab, kDkvWaitAccFree);   // the previous epilogue has read dV, dK
       for (int p = 0; p < T; ++p, ++g) {
         const int st = g % S, b = g % NB;
-        mbar_wait(&bar_tr_ready[b], (g / NB) & 1, ab, kDkvWaitTR);
-        tc_fence_after();
         const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes),
                        dscZ = dscdO.advanced(C::kStepTileBytes);
         // packed BF16 operands of query slice k (16 queries): r^T over columns 16 k .. 16 k + 7 of the buffer, t^T over the next eight
         const uint32_t tR = tmem_base + 128 * b, tT = tR + 8;
         const uint32_t acc = (p > 0) ? 1u : 0u;
+        mbar_wait(&bar_r_ready[b], (g / NB) & 1, ab, kDkvWaitTR);        // r^T is complete: its products run while t^T is computed
+        tc_fence_after();
         if (elect_one_sync()) {
           if (D == 64 && use_z) {
             // d = 64: the dO and Z step tiles are adjacent 64-column atoms of one MN-major operand and the dV and dK
             // accumulators are adjacent TMEM columns, so r^T [dO | Z] is ONE full-rate N = 128 product
-            // (an N = 64 instruction costs as much as 0.7 of an N = 128 one).  dK gets its main term t^T Q afterwards.
+            // (an N = 64 instruction costs as much as 0.7 of an N = 128 one).
 #pragma unroll
             for (int k = 0; k < C::kStepRows / 16; ++k)    // [dV | dK] += r^T [dO | -BF16(lambda Q)]
               umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_fused, k > 0 ? 1u : acc);
-#pragma unroll
-            for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += t^T Q
-              umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, 1u);
           } else {
 #pragma unroll
             for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
               umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-#pragma unroll
-            for (int k = 0; k < C::kStepRows / 16; ++k)      // dK += t^T Q
-              umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
             if (use_z) {
 #pragma unroll
               for (int k = 0; k < C::kStepRows / 16; ++k)    // dK += r^T (-BF16(lambda Q))   (Algorithm 1 lines 17-18)
-                umma_ts(tmem_base + C::kColAcc1, tR + 16 * k, dscZ.at(k * 2048), idesc_a, 1u);
+                umma_ts(tmem_base + C::kColAcc1, tR + 16 * k, dscZ.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
             }
           }
+        }
+        __syncwarp();
+        mbar_wait(&bar_t_ready[b], (g / NB) & 1, ab, kDkvWaitTR);
+        tc_fence_after();
+        if (elect_one_sync()) {
+          const uint32_t acc_k = use_z ? 1u : acc;           // with the correction, dK already holds this step's r^T Z
+#pragma unroll
+          for (int k = 0; k < C::kStepRows / 16; ++k)        // dK += t^T Q
+            umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc_k);
           umma_commit(&bar_buf_free[b]);
           umma_commit(&bar_q_empty[st]);
           if (p == T - 1) umma_commit(&bar_acc_done);
@@ -761,19 +800,26 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         const int g = g0 + n, st = g % S, b = g % NB;
         // The scores of this step were issued after its stage (and with it the row statistics) had landed in shared
         // memory, so their completion covers both.
-        mbar_wait(&bar_sdp_full[b], (g / NB) & 1, ab, kDkvWaitSdP);
+        mbar_wait(&bar_s_full[b], (g / NB) & 1, ab, kDkvWaitSdP);
         tc_fence_after();
         const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
         const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes) + C::kSliceCols * slice;
         const int nh = n % Th;                                      // step within the current query head
         const int q0 = q_start + nh * C::kStepRows + C::kSliceCols * slice;   // query row (inside the head) of the slice's column 0
+        float pkeep[32];
         if ((CAUSAL && nh < 2) || q_start + (nh + 1) * C::kStepRows > tl.seq_end)
-          dkv_slice<true>(tS16, tdP16, nl, nl + 64, scale_log2, CAUSAL ? tl.row0 + row - q0 : 0, tl.seq_end - 1 - q0);
+          dkv_phase1<true>(tS16, nl, scale_log2, CAUSAL ? tl.row0 + row - q0 : 0, tl.seq_end - 1 - q0, pkeep);
         else
-          dkv_slice<false>(tS16, tdP16, nl, nl + 64, scale_log2, 0, 0);
+          dkv_phase1<false>(tS16, nl, scale_log2, 0, 0, pkeep);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&bar_tr_ready[b]);
+        mbar_arrive(&bar_r_ready[b]);
+        mbar_wait(&bar_dp_full[b], (g / NB) & 1, ab, kDkvWaitSdP);
+        tc_fence_after();
+        dkv_phase2(tS16, tdP16, nl + 64, pkeep);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bar_t_ready[b]);
       }
 
       mbar_wait(&bar_acc_done, ti & 1, ab, kDkvWaitAcc);

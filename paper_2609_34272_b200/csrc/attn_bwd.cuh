@@ -24,7 +24,9 @@
 // 32-column slice)).  A buffer is back with the tensor core after half the ALU time one warpgroup per step would
 // take -- that time bounds the loop  scores -> ALUs -> second-stage products -> buffer free  each buffer runs
 // through -- while the two groups, at different phases, hide each other's TMEM and barrier latencies.
-// The packed BF16 operands r / t overwrite the consumed S columns of their own 16-column chunk.  The tensor-core queue is only one or two instructions deep, so an issuing warp is stalled
+// The packed BF16 operands r / t overwrite the consumed S columns of their own 16-column chunk.
+// The dK/dV kernel further splits a step's arithmetic in two phases with their own barriers (r^T from S^T first, then
+// t^T from dP^T), so that dV += r^T dO and dK += r^T Z run on the tensor core while t^T is still being computed.  The tensor-core queue is only one or two instructions deep, so an issuing warp is stalled
 // for as long as its MMAs execute and anything else it does (barrier polls, commits) would idle the pipe.
 // Two warps therefore issue: warp 1 the score products of every step, warp 2 the second-stage products; each
 // one's bookkeeping overlaps the other's MMAs.  Reuse of a score buffer is ordered by an explicit barrier

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "attn_bwd.cuh"
+#include "attn_bwd_w128.cuh"
 #include "attn_fwd.cuh"
 
 namespace {
@@ -94,12 +95,12 @@ int device_state(DeviceState **out) {
       ok &= allow_smem(attn_fwd_kernel<128, false, false, 2>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
       ok &= allow_smem(attn_fwd_kernel<128, false, true, 0>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
       ok &= allow_smem(attn_fwd_kernel<128, false, true, 2>, FwdCfg<128>::kSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dkv_w128_kernel<true>, BwdW128::kDkvSmemBytes) == cudaSuccess;
+      ok &= allow_smem(bwd_dkv_w128_kernel<false>, BwdW128::kDkvSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, true>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<64, false>, BwdCfg<64>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<128, true>, BwdCfg<128>::kDqSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dq_kernel<128, false>, BwdCfg<128>::kDqSmemBytes) == cudaSuccess;
-      ok &= allow_smem(bwd_dkv_kernel<64, true>, BwdCfg<64>::kDkvSmemBytes) == cudaSuccess;
-      ok &= allow_smem(bwd_dkv_kernel<64, false>, BwdCfg<64>::kDkvSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dkv_kernel<128, true>, BwdCfg<128>::kDkvSmemBytes) == cudaSuccess;
       ok &= allow_smem(bwd_dkv_kernel<128, false>, BwdCfg<128>::kDkvSmemBytes) == cudaSuccess;
       if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
@@ -141,8 +142,10 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
                void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
                int n_plan_tiles, int nblk, void *stream);
 
-// Row statistics {-LSE log2 e, -D}: per head ceil(N / 64) blocks of 64 rows (the last one zero-padded), 512 B each.
-size_t stats_bytes(int heads, int N) { return align256(static_cast<size_t>(heads) * ((N + 63) / 64) * 512); }
+// Row statistics {-LSE log2 e, -D}: blocks of 64 rows, 512 B each (per head ceil(N / 64) of them, the last one
+// zero-padded), plus one spare block: the 128-wide steps fetch two blocks at a time and may reach one past the end.
+size_t stats_blocks_bytes(size_t blocks) { return align256((blocks + 1) * 512); }
+size_t stats_bytes(int heads, int N) { return stats_blocks_bytes(static_cast<size_t>(heads) * ((N + 63) / 64)); }
 
 }  // namespace
 
@@ -266,7 +269,7 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
     return GPROJ_ERR_FLAGS;
   const bool run_dq = !(flags & GPROJ_FLAG_ONLY_DKV_PASS), run_dkv = !(flags & GPROJ_FLAG_ONLY_DQ_PASS);
   if (!run_dq && !run_dkv) return GPROJ_ERR_FLAGS;
-  const size_t stats_sz = align256(static_cast<size_t>(B) * H * nblk * 512);
+  const size_t stats_sz = stats_blocks_bytes(static_cast<size_t>(B) * H * nblk);
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
       workspace_bytes < stats_sz + align256(static_cast<size_t>(B) * H * N * static_cast<size_t>(d) * 2))
     return GPROJ_ERR_WORKSPACE;
@@ -307,8 +310,23 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
           flags,                                                                                                        \
           st->status_ptr);                                                                                              \
   } while (0)
-  if (d == 64) { if (causal) GPROJ_LAUNCH_BWD(64, true); else GPROJ_LAUNCH_BWD(64, false); }
+  // At d = 64 the dK/dV side runs with 128-wide steps (every score product an N = 128 instruction); it streams 128-row
+  // boxes, which the stationary-tile maps of the dQ side already are.
+#define GPROJ_LAUNCH_BWD_W128(CC)                                                                                       \
+  do {                                                                                                                  \
+    if (run_dq)                                                                                                         \
+      bwd_dq_kernel<64, CC><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kDqSmemBytes, s>>>(                                \
+          mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, static_cast<__nv_bfloat16 *>(dQ), Zneg, plan_q,    \
+          nblk, N, BH, H, G, total_tiles, scale_log2, softmax_scale, flags, st->status_ptr);                              \
+    if (run_dkv)                                                                                                        \
+      bwd_dkv_w128_kernel<CC><<<grid_kv, BwdW128::kThreads, BwdW128::kDkvSmemBytes, s>>>(                                \
+          mK128, mV128, mQ128, mdO128, mZst, mdKst, mdVst, stats, static_cast<__nv_bfloat16 *>(dK),                       \
+          static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,    \
+          flags, st->status_ptr);                                                                                       \
+  } while (0)
+  if (d == 64) { if (causal) GPROJ_LAUNCH_BWD_W128(true); else GPROJ_LAUNCH_BWD_W128(false); }
   else         { if (causal) GPROJ_LAUNCH_BWD(128, true); else GPROJ_LAUNCH_BWD(128, false); }
+#undef GPROJ_LAUNCH_BWD_W128
 #undef GPROJ_LAUNCH_BWD
   if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
   tl_launch_count = (run_dq ? 1 : 0) + (run_dkv ? 1 : 0);
@@ -397,7 +415,7 @@ int gproj_attn_fwd_varlen(const void *Q, const void *K, const void *V, void *O, 
 size_t gproj_attn_bwd_varlen_workspace_bytes(const int *cu_seqlens, int num_seqs, int H, int d) {
   PackedShape ps;
   if (!packed_shape(cu_seqlens, num_seqs, &ps) || check_shape(1, H, ps.total, d) != GPROJ_OK) return 0;
-  return align256(static_cast<size_t>(H) * ps.nblk * 512) + align256(static_cast<size_t>(H) * ps.total * static_cast<size_t>(d) * 2);
+  return stats_blocks_bytes(static_cast<size_t>(H) * ps.nblk) + align256(static_cast<size_t>(H) * ps.total * static_cast<size_t>(d) * 2);
 }
 
 int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,

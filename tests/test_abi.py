@@ -42,9 +42,10 @@ def test_workspace_bytes(lib):
     # one BF16 query-shaped array + two FP32 row arrays (the paper's "Cost" paragraph allows more)
     B, H, N, d = 2, 3, 256, 64
     rows = B * H * N
-    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, d) == rows * 8 + rows * d * 2
+    # row statistics: 8 bytes per row in 64-row blocks plus one spare block (256-byte aligned), then the BF16 array
+    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, d) == rows * 8 + 512 + rows * d * 2
     # ragged length: statistics are padded to whole 64-row blocks per head (2 blocks x 512 B), the query-shaped array is not
-    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 2 * 512 + 100 * 64 * 2
+    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 3 * 512 + 100 * 64 * 2
     assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 0, 64) == 0
     assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 128, 96) == 0
 

@@ -169,7 +169,7 @@ int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const v
  * that much memory until the process exits.
  *   - Same inputs, outputs, flags and arithmetic as gproj_attn_bwd; results are bitwise the same.
  *   - Shapes whose gproj_attn_bwd_workspace_bytes() exceeds GPROJ_STATIC_SCRATCH_BYTES are rejected with
- *     GPROJ_ERR_WORKSPACE (workloads up to B*H*N*d = 8 Mi elements at d = 64 fit); nothing is launched.
+ *     GPROJ_ERR_WORKSPACE (problems up to about 7.5 Mi elements B*H*N*d at d = 64 fit, e.g. B*H = 16, N = 4096); nothing is launched.
  *   - The first call on each device looks up the array's device address (with that device current); make
  *     that first call before any stream capture begins.  No call allocates or frees anything.
  *   - All calls on a device share the one array, and it keeps whatever the last call left there.  Nothing

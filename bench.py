@@ -263,8 +263,8 @@ def main():
         "fwd_tflops": world * fl["fwd"] / fwd_t / 1e12,
         "bwd_frac_of_bf16_peak": value / world / peak, "peak_source": peak_kind,
         "wall_ms_per_step_incl_l2_flush": 1e3 * wall / steps,
-        "kernels_ms": {"bwd_dq_kernel": dq_ms, "bwd_dkv_kernel": dkv_ms},
-        "roofline": {"bound": "tensor", "kernel": "bwd_dkv_kernel", "achieved": dkv_achieved, "peak": peak, "unit": "TFLOP/s",
+        "kernels_ms": {"bwd_dq_kernel": dq_ms, ("bwd_dkv_w128_kernel" if w.d == 64 else "bwd_dkv_kernel"): dkv_ms},
+        "roofline": {"bound": "tensor", "kernel": "bwd_dkv_w128_kernel" if w.d == 64 else "bwd_dkv_kernel", "achieved": dkv_achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": dkv_achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(("bwd_dkv_kernel", args.workload)),
                      "peak_source": peak_kind + (" (sustained bf16 GEMM, run was power-capped)" if capped else " (burst bf16 GEMM)"),
                      "algorithmic_flops_per_launch": fl["dkv_kernel"]},

@@ -52,7 +52,6 @@ def run_gpu(inp, lens, alpha, causal, flags=0):
     cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
     plan = g.VarlenPlan(cu, causal)
     dev = {k: v.cuda() for k, v in inp.items()}
-    # poison the outputs' memory pool first so that a row nobody writes cannot pass by luck
     O, LSE = g.gproj_attn_fwd_varlen(dev["Q"], dev["K"], dev["V"], plan, alpha)
     dQ, dK, dV = g.gproj_attn_bwd_varlen(dev["Q"], dev["K"], dev["V"], O, LSE, dev["dO"], plan, alpha, flags=flags)
     rc, detail = g.gproj_last_device_status()

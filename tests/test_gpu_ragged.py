@@ -114,3 +114,28 @@ def test_minus24_witness_at_its_own_size():
     assert np.all(on["O"][0, 0, :, 0] == vals["o"][0]) and np.all(on["O"][0, 0, :, 1] == vals["o"][1])
     assert np.all(on["dQ"][0, 0, :, 0] == vals["dq0_gproj"][0])
     assert np.all(off["dQ"][0, 0, :, 0] == vals["dq0_uncorrected"][0])
+
+
+def test_many_heads_short_sequences():
+    # more (batch, head) problems than SMs, one tile each: exercises the tile -> (head, tile) decode of the persistent
+    # schedule far from the benchmark shapes
+    w = Workload("many_heads", 8, 40, 96, 64, True, k_offset=4.0, seed=4711)
+    inp = make_inputs(w)
+    ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, True)
+    check(run_gpu(inp, w.softmax_scale, True), ex)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes(seed):
+    # seeded random shapes: lengths off every grid, head counts with and without grouping, both head dimensions
+    rng = np.random.default_rng(1234 + seed)
+    d = int(rng.choice([64, 128]))
+    Hkv = int(rng.integers(1, 4))
+    G = int(rng.choice([1, 1, 2, 3]))
+    B = int(rng.integers(1, 3))
+    N = int(rng.integers(2, 700))
+    causal = bool(rng.integers(0, 2))
+    w = Workload("rand", B, Hkv * G, N, d, causal, k_offset=float(rng.choice([0.0, 4.0, 16.0])), seed=900 + seed, Hkv=Hkv)
+    inp = make_inputs(w)
+    ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, causal)
+    print("shape", B, Hkv * G, Hkv, N, d, causal, check(run_gpu(inp, w.softmax_scale, causal), ex))

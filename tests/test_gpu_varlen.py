@@ -126,3 +126,19 @@ def test_malformed_cu_seqlens_is_rejected():
     for bad in ([1, 5], [0, 5, 3], [0, 0]):
         with pytest.raises(g.GprojError):
             g.VarlenPlan(bad, True)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_packings(seed):
+    rng = np.random.default_rng(4321 + seed)
+    d = int(rng.choice([64, 128]))
+    Hkv = int(rng.integers(1, 3))
+    G = int(rng.choice([1, 2]))
+    lens = [int(x) for x in rng.integers(0, 400, size=int(rng.integers(2, 7)))]
+    lens = [0 if n == 1 else n for n in lens]      # one-token sequences (exact zero dQ, dK) have their own dense test
+    if sum(lens) == 0:
+        lens[0] = 17
+    causal = bool(rng.integers(0, 2))
+    inp = make_packed(Hkv * G, Hkv, lens, d, seed=7000 + seed)
+    alpha = float(np.float32(d ** -0.5))
+    print("packing", lens, Hkv * G, Hkv, d, causal, check(run_gpu(inp, lens, alpha, causal), oracle_packed(inp, lens, alpha, causal)))

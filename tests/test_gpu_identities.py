@@ -231,3 +231,37 @@ def test_host_buffer_entry_point_matches_device_calls():
     with pytest.raises(g.GprojError) as e:
         g.gproj_attn_fwd_bwd_host(host["Q"], host["K"], host["V"], host["dO"], hdQ, hdK, hdV, w.softmax_scale, True, small)
     assert e.value.status == -4
+
+
+def test_cuda_graph_capture_and_replay():
+    # The entry points only enqueue work on the given stream (no allocation, no synchronisation once the per-device
+    # set-up of the first call is done), so forward + backward can be captured into a CUDA graph and replayed.
+    w = Workload("graph", 1, 4, 512, 64, True, k_offset=4.0, seed=17)
+    inp = {k: v.cuda() for k, v in make_inputs(w).items()}
+    O = torch.empty_like(inp["Q"]); LSE = torch.empty(w.B, w.H, w.N, dtype=torch.float32, device="cuda")
+    dQ, dK, dV = (torch.empty_like(inp["Q"]) for _ in range(3))
+    ws = torch.empty(g.gproj_attn_bwd_workspace_bytes(w.B, w.H, w.N, w.d), dtype=torch.uint8, device="cuda")
+
+    def step():
+        g.gproj_attn_fwd(inp["Q"], inp["K"], inp["V"], w.softmax_scale, True, O=O, LSE=LSE)
+        g.gproj_attn_bwd(inp["Q"], inp["K"], inp["V"], O, LSE, inp["dO"], w.softmax_scale, True, workspace=ws, dQ=dQ, dK=dK, dV=dV)
+
+    step()                                               # eager: also performs the one-time set-up
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (O, LSE, dQ, dK, dV)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                           # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in (O, LSE, dQ, dK, dV):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, hex(detail)
+    for a, b in zip(ref, (O, LSE, dQ, dK, dV)):
+        assert torch.equal(a, b)

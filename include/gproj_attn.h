@@ -12,8 +12,8 @@
  *     causal != 0 means row i attends to j <= i.  The *_gqa entry points take separate query / KV head counts.
  *   - The caller owns all memory.  The library never allocates, frees or synchronises; work is
  *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).
- *     After the first call on a device (one-time attribute set-up) the compute entry points can be captured
- *     into a CUDA graph.
+ *     After the first call on a device (one-time attribute set-up), gproj_attn_fwd and gproj_attn_bwd with a
+ *     caller-supplied workspace have been captured into a CUDA graph and replayed (that is what is tested).
  *   - Return value: GPROJ_OK (0) or a negative gproj_status.  Nothing throws, aborts or traps.
  *     Inputs are never modified; outputs are fully overwritten; non-finite inputs are undefined
  *     behaviour (the paper's error decomposition assumes finite quantities).

@@ -14,6 +14,7 @@ Two tiers:
 """
 from .exact import (  # noqa: F401
     attn_fwd_bwd_f64,
+    attn_rect_f64,
     head_rows_f64,
     head_keys_f64,
     num_threads,

@@ -28,6 +28,14 @@ def _load():
         lib.gproj_oracle_head_keys.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_int, ctypes.c_int,
                                                ctypes.c_double, ctypes.c_int, f64p, f64p, i32p, ctypes.c_int,
                                                f64p, f64p]
+        lib.gproj_oracle_rect_rows.restype = ctypes.c_int
+        lib.gproj_oracle_rect_rows.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                               ctypes.c_double, ctypes.c_int, i32p, ctypes.c_int,
+                                               f64p, f64p, f64p, f64p]
+        lib.gproj_oracle_rect_keys.restype = ctypes.c_int
+        lib.gproj_oracle_rect_keys.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                               ctypes.c_double, ctypes.c_int, f64p, f64p, i32p, ctypes.c_int,
+                                               f64p, f64p]
         lib.gproj_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -123,6 +131,42 @@ def attn_fwd_bwd_f64(Q, K, V, dO, alpha, causal, heads=None):
             out[key] = out[key].reshape((B, H) + out[key].shape[1:])
         for key in ("dK", "dV"):
             out[key] = out[key].reshape((B, Hkv) + out[key].shape[1:])
+    return out
+
+
+def attn_rect_f64(Q, K, V, dO, alpha, causal):
+    """Exact forward and VJP with N_q queries and N_k keys: Q, dO ``[B, H, Nq, d]``, K, V ``[B, Hkv, Nk, d]`` (BF16 bits).
+
+    Causal support of query i: keys j <= i + (Nk - Nq) (the diagonal ends at the last query and the last key); a row with
+    an empty support has O = dQ = 0 and LSE = +inf (Algorithm 1, line 14, gives such a row no correction either).
+    Returns O, LSE, MUA, dQ ([B, H, Nq, ..]) and dK, dV ([B, Hkv, Nk, d]) in FP64.
+    """
+    Q, K, V, dO = map(_u16, (Q, K, V, dO))
+    B, H, Nq, d = Q.shape
+    Hkv, Nk = K.shape[1], K.shape[2]
+    if K.shape != (B, Hkv, Nk, d) or V.shape != K.shape or dO.shape != Q.shape or H % Hkv != 0:
+        raise ValueError("shape mismatch")
+    G = H // Hkv
+    out = {"O": np.empty((B, H, Nq, d)), "LSE": np.empty((B, H, Nq)), "MUA": np.empty((B, H, Nq)), "dQ": np.empty((B, H, Nq, d)),
+           "dK": np.zeros((B, Hkv, Nk, d)), "dV": np.zeros((B, Hkv, Nk, d))}
+    rows = np.arange(Nq, dtype=np.int32); keys = np.arange(Nk, dtype=np.int32)
+    lib = _load()
+    for b in range(B):
+        for h in range(H):
+            q, u, k, v = Q[b, h], dO[b, h], K[b, h // G], V[b, h // G]
+            args = (_p(q, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(v, ctypes.c_uint16), _p(u, ctypes.c_uint16),
+                    Nq, Nk, d, float(alpha), int(bool(causal)))
+            O = np.empty((Nq, d)); LSE = np.empty(Nq); MUA = np.empty(Nq); dQ = np.empty((Nq, d))
+            if lib.gproj_oracle_rect_rows(*args, _p(rows, ctypes.c_int), Nq, _p(O, ctypes.c_double), _p(LSE, ctypes.c_double),
+                                          _p(MUA, ctypes.c_double), _p(dQ, ctypes.c_double)) != 0:
+                raise RuntimeError("gproj_oracle_rect_rows failed")
+            dK = np.empty((Nk, d)); dV = np.empty((Nk, d))
+            if lib.gproj_oracle_rect_keys(*args, _p(LSE, ctypes.c_double), _p(MUA, ctypes.c_double), _p(keys, ctypes.c_int), Nk,
+                                          _p(dK, ctypes.c_double), _p(dV, ctypes.c_double)) != 0:
+                raise RuntimeError("gproj_oracle_rect_keys failed")
+            out["O"][b, h], out["LSE"][b, h], out["MUA"][b, h], out["dQ"][b, h] = O, LSE, MUA, dQ
+            out["dK"][b, h // G] += dK
+            out["dV"][b, h // G] += dV
     return out
 
 

@@ -160,3 +160,106 @@ int gproj_oracle_head_keys(const uint16_t *q, const uint16_t *k, const uint16_t 
     free(Q); free(K); free(V); free(U);
     return 0;
 }
+
+/*
+ * Rectangular problems: N_q queries against N_k keys of one head (the paper's synthetic suite lists "unequal lengths" and
+ * "empty causal rows", Appendix "Synthetic Numerical Suite"; Algorithm 1 line 14 gives the rule for a row of zero mass).
+ * Support of query row i: all keys (causal = 0), or the keys j <= i + (N_k - N_q), i.e. the causal diagonal ends at the
+ * LAST query and the LAST key (the alignment of the FlashAttention kernels the paper builds on).  A row whose support is
+ * empty has no probabilities: O_i = 0, dq_i = 0, mu_a,i = 0, it contributes to no dk_j / dv_j, and its LSE is reported
+ * as +infinity, so that exp(s - LSE) = 0 wherever that row is re-evaluated.
+ * These are separate functions; the square ones above are left as they were.
+ */
+int gproj_oracle_rect_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v, const uint16_t *u,
+                           int Nq, int Nk, int d, double alpha, int causal,
+                           const int *rows, int nrows,
+                           double *O, double *LSE, double *MUA, double *dQ)
+{
+    if (Nq <= 0 || Nk <= 0 || d <= 0 || nrows < 0) return -1;
+    double *Q = decode_tile(q, (size_t)Nq * d), *K = decode_tile(k, (size_t)Nk * d);
+    double *V = decode_tile(v, (size_t)Nk * d), *U = decode_tile(u, (size_t)Nq * d);
+    int fail = (!Q || !K || !V || !U);
+    const int off = Nk - Nq;
+
+#pragma omp parallel
+    {
+        double *s = (double *)malloc((size_t)Nk * sizeof(double));
+        double *a = (double *)malloc((size_t)Nk * sizeof(double));
+        if (!s || !a) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for schedule(dynamic, 4)
+            for (int r = 0; r < nrows; ++r) {
+                int i = rows[r];
+                int L = causal ? i + off + 1 : Nk;          /* number of supported keys: j = 0 .. L-1 */
+                if (L > Nk) L = Nk;
+                double *o = O + (size_t)r * d, *dq = dQ + (size_t)r * d;
+                for (int c = 0; c < d; ++c) { o[c] = 0.0; dq[c] = 0.0; }
+                if (L <= 0) { LSE[r] = INFINITY; MUA[r] = 0.0; continue; }
+                const double *qi = Q + (size_t)i * d, *ui = U + (size_t)i * d;
+                double smax = -INFINITY;
+                for (int j = 0; j < L; ++j) {
+                    const double *kj = K + (size_t)j * d, *vj = V + (size_t)j * d;
+                    double dot = 0.0, av = 0.0;
+                    for (int c = 0; c < d; ++c) { dot += qi[c] * kj[c]; av += ui[c] * vj[c]; }
+                    s[j] = alpha * dot;
+                    a[j] = av;
+                    if (s[j] > smax) smax = s[j];
+                }
+                double Z = 0.0;
+                for (int j = 0; j < L; ++j) Z += exp(s[j] - smax);
+                double mua = 0.0;
+                for (int j = 0; j < L; ++j) { s[j] = exp(s[j] - smax) / Z; mua += s[j] * a[j]; }   /* s now holds p */
+                for (int j = 0; j < L; ++j) {
+                    const double *kj = K + (size_t)j * d, *vj = V + (size_t)j * d;
+                    double p = s[j], g = p * (a[j] - mua);
+                    for (int c = 0; c < d; ++c) { o[c] += p * vj[c]; dq[c] += g * kj[c]; }
+                }
+                for (int c = 0; c < d; ++c) dq[c] *= alpha;
+                LSE[r] = smax + log(Z);
+                MUA[r] = mua;
+            }
+        }
+        free(s);
+        free(a);
+    }
+    free(Q); free(K); free(V); free(U);
+    return fail ? -1 : 0;
+}
+
+int gproj_oracle_rect_keys(const uint16_t *q, const uint16_t *k, const uint16_t *v, const uint16_t *u,
+                           int Nq, int Nk, int d, double alpha, int causal,
+                           const double *LSE, const double *MUA,
+                           const int *keys, int nkeys,
+                           double *dK, double *dV)
+{
+    if (Nq <= 0 || Nk <= 0 || d <= 0 || nkeys < 0) return -1;
+    double *Q = decode_tile(q, (size_t)Nq * d), *K = decode_tile(k, (size_t)Nk * d);
+    double *V = decode_tile(v, (size_t)Nk * d), *U = decode_tile(u, (size_t)Nq * d);
+    if (!Q || !K || !V || !U) { free(Q); free(K); free(V); free(U); return -1; }
+    const int off = Nk - Nq;
+
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int r = 0; r < nkeys; ++r) {
+        int j = keys[r];
+        const double *kj = K + (size_t)j * d, *vj = V + (size_t)j * d;
+        double *dk = dK + (size_t)r * d, *dv = dV + (size_t)r * d;
+        for (int c = 0; c < d; ++c) { dk[c] = 0.0; dv[c] = 0.0; }
+        int i0 = causal ? j - off : 0;                      /* first query whose support holds key j */
+        if (i0 < 0) i0 = 0;
+        for (int i = i0; i < Nq; ++i) {
+            const double *qi = Q + (size_t)i * d, *ui = U + (size_t)i * d;
+            double dot = 0.0, av = 0.0;
+            for (int c = 0; c < d; ++c) { dot += qi[c] * kj[c]; av += ui[c] * vj[c]; }
+            double p = exp(alpha * dot - LSE[i]);
+            double g = p * (av - MUA[i]);
+            for (int c = 0; c < d; ++c) { dk[c] += g * qi[c]; dv[c] += p * ui[c]; }
+        }
+        for (int c = 0; c < d; ++c) dk[c] *= alpha;
+    }
+    free(Q); free(K); free(V); free(U);
+    return 0;
+}

@@ -116,6 +116,26 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
                       unsigned fwd_flags, void *stream);
 
 /*
+ * Unequal query and key lengths (Appendix "Synthetic Numerical Suite": unequal lengths, empty causal rows).  Q, O, dO, dQ
+ * are [B][H][Nq][d] and LSE [B][H][Nq]; K, V, dK, dV are [B][Hkv][Nk][d]; Nq >= 1, Nk >= 1, otherwise as the grouped-query
+ * functions, which are the case Nq = Nk.  Non-causal: every query sees all Nk keys.  Causal: the diagonal ends at the
+ * last query and the last key, i.e. the support of query i is the keys j <= i + (Nk - Nq) (the paper does not fix an
+ * alignment; this is the one under which appending cached keys in front of a block of new queries stays causal).  For
+ * Nq > Nk the first Nq - Nk queries then have an EMPTY support: their O and dQ rows are written as zero and their LSE as
+ * +infinity, so that P = exp(S - LSE) = 0 wherever the backward meets them; they add nothing to dK or dV, and they get
+ * no correction (Algorithm 1, line 14: lambda = 0 when the rounded row mass is zero).  The backward takes the LSE this
+ * forward wrote.  Workspace: gproj_attn_bwd_workspace_bytes(B, H, Nq, d), i.e. sized by the QUERY rows.  Errors as for
+ * gproj_attn_fwd_ex / gproj_attn_bwd_gqa, with GPROJ_ERR_SHAPE also for Nk <= 0 or B*Hkv*Nk >= 2^31.
+ */
+int gproj_attn_fwd_rect(const void *Q, const void *K, const void *V, void *O, float *LSE,
+                        int B, int H, int Hkv, int Nq, int Nk, int d, float softmax_scale, int causal,
+                        unsigned fwd_flags, void *stream);
+int gproj_attn_bwd_rect(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                        void *dQ, void *dK, void *dV,
+                        int B, int H, int Hkv, int Nq, int Nk, int d, float softmax_scale, int causal,
+                        void *workspace, size_t workspace_bytes, unsigned flags, void *stream);
+
+/*
  * Packed (variable-length) sequences.  The paper's synthetic suite exercises "packed segments" and "unequal lengths"
  * (Appendix "Synthetic Numerical Suite"); its training layout packs documents into one row axis.  Here the tensors are
  * [H][T][d] (queries, O, dO, dQ) and [Hkv][T][d] (keys, values, dK, dV) with T = cu_seqlens[num_seqs] rows per head; sequence

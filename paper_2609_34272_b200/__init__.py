@@ -12,11 +12,13 @@ from .binding import (  # noqa: F401
     GprojError,
     VarlenPlan,
     gproj_attn_bwd,
+    gproj_attn_bwd_rect,
     gproj_attn_bwd_static_scratch,
     gproj_attn_bwd_varlen,
     gproj_attn_bwd_workspace_bytes,
     gproj_attn_fwd,
     gproj_attn_fwd_bwd_host,
+    gproj_attn_fwd_rect,
     gproj_attn_host_staging_bytes,
     gproj_attn_fwd_varlen,
     gproj_last_device_status,

@@ -22,7 +22,7 @@ FWD_FLAG_FMA_SOFTMAX = 1
 STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd", "gproj_attn_fwd_gqa", "gproj_attn_bwd_gqa", "gproj_attn_fwd_ex",
-           "gproj_attn_bwd_static_scratch",
+           "gproj_attn_bwd_static_scratch", "gproj_attn_fwd_rect", "gproj_attn_bwd_rect",
            "gproj_attn_varlen_plan_bytes", "gproj_attn_varlen_plan", "gproj_attn_fwd_varlen",
            "gproj_attn_bwd_varlen_workspace_bytes", "gproj_attn_bwd_varlen",
            "gproj_attn_host_staging_bytes", "gproj_attn_fwd_bwd_host",
@@ -59,6 +59,10 @@ def load():
         lib.gproj_attn_fwd_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, i, u, vp]
         lib.gproj_attn_bwd_gqa.restype = i
         lib.gproj_attn_bwd_gqa.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, sz, u, vp]
+        lib.gproj_attn_fwd_rect.restype = i
+        lib.gproj_attn_fwd_rect.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, u, vp]
+        lib.gproj_attn_bwd_rect.restype = i
+        lib.gproj_attn_bwd_rect.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, vp, sz, u, vp]
         lib.gproj_attn_bwd_static_scratch.restype = i
         lib.gproj_attn_bwd_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, f, i, u, vp]
         ip = ctypes.POINTER(ctypes.c_int)
@@ -171,6 +175,52 @@ def gproj_attn_bwd(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, workspac
                                            workspace.numel() * workspace.element_size(), int(flags), _stream(Q.device))
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_bwd")
+    return dQ, dK, dV
+
+
+def _rect_shapes(Q, K, V):
+    _check_bf16("Q", Q)
+    B, H, Nq, d = Q.shape
+    _check_bf16("K", K); _check_bf16("V", V, K.shape)
+    if K.dim() != 4 or K.shape[0] != B or K.shape[3] != d or H % K.shape[1] != 0:
+        raise ValueError(f"K/V shape {tuple(K.shape)} does not match Q {tuple(Q.shape)} (need [B, Hkv, Nk, d], H % Hkv == 0)")
+    return B, H, K.shape[1], Nq, K.shape[2], d
+
+
+def gproj_attn_fwd_rect(Q, K, V, softmax_scale, causal, O=None, LSE=None, fwd_flags=0):
+    """Forward with Nq queries and Nk keys: Q [B, H, Nq, d]; K, V [B, Hkv, Nk, d].  Causal: query i sees the keys
+    j <= i + (Nk - Nq); a query that sees none gets O = 0 and LSE = +inf."""
+    B, H, Hkv, Nq, Nk, d = _rect_shapes(Q, K, V)
+    O = torch.empty_like(Q) if O is None else O
+    LSE = torch.empty((B, H, Nq), dtype=torch.float32, device=Q.device) if LSE is None else LSE
+    _check_bf16("O", O, Q.shape)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_fwd_rect(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), B, H, Hkv, Nq, Nk, d,
+                                        float(softmax_scale), int(bool(causal)), int(fwd_flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_fwd_rect")
+    return O, LSE
+
+
+def gproj_attn_bwd_rect(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, workspace=None, dQ=None, dK=None, dV=None):
+    """Backward of gproj_attn_fwd_rect (same shapes; dK, dV like K).  Workspace: gproj_attn_bwd_workspace_bytes(B, H, Nq, d)."""
+    B, H, Hkv, Nq, Nk, d = _rect_shapes(Q, K, V)
+    for name, t in (("O", O), ("dO", dO)):
+        _check_bf16(name, t, Q.shape)
+    if not (LSE.is_cuda and LSE.dtype == torch.float32 and LSE.is_contiguous() and tuple(LSE.shape) == (B, H, Nq)):
+        raise TypeError("LSE must be a contiguous CUDA float32 tensor [B, H, Nq]")
+    if workspace is None:
+        workspace = torch.empty(max(gproj_attn_bwd_workspace_bytes(B, H, Nq, d), 256), dtype=torch.uint8, device=Q.device)
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(K) if dV is None else dV
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_bwd_rect(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
+                                        dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, Hkv, Nq, Nk, d, float(softmax_scale),
+                                        int(bool(causal)), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                        int(flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_bwd_rect")
     return dQ, dK, dV
 
 

@@ -98,13 +98,15 @@ struct TileSched {
 // One 128-row tile of one sequence.  Rows are counted inside a head ([heads][rows][d] tensors): dense calls have one
 // sequence [0, N) per head; packed (variable-length) calls have several, listed tile by tile in a plan the host
 // prepared: {row0, seq0, seq_end, blk0} with blk0 the sequence's first 64-row block of row statistics.
-struct TileInfo { int row0, seq0, seq_end, blk0; };
-__device__ __forceinline__ TileInfo tile_info(const int4 *plan, int idx, int dense_tile, int N) {
+// [oseq0, oseq_end) is the range of the OTHER operand's rows the tile works against (keys for a query tile, queries for a
+// key tile); it differs from [seq0, seq_end) only in dense calls with unequal query and key lengths.
+struct TileInfo { int row0, seq0, seq_end, blk0, oseq0, oseq_end; };
+__device__ __forceinline__ TileInfo tile_info(const int4 *plan, int idx, int dense_tile, int N, int N_other) {
   if (plan != nullptr) {
     const int4 e = __ldg(plan + idx);
-    return TileInfo{e.x, e.y, e.z, e.w};
+    return TileInfo{e.x, e.y, e.z, e.w, e.y, e.z};
   }
-  return TileInfo{128 * dense_tile, 0, N, 0};
+  return TileInfo{128 * dense_tile, 0, N, 0, 0, N_other};
 }
 // Rows [row0, row0 + 128) may be written by a TMA store (which clips at the tensor's end N) unless the tile is the
 // ragged tail of a sequence that is followed by another one.
@@ -259,7 +261,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const float *__restrict__ LSE, float *__restrict__ stats,
               __nv_bfloat16 *__restrict__ dQg, __nv_bfloat16 *__restrict__ Zg,   // plain-store targets of clipped tiles
               const int4 *__restrict__ plan, int nblk,                          // packed sequences: tile list; 64-row statistic blocks per head
-              int N, int BH, int Hq, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+              int N, int Nk, int BH, int Hq, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+  // N: query rows per head (own operand), Nk: key rows per head.  Causal support of query i: keys j <= i + (L_k - L_q).
   using C = BwdCfg<D>;
   constexpr int NB = C::kNB, R = C::kDqResBufs, S = C::kDqStages;
   extern __shared__ uint8_t smem_raw[];
@@ -305,11 +308,13 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 
   TileSched sched(total_tiles);
   // tile decode: causal -> longest rows first
-  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH), N); };
-  // 64-key steps of a query tile: its sequence's keys up to the tile's last row (causal) or all of them
+  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH), N, Nk); };
+  // 64-key steps of a query tile: the keys its last row sees (causal) or all of them; at least one step, fully masked
+  // if the tile sees no key at all, so that every tile runs through the same pipeline.
   auto steps_of = [&](const TileInfo &t) {
-    const int kend = CAUSAL ? min(t.row0 + 128, t.seq_end) : t.seq_end;
-    return (kend - t.seq0 + C::kStepRows - 1) / C::kStepRows;
+    const int Lk = t.oseq_end - t.oseq0, off = Lk - (t.seq_end - t.seq0);
+    const int kend = CAUSAL ? min(Lk, t.row0 - t.seq0 + 128 + off) : Lk;
+    return max(1, (max(kend, 0) + C::kStepRows - 1) / C::kStepRows);
   };
 
   if (warp == 0) {
@@ -324,7 +329,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kDqWaitKVEmpty);
           mbar_expect_tx(&bar_kv_full[st], C::kDqStageBytes);
           uint8_t *dst = sKV + st * C::kDqStageBytes;
-          const int kvh = kv_head_of(bh, Hq, G), krow = tl.seq0 + n * C::kStepRows;   // grouped-query: the group's shared K / V head
+          const int kvh = kv_head_of(bh, Hq, G), krow = tl.oseq0 + n * C::kStepRows;   // grouped-query: the group's shared K / V head
           for (int s = 0; s < C::kSlabs; ++s) {
             tma_load_3d(dst + s * C::kStepSlabBytes, &tmK, &bar_kv_full[st], s * 64, krow, kvh);
             tma_load_3d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmV, &bar_kv_full[st], s * 64, krow, kvh);
@@ -482,10 +487,15 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
         // Probabilities are zeroed beyond the causal diagonal and, in the ragged last step, for the zero-filled keys
         // past N (which would otherwise enter the row masses).  Rows of a causal tile never reach such keys.
-        const int key0 = tl.seq0 + n * C::kStepRows + C::kSliceCols * slice;   // row (inside the head) of the slice's column 0
-        if (CAUSAL && (n + 1) * C::kStepRows > tl.row0 - tl.seq0)              dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, qrow - key0, rho2, msum2);
-        else if (!CAUSAL && tl.seq0 + (n + 1) * C::kStepRows > tl.seq_end)     dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, tl.seq_end - 1 - key0, rho2, msum2);
-        else                                             dq_slice<false>(tS16, tdP16, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
+        const int Lk = tl.oseq_end - tl.oseq0, off = Lk - (tl.seq_end - tl.seq0);
+        const int krel0 = n * C::kStepRows + C::kSliceCols * slice;          // key (inside its sequence) of the slice's column 0
+        const bool masked = (CAUSAL && (n + 1) * C::kStepRows - 1 > tl.row0 - tl.seq0 + off) || (n + 1) * C::kStepRows > Lk;
+        if (masked) {
+          const int lim_c = CAUSAL ? qrow - tl.seq0 + off - krel0 : (1 << 30);
+          dq_slice<true>(tS16, tdP16, scale_log2, neg_lse2, Dv, min(lim_c, Lk - 1 - krel0), rho2, msum2);
+        } else {
+          dq_slice<false>(tS16, tdP16, scale_log2, neg_lse2, Dv, 0, rho2, msum2);
+        }
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar_tr_ready[b]);
@@ -593,7 +603,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const float *__restrict__ stats,
                __nv_bfloat16 *__restrict__ dKg, __nv_bfloat16 *__restrict__ dVg,   // plain-store targets of clipped tiles
                const int4 *__restrict__ plan, int nblk,                           // packed sequences: tile list; statistic blocks per head
-               int N, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+               int N, int Nq, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
   // BH counts (batch, KV head) pairs here.  With grouped queries (G > 1) one work item walks the query steps of all G
   // query heads of its KV head, so their contributions are summed in the FP32 accumulators (Section 3.1: key and value
   // contributions also sum over the query heads that share a KV head).
@@ -650,9 +660,16 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   // Ragged N: query steps round up.  A zero-filled query column past N contributes exactly nothing (its dO, Q and Z rows
   // are zero and its padded statistics are zero, so t = 0 and r multiplies zero rows); key rows past N are clipped on store.
   // In a packed layout the query columns past the end of the sequence are the next sequence's rows and are masked.
-  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, lin / BH, N); };
-  auto q_start_of = [&](const TileInfo &t) { return CAUSAL ? t.row0 : t.seq0; };          // first query row that sees this key tile
-  auto steps_of = [&](const TileInfo &t) { return (t.seq_end - q_start_of(t) + C::kStepRows - 1) / C::kStepRows; };
+  // N: key rows per head (own operand), Nq: query rows per head.  A key j is seen by the queries i >= j - (L_k - L_q).
+  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, lin / BH, N, Nq); };
+  // First query (inside its sequence, rounded down to a 64-row statistics block) that sees this key tile, and the steps
+  // from there to the end of the queries; at least one step, fully masked if no query sees the tile.
+  auto q_start_of = [&](const TileInfo &t) {
+    const int Lq = t.oseq_end - t.oseq0, off = (t.seq_end - t.seq0) - Lq;
+    const int first = CAUSAL ? (max(0, t.row0 - t.seq0 - off) & ~63) : 0;
+    return min(first, ((Lq - 1) >> 6) << 6);
+  };
+  auto steps_of = [&](const TileInfo &t) { return max(1, (t.oseq_end - t.oseq0 - q_start_of(t) + C::kStepRows - 1) / C::kStepRows); };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (Q, dO, Z, stats) step tiles
@@ -667,13 +684,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
           if (g >= S) mbar_wait(&bar_q_empty[st], ((g / S) - 1) & 1, ab, kDkvWaitQEmpty);
           mbar_expect_tx(&bar_q_full[st], stage_tx);
           uint8_t *dst = sStage + st * C::kDkvStageBytes;
-          const int qh = q_head0 + n / T, qrow = q_start + (n % T) * C::kStepRows;
+          const int qh = q_head0 + n / T, qrel = q_start + (n % T) * C::kStepRows, qrow = tl.oseq0 + qrel;
           for (int s = 0; s < C::kSlabs; ++s) {
             tma_load_3d(dst + s * C::kStepSlabBytes, &tmQ, &bar_q_full[st], s * 64, qrow, qh);
             tma_load_3d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow, qh);
             if (use_z) tma_load_3d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow, qh);
           }
-          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + (static_cast<size_t>(qh) * nblk + tl.blk0 + ((qrow - tl.seq0) >> 6)) * 128, 512, &bar_q_full[st]);
+          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + (static_cast<size_t>(qh) * nblk + tl.blk0 + (qrel >> 6)) * 128, 512, &bar_q_full[st]);
         }
       }
       if (cta_abort) {
@@ -807,10 +824,12 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
         const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
         const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes) + C::kSliceCols * slice;
         const int nh = n % Th;                                      // step within the current query head
-        const int q0 = q_start + nh * C::kStepRows + C::kSliceCols * slice;   // query row (inside the head) of the slice's column 0
+        const int Lq = tl.oseq_end - tl.oseq0, off = (tl.seq_end - tl.seq0) - Lq, krel0 = tl.row0 - tl.seq0;
+        const int qs = q_start + nh * C::kStepRows;                           // first query (inside its sequence) of the step
+        const int q0 = qs + C::kSliceCols * slice;                            // ... of the slice's column 0
         float pkeep[32];
-        if ((CAUSAL && nh < 2) || q_start + (nh + 1) * C::kStepRows > tl.seq_end)
-          dkv_phase1<true>(tS16, nl, scale_log2, CAUSAL ? tl.row0 + row - q0 : 0, tl.seq_end - 1 - q0, pkeep);
+        if ((CAUSAL && qs < krel0 + 128 - off) || qs + C::kStepRows > Lq)
+          dkv_phase1<true>(tS16, nl, scale_log2, CAUSAL ? krel0 + row - off - q0 : 0, Lq - 1 - q0, pkeep);
         else
           dkv_phase1<false>(tS16, nl, scale_log2, 0, 0, pkeep);
         tmem_wait_st();

@@ -91,7 +91,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
                     const float *__restrict__ stats,
                     __nv_bfloat16 *__restrict__ dKg, __nv_bfloat16 *__restrict__ dVg,
                     const int4 *__restrict__ plan, int nblk,
-                    int N, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+                    int N, int Nq, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
   // BH counts (batch, KV head) pairs.  With grouped queries one work item walks the query steps of all G query heads of
   // its KV head, so that their contributions are summed in the FP32 accumulators (Section 3.1).
   using C = BwdW128;
@@ -148,9 +148,16 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   TileSched sched(total_tiles);
   // A step may reach past the end of the sequence: those query columns are zero fill or the next packed sequence's rows,
   // and are masked.
-  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, lin / BH, N); };
-  auto q_start_of = [&](const TileInfo &t) { return CAUSAL ? t.row0 : t.seq0; };          // first query row that sees this key tile
-  auto steps_of = [&](const TileInfo &t) { return (t.seq_end - q_start_of(t) + C::kStepRows - 1) / C::kStepRows; };
+  // N: key rows per head (own operand), Nq: query rows per head.  A key j is seen by the queries i >= j - (L_k - L_q).
+  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, lin / BH, N, Nq); };
+  // First query (inside its sequence, rounded down to a 64-row statistics block) that sees this key tile, and the steps
+  // from there to the end of the queries; at least one step, fully masked if no query sees the tile.
+  auto q_start_of = [&](const TileInfo &t) {
+    const int Lq = t.oseq_end - t.oseq0, off = (t.seq_end - t.seq0) - Lq;
+    const int first = CAUSAL ? (max(0, t.row0 - t.seq0 - off) & ~63) : 0;
+    return min(first, ((Lq - 1) >> 6) << 6);
+  };
+  auto steps_of = [&](const TileInfo &t) { return max(1, (t.oseq_end - t.oseq0 - q_start_of(t) + C::kStepRows - 1) / C::kStepRows); };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (Q, dO, Z, stats) step tiles
@@ -165,12 +172,12 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
           if (g >= S) mbar_wait(&bar_q_empty[st], ((g / S) - 1) & 1, ab, kWkQEmpty);
           mbar_expect_tx(&bar_q_full[st], stage_tx);
           uint8_t *dst = sStage + st * C::kDkvStageBytes;
-          const int qh = q_head0 + n / T, qrow = q_start + (n % T) * C::kStepRows;
+          const int qh = q_head0 + n / T, qrel = q_start + (n % T) * C::kStepRows, qrow = tl.oseq0 + qrel;
           tma_load_3d(dst, &tmQ, &bar_q_full[st], 0, qrow, qh);
           tma_load_3d(dst + C::kTileBytes, &tmdO, &bar_q_full[st], 0, qrow, qh);
           if (use_z) tma_load_3d(dst + 2 * C::kTileBytes, &tmZ, &bar_q_full[st], 0, qrow, qh);
           // two 64-row statistic blocks (the second may lie past the sequence's last block: its columns are masked)
-          bulk_load_1d(dst + 3 * C::kTileBytes, stats + (static_cast<size_t>(qh) * nblk + tl.blk0 + ((qrow - tl.seq0) >> 6)) * 128, 1024,
+          bulk_load_1d(dst + 3 * C::kTileBytes, stats + (static_cast<size_t>(qh) * nblk + tl.blk0 + (qrel >> 6)) * 128, 1024,
                        &bar_q_full[st]);
         }
       }
@@ -292,12 +299,14 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         // memory, so their completion covers both.  Slice w of the 128 columns lies in statistic block w / 2.
         const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kTileBytes) + (wg >> 1) * 128 + (wg & 1) * 32;
         const int nh = n % Th;                                              // step within the current query head
-        const int q0 = q_start + nh * C::kStepRows + C::kSliceCols * wg;    // query row (inside the head) of the slice's column 0
-        const bool masked = (CAUSAL && nh == 0) || q_start + (nh + 1) * C::kStepRows > tl.seq_end;
+        const int Lq = tl.oseq_end - tl.oseq0, off = (tl.seq_end - tl.seq0) - Lq, krel0 = tl.row0 - tl.seq0;
+        const int qs = q_start + nh * C::kStepRows;                         // first query (inside its sequence) of the step
+        const int q0 = qs + C::kSliceCols * wg;                             // ... of the slice's column 0
+        const bool masked = (CAUSAL && qs < krel0 + 128 - off) || qs + C::kStepRows > Lq;
         float pkeep[32];
         mbar_wait(&bar_s_full[sb], (g >> 1) & 1, ab, kWkS);
         tc_fence_after();
-        if (masked) dkv_phase1<true>(tS, nl, scale_log2, CAUSAL ? tl.row0 + row - q0 : 0, tl.seq_end - 1 - q0, pkeep);
+        if (masked) dkv_phase1<true>(tS, nl, scale_log2, CAUSAL ? krel0 + row - off - q0 : 0, Lq - 1 - q0, pkeep);
         else        dkv_phase1<false>(tS, nl, scale_log2, 0, 0, pkeep);
         tmem_wait_st();
         tc_fence_before();

@@ -30,6 +30,9 @@
 
 namespace gproj {
 
+// Floor of the running row maximum (see the softmax loop): far below any score, far above -FLT_MAX.
+constexpr float kFwdMaxFloor = -1.0e30f;
+
 template <int D>
 struct FwdCfg {
   static constexpr int kBlockM = 128;                  // rows of one query tile (two per work item)
@@ -86,7 +89,7 @@ template <int D, bool CAUSAL, bool FMA_SOFTMAX, int MODE>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                __nv_bfloat16 *__restrict__ Og, const int4 *__restrict__ plan, float *__restrict__ LSE, int N, int BH, int Hq, int G, int tiles_per_item, int total_items, float scale_log2, float alpha,
+                __nv_bfloat16 *__restrict__ Og, const int4 *__restrict__ plan, float *__restrict__ LSE, int N, int Nk, int BH, int Hq, int G, int tiles_per_item, int total_items, float scale_log2, float alpha,
                 int *status) {
   using C = FwdCfg<D>;
   constexpr int S = C::kStages;
@@ -133,22 +136,31 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   // Work items ordered by decreasing work (causal: last pair first).  Item -> (sequence, first query tile, tiles) and head.
   // Dense calls: one sequence [0, N) per head, items are pairs (or single tiles); packed calls: single tiles from the plan.
-  struct Item { int seq0, len, qt0, nq, n_kt; };   // qt0: index of the first query tile inside its sequence; nq: query tiles; n_kt: key tiles walked
+  // qt0: index of the first query tile inside its sequence; nq: query tiles; n_kt: key tiles walked; kseq0, klen: the keys.
+  // Causal support of query i: keys j <= i + off with off = klen - len (the diagonal ends at the last query and last key).
+  struct Item { int seq0, len, qt0, nq, n_kt, kseq0, klen, off; };
   TileSched sched(total_items);
   auto decode = [&](int lin) {
     Item it;
     if (plan != nullptr) {
-      const TileInfo ti = tile_info(plan, lin / BH, 0, N);
+      const TileInfo ti = tile_info(plan, lin / BH, 0, N, Nk);
       it.seq0 = ti.seq0; it.len = ti.seq_end - ti.seq0; it.qt0 = (ti.row0 - ti.seq0) / C::kBlockM; it.nq = 1;
+      it.kseq0 = ti.oseq0; it.klen = ti.oseq_end - ti.oseq0;
     } else {
       const int pair = CAUSAL ? (n_pairs - 1 - lin / BH) : (lin / BH);
       it.seq0 = 0; it.len = N; it.qt0 = TPI * pair; it.nq = min(TPI, n_qt - it.qt0);
+      it.kseq0 = 0; it.klen = Nk;
     }
-    it.n_kt = CAUSAL ? it.qt0 + it.nq : (it.len + C::kBlockN - 1) / C::kBlockN;
+    it.off = it.klen - it.len;
+    // key tiles up to the last key the item's last row sees; at least one (fully masked if the item sees no key at all)
+    const int kend = CAUSAL ? min(it.klen, (it.qt0 + it.nq) * C::kBlockM + it.off) : it.klen;
+    it.n_kt = max(1, (max(kend, 0) + C::kBlockN - 1) / C::kBlockN);
     return it;
   };
-  // query tile t of the item takes part in key step j?
-  auto active = [&](const Item &it, int t, int j) { return t < it.nq && (!CAUSAL || j <= it.qt0 + t); };
+  // query tile t of the item takes part in key step j?  (key tile 0 always, so that every tile has a first step)
+  auto active = [&](const Item &it, int t, int j) {
+    return t < it.nq && (!CAUSAL || j <= max(0, ((it.qt0 + t) * C::kBlockM + C::kBlockM - 1 + it.off) >> 7));
+  };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of K_j, V_j
@@ -161,7 +173,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kFwdWaitKVEmpty);
           uint8_t *dK = sKV + st * 2 * C::kTileBytes, *dV = dK + C::kTileBytes;
-          const int kvh = kv_head_of(bh, Hq, G), krow = it.seq0 + j * C::kBlockN;   // grouped-query: the group's shared K / V head
+          const int kvh = kv_head_of(bh, Hq, G), krow = it.kseq0 + j * C::kBlockN;   // grouped-query: the group's shared K / V head
           mbar_expect_tx(&bar_k_full[st], C::kTileBytes);
           for (int s = 0; s < C::kSlabs; ++s) tma_load_3d(dK + s * C::kSlabBytes, &tmK, &bar_k_full[st], s * 64, krow, kvh);
           mbar_expect_tx(&bar_v_full[st], C::kTileBytes);
@@ -282,6 +294,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const Item it = decode(lin);
       const int bh = lin % BH, T = it.n_kt;
       const int qt = it.qt0 + (split ? 0 : t);        // this warpgroup's query tile inside the sequence
+      // Masking, reduced to two numbers per tile: column c of key tile j is outside the row's support when
+      // 128 j + c > rk, with rk the last key the row sees (causal diagonal and end of the keys, whichever comes first);
+      // no key tile before jm needs the test for any row of the tile.
+      const int rk = CAUSAL ? min(row + qt * C::kBlockM + it.off, it.klen - 1) : it.klen - 1;
+      const int jl = CAUSAL ? max(0, (qt * C::kBlockM + C::kBlockM - 1 + it.off) >> 7) : T;   // last key tile of this query tile
+      const int jm = CAUSAL ? min((qt * C::kBlockM + it.off + 1) >> 7, it.klen >> 7) : (it.klen >> 7);
       // Split mode: stay in step with the item (its Q has landed), so that a warpgroup without key tiles cannot run ahead.
       if (split) mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
       if (!split && t >= it.nq) {
@@ -298,7 +316,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int cnt_item0 = cnt;
       for (int j = split ? t : 0; j < T; j += split ? 2 : 1) {
         const bool first = split ? (j < 2) : (j == 0);     // this warpgroup's first key tile of the item
-        if (!split && !active(it, t, j)) {
+        if (!split && j > jl) {
           // no work in this step (causal: the first tile of the pair ends one key tile earlier): pass the turn on
           if (take_turns) {
             if (t == 1 || turn > 0) mbar_wait(&bar_turn[t], (t == 1 ? turn : turn - 1) & 1, ab, kFwdWaitTurn);
@@ -315,9 +333,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tmem_wait_ld();
         if (C::kSepP) { tc_fence_before(); mbar_arrive(&bar_s_free[t]); }   // the next S_t may be issued while this one is in the ALUs
         // Keys beyond the causal diagonal, and the zero-filled columns past the last key of a ragged tile, get -inf.
-        const bool diag = CAUSAL && j == qt, tail = (j + 1) * C::kBlockN > it.len;
-        if (diag || tail) {
-          const int lim = min(diag ? row : C::kBlockN - 1, tail ? it.len - j * C::kBlockN - 1 : C::kBlockN - 1);
+        if (j >= jm) {
+          const int lim = rk - j * C::kBlockN;
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
@@ -334,7 +351,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             mxp[i] = fmax3(mxp[i], __uint_as_float(xr[(e + i) >> 5][(e + i) & 31]), __uint_as_float(xr[(e + 8 + i) >> 5][(e + 8 + i) & 31]));
-        const float mx = fmaxf(fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])), fmaxf(fmaxf(mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7])));
+        // The floor keeps the maximum finite for a row that has seen no key yet (unequal lengths: rows before the causal
+        // diagonal reaches key 0), so that such a row gives z = exp2(-inf) = 0 instead of NaN from (-inf) - (-inf).
+        const float mx = fmax3(fmax3(mxp[0], mxp[1], mxp[2]), fmax3(mxp[3], mxp[4], mxp[5]), fmax3(mxp[6], mxp[7], kFwdMaxFloor));
         // Lazy maximum: the running maximum is only raised when the tile's maximum exceeds it by more than 2^kLazyLog2
         // in the exponent domain; otherwise the stale value stays (z <= 2^kLazyLog2, harmless in FP32 / BF16) and neither
         // l nor the accumulator needs a rescale.  The first tile always sets it (m_run = -inf).
@@ -385,7 +404,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       // Split mode: O = (O_0 s_0 + O_1 s_1) / (l_0 s_0 + l_1 s_1) with s_t = exp2((m_t - max(m_0, m_1)) alpha log2 e).
       const bool has1 = split && T >= 2;               // the second warpgroup had at least one key tile
-      float a0 = 1.0f / l_run, a1 = 0.f;
+      float a0 = (l_run > 0.f) ? 1.0f / l_run : 0.f, a1 = 0.f;   // a row with an empty support has l = 0: O = 0
       if (split) {
         mbar_wait(&bar_merge, ti & 1, ab, kFwdWaitMerge);
         tc_fence_after();
@@ -395,7 +414,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const float s0 = fast_exp2(__fmul_rn(__fsub_rn(m_run, m), scale_log2)), s1 = fast_exp2(__fmul_rn(__fsub_rn(m1, m), scale_log2));
           l_run = fmaf(l_run, s0, l1 * s1);
           m_run = m;
-          const float inv = 1.0f / l_run;
+          const float inv = (l_run > 0.f) ? 1.0f / l_run : 0.f;   // neither half has seen a key: O = 0
           a0 = s0 * inv;
           a1 = s1 * inv;
         }
@@ -428,7 +447,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_arrive(&bar_o_free[t]);                     // O_t may be overwritten by the next work item
       if (split) mbar_arrive(&bar_o_free[1]);          // warpgroup 0 has read both accumulators
       const int qrow0 = it.seq0 + qt * C::kBlockM;      // first row of the tile inside the head
-      if (qt * C::kBlockM + row < it.len) LSE[static_cast<size_t>(bh) * N + qrow0 + row] = fmaf(m_run, alpha, logf(l_run));
+      if (qt * C::kBlockM + row < it.len) LSE[static_cast<size_t>(bh) * N + qrow0 + row] = (l_run > 0.f) ? fmaf(m_run, alpha, logf(l_run)) : INFINITY;
       fence_proxy_async_smem();
       named_bar_sync(1 + t, 128);
       const TileInfo tinfo{qrow0, it.seq0, it.seq0 + it.len, 0};

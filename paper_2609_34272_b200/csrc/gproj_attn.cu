@@ -135,10 +135,10 @@ int check_shape(int B, int H, int N, int d) {
 
 size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
-int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N, int d,
+int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N, int Nk, int d,
                float softmax_scale, int causal, unsigned fwd_flags, const int4 *plan, int n_plan_tiles, void *stream);
 int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
-               void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+               void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int Nk, int d, float softmax_scale, int causal,
                void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
                int n_plan_tiles, int nblk, void *stream);
 
@@ -163,7 +163,7 @@ int gproj_attn_fwd_gqa(const void *Q, const void *K, const void *V, void *O, flo
 
 int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N,
                       int d, float softmax_scale, int causal, unsigned fwd_flags, void *stream) {
-  return launch_fwd(Q, K, V, O, LSE, B, H, Hkv, N, d, softmax_scale, causal, fwd_flags, nullptr, 0, stream);
+  return launch_fwd(Q, K, V, O, LSE, B, H, Hkv, N, N, d, softmax_scale, causal, fwd_flags, nullptr, 0, stream);
 }
 
 }  // extern "C"
@@ -172,13 +172,13 @@ namespace {
 
 // Dense call: plan == nullptr, one sequence [0, N) per head.  Packed call: B = 1, N = total tokens, plan = device tile
 // list (query order) with n_plan_tiles entries.
-int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N, int d,
+int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N, int Nk, int d,
                float softmax_scale, int causal, unsigned fwd_flags, const int4 *plan, int n_plan_tiles, void *stream) {
   if (!Q || !K || !V || !O || !LSE) return GPROJ_ERR_NULL;
   if (fwd_flags & ~GPROJ_FWD_FLAG_FMA_SOFTMAX) return GPROJ_ERR_FLAGS;
   const bool fma = (fwd_flags & GPROJ_FWD_FLAG_FMA_SOFTMAX) != 0;
   if (int rc = check_shape(B, H, N, d)) return rc;
-  if (Hkv <= 0 || H % Hkv != 0) return GPROJ_ERR_SHAPE;
+  if (Hkv <= 0 || H % Hkv != 0 || check_shape(B, Hkv, Nk, d) != GPROJ_OK) return GPROJ_ERR_SHAPE;
   const int G = H / Hkv;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || (reinterpret_cast<uintptr_t>(LSE) & 3u))
     return GPROJ_ERR_ALIGN;
@@ -189,7 +189,7 @@ int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE,
   const int BH = B * H;
   const int BHkv = B * Hkv;
   CUtensorMap mQ, mK, mV, mO;
-  if (!make_map(&mQ, Q, BH, N, d, 128) || !make_map(&mK, K, BHkv, N, d, 128) || !make_map(&mV, V, BHkv, N, d, 128) ||
+  if (!make_map(&mQ, Q, BH, N, d, 128) || !make_map(&mK, K, BHkv, Nk, d, 128) || !make_map(&mV, V, BHkv, Nk, d, 128) ||
       !make_map(&mO, O, BH, N, d, 128))
     return GPROJ_ERR_CUDA;
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
@@ -203,7 +203,7 @@ int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE,
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define GPROJ_LAUNCH_FWD(DD, CC, FF, MM)                                                                            \
   attn_fwd_kernel<DD, CC, FF, MM><<<grid, FwdCfg<DD>::kThreads, FwdCfg<DD>::kSmemBytes, s>>>(                         \
-      mQ, mK, mV, mO, static_cast<__nv_bfloat16 *>(O), plan, LSE, N, BH, H, G, tiles_per_item, total_items, scale_log2,      \
+      mQ, mK, mV, mO, static_cast<__nv_bfloat16 *>(O), plan, LSE, N, Nk, BH, H, G, tiles_per_item, total_items, scale_log2,      \
       softmax_scale, st->status_ptr)
 #define GPROJ_LAUNCH_FWD_C(DD, FF, MM)                                                                              \
   do { if (causal) GPROJ_LAUNCH_FWD(DD, true, FF, MM); else GPROJ_LAUNCH_FWD(DD, false, FF, MM); } while (0)
@@ -243,7 +243,7 @@ int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, c
 int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
                        void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
                        void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
-  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, Hkv, N, d, softmax_scale, causal, workspace, workspace_bytes, flags,
+  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, Hkv, N, N, d, softmax_scale, causal, workspace, workspace_bytes, flags,
                     nullptr, nullptr, 0, (N + 63) / 64, stream);
 }
 
@@ -254,12 +254,12 @@ namespace {
 // Dense call: plans == nullptr.  Packed call: B = 1, N = total tokens, plan_q / plan_kv = device tile lists in the order
 // of the dQ-side and the dK/dV-side kernel, nblk = 64-row statistic blocks per head.
 int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
-               void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
+               void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int Nk, int d, float softmax_scale, int causal,
                void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
                int n_plan_tiles, int nblk, void *stream) {
   if (!Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return GPROJ_ERR_NULL;
   if (int rc = check_shape(B, H, N, d)) return rc;
-  if (Hkv <= 0 || H % Hkv != 0) return GPROJ_ERR_SHAPE;
+  if (Hkv <= 0 || H % Hkv != 0 || check_shape(B, Hkv, Nk, d) != GPROJ_OK) return GPROJ_ERR_SHAPE;
   const int G = H / Hkv;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
       !aligned16(dK) || !aligned16(dV) || (reinterpret_cast<uintptr_t>(LSE) & 3u))
@@ -281,15 +281,16 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
   __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + stats_sz);
 
   CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64, mdQst, mZst, mdKst, mdVst;
-  bool ok = make_map(&mQ128, Q, BH, N, d, 128) && make_map(&mdO128, dO, BH, N, d, 128) && make_map(&mK64, K, BHkv, N, d, 64) &&
-            make_map(&mV64, V, BHkv, N, d, 64) && make_map(&mK128, K, BHkv, N, d, 128) && make_map(&mV128, V, BHkv, N, d, 128) &&
+  bool ok = make_map(&mQ128, Q, BH, N, d, 128) && make_map(&mdO128, dO, BH, N, d, 128) && make_map(&mK64, K, BHkv, Nk, d, 64) &&
+            make_map(&mV64, V, BHkv, Nk, d, 64) && make_map(&mK128, K, BHkv, Nk, d, 128) && make_map(&mV128, V, BHkv, Nk, d, 128) &&
             make_map(&mQ64, Q, BH, N, d, 64) && make_map(&mdO64, dO, BH, N, d, 64) && make_map(&mZ64, Zneg, BH, N, d, 64) &&
-            make_map(&mdQst, dQ, BH, N, d, 128) && make_map(&mZst, Zneg, BH, N, d, 128) && make_map(&mdKst, dK, BHkv, N, d, 128) &&
-            make_map(&mdVst, dV, BHkv, N, d, 128);
+            make_map(&mdQst, dQ, BH, N, d, 128) && make_map(&mZst, Zneg, BH, N, d, 128) && make_map(&mdKst, dK, BHkv, Nk, d, 128) &&
+            make_map(&mdVst, dV, BHkv, Nk, d, 128);
   if (!ok) return GPROJ_ERR_CUDA;
 
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
-  const int n_qt = plan_q ? n_plan_tiles : (N + 127) / 128, total_tiles = BH * n_qt, total_kv_tiles = BHkv * n_qt;
+  const int n_qt = plan_q ? n_plan_tiles : (N + 127) / 128, n_kt = plan_q ? n_plan_tiles : (Nk + 127) / 128;
+  const int total_tiles = BH * n_qt, total_kv_tiles = BHkv * n_kt;
   if (total_tiles <= 0) return GPROJ_OK;   // nothing but empty sequences
   const dim3 grid(static_cast<unsigned>(total_tiles < st->sm_count ? total_tiles : st->sm_count));   // persistent: one CTA per SM
   const dim3 grid_kv(static_cast<unsigned>(total_kv_tiles < st->sm_count ? total_kv_tiles : st->sm_count));
@@ -300,13 +301,13 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
     if (run_dq)                                                                                                         \
       bwd_dq_kernel<DD, CC><<<grid, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDqSmemBytes, s>>>(                               \
           mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, static_cast<__nv_bfloat16 *>(dQ), Zneg, plan_q, nblk,   \
-          N, BH, H, G, total_tiles, scale_log2, softmax_scale,                                                        \
+          N, Nk, BH, H, G, total_tiles, scale_log2, softmax_scale,                                                    \
           flags,                                                                                                        \
           st->status_ptr);                                                                                              \
     if (run_dkv)                                                                                                        \
       bwd_dkv_kernel<DD, CC><<<grid_kv, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
           mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, static_cast<__nv_bfloat16 *>(dK),                        \
-          static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,     \
+          static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, Nk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale, \
           flags,                                                                                                        \
           st->status_ptr);                                                                                              \
   } while (0)
@@ -317,11 +318,11 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
     if (run_dq)                                                                                                         \
       bwd_dq_kernel<64, CC><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kDqSmemBytes, s>>>(                                \
           mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, static_cast<__nv_bfloat16 *>(dQ), Zneg, plan_q,    \
-          nblk, N, BH, H, G, total_tiles, scale_log2, softmax_scale, flags, st->status_ptr);                              \
+          nblk, N, Nk, BH, H, G, total_tiles, scale_log2, softmax_scale, flags, st->status_ptr);                          \
     if (run_dkv)                                                                                                        \
       bwd_dkv_w128_kernel<CC><<<grid_kv, BwdW128::kThreads, BwdW128::kDkvSmemBytes, s>>>(                                \
           mK128, mV128, mQ128, mdO128, mZst, mdKst, mdVst, stats, static_cast<__nv_bfloat16 *>(dK),                       \
-          static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,    \
+          static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, Nk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,\
           flags, st->status_ptr);                                                                                       \
   } while (0)
   if (d == 64) { if (causal) GPROJ_LAUNCH_BWD_W128(true); else GPROJ_LAUNCH_BWD_W128(false); }
@@ -336,6 +337,19 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
 }  // namespace
 
 extern "C" {
+
+// ---- unequal query and key lengths ------------------------------------------------------------------
+int gproj_attn_fwd_rect(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int Nq,
+                        int Nk, int d, float softmax_scale, int causal, unsigned fwd_flags, void *stream) {
+  return launch_fwd(Q, K, V, O, LSE, B, H, Hkv, Nq, Nk, d, softmax_scale, causal, fwd_flags, nullptr, 0, stream);
+}
+
+int gproj_attn_bwd_rect(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                        void *dQ, void *dK, void *dV, int B, int H, int Hkv, int Nq, int Nk, int d, float softmax_scale,
+                        int causal, void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
+  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, Hkv, Nq, Nk, d, softmax_scale, causal, workspace, workspace_bytes,
+                    flags, nullptr, nullptr, 0, (Nq + 63) / 64, stream);
+}
 
 // ---- packed (variable-length) sequences ------------------------------------------------------------
 }  // extern "C"
@@ -408,7 +422,7 @@ int gproj_attn_fwd_varlen(const void *Q, const void *K, const void *V, void *O, 
   if (!packed_shape(cu_seqlens, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
   if (!plan_device) return GPROJ_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
-  return launch_fwd(Q, K, V, O, LSE, 1, H, Hkv, ps.total, d, softmax_scale, causal, fwd_flags,
+  return launch_fwd(Q, K, V, O, LSE, 1, H, Hkv, ps.total, ps.total, d, softmax_scale, causal, fwd_flags,
                     static_cast<const int4 *>(plan_device), ps.n_tiles, stream);
 }
 
@@ -427,7 +441,7 @@ int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const voi
   if (!plan_device) return GPROJ_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
   const int4 *plan = static_cast<const int4 *>(plan_device);
-  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, 1, H, Hkv, ps.total, d, softmax_scale, causal, workspace, workspace_bytes,
+  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, 1, H, Hkv, ps.total, ps.total, d, softmax_scale, causal, workspace, workspace_bytes,
                     flags, plan, plan + ps.n_tiles, ps.n_tiles, ps.nblk, stream);
 }
 

@@ -270,7 +270,7 @@ def main():
                      "algorithmic_flops_per_launch": fl["dkv_kernel"]},
         "e2e": {"value": world * fl["bwd7"] / (e2e_ms / 1e3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 4 * tensor_bytes, "d2h_bytes_per_step": 3 * tensor_bytes,
-                "what": "gproj_attn_fwd_bwd_host: pinned host Q,K,V,dO -> device, forward, backward, dQ,dK,dV -> pinned host; same FLOP count"},
+                "what": "gproj_attn_fwd_bwd_host: pinned host Q,K,V,dO -> device, forward, backward, dQ,dK,dV -> pinned host (slabs of heads pipelined on internal copy streams); same FLOP count"},
         "gpu_launches": 3 * steps,
         "clocks": clocks,
     }

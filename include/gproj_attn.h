@@ -9,9 +9,11 @@
  *     s_ij = softmax_scale * q_i . k_j over the row's support.
  *   - Supported shapes: d in {64, 128}; any N >= 1 (tiles of 128 rows; a ragged last tile is zero-filled on load,
  *     masked where it would enter a row statistic and clipped on store); B, H >= 1 with B*H*N < 2^31; N_q = N_k = N;
- *     causal != 0 means row i attends to j <= i.  The *_gqa entry points take separate query / KV head counts.
- *   - The caller owns all memory.  The library never allocates, frees or synchronises; work is
- *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).
+ *     causal != 0 means row i attends to j <= i.  The *_gqa entry points take separate query / KV head counts, the
+ *     *_rect entry points separate query / key lengths.
+ *   - The caller owns all memory.  The library never allocates device memory, frees or synchronises; work is
+ *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).  (The host-buffer entry point
+ *     also uses two streams of its own, see there.)
  *     After the first call on a device (one-time attribute set-up), gproj_attn_fwd and gproj_attn_bwd with a
  *     caller-supplied workspace have been captured into a CUDA graph and replayed (that is what is tested).
  *   - Return value: GPROJ_OK (0) or a negative gproj_status.  Nothing throws, aborts or traps.
@@ -168,13 +170,17 @@ int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const voi
  * Forward and backward in one call from HOST buffers (a convenience around the entry points above; the paper's
  * Algorithm 1 starts from tensors already on the device).  Q, K, V, dO are copied to the device, the forward
  * (Eq. "gproj-forward") and the backward (Algorithm 1) run, and dQ, dK, dV (and O, LSE when those pointers are not NULL)
- * are copied back, all enqueued in order on `stream`.
+ * are copied back.  Large problems are cut into up to 16 slabs of whole KV heads (about 2 MiB of Q each) that are pipelined:
+ * the kernels run on `stream`, the copies in and out on two internal streams, ordered by events so that nothing of the call
+ * starts before the work already queued on `stream` and `stream` reaches the end of the call only after the last copy-out.
  *   - Q, K, V, dO, O, LSE, dQ, dK, dV are HOST pointers with the layouts of gproj_attn_fwd_gqa / gproj_attn_bwd_gqa.  Page-locked
  *     memory makes the call asynchronous; pageable memory works but serialises in the CUDA runtime.  The buffers must stay
  *     valid until the stream has reached the end of the call's work.
  *   - `staging` is DEVICE memory owned by the caller, 256-byte aligned, at least gproj_attn_host_staging_bytes() bytes (copies
- *     of the eight tensors, LSE and the backward workspace); GPROJ_ERR_WORKSPACE otherwise.  Nothing is allocated.
- *   - flags: those of gproj_attn_bwd without the ONLY_* bits.
+ *     of the eight tensors, LSE and the backward workspace); GPROJ_ERR_WORKSPACE otherwise.  No device memory is allocated;
+ *     the first pipelined call on a device creates the two streams and 34 events, which live until the process exits.
+ *   - flags: those of gproj_attn_bwd without the ONLY_* bits (GPROJ_ERR_FLAGS for those).
+ *   - Calls from several host threads on one device are serialised while they enqueue.
  */
 size_t gproj_attn_host_staging_bytes(int B, int H, int Hkv, int N, int d);
 int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const void *dO, void *O, float *LSE,

@@ -37,14 +37,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+#ifndef GPROJ_HOST_SLAB_LOG2
+#define GPROJ_HOST_SLAB_LOG2 21
+#endif
+constexpr int kHostSlabLog2 = GPROJ_HOST_SLAB_LOG2;   // log2 of the Q bytes per slab of the host-buffer entry point
+constexpr int kMaxSlabs = 16;   // the host-buffer entry point pipelines at most this many slabs of heads
+
 struct DeviceState {
   bool ready = false;
   bool arch_ok = false;
   int *status_ptr = nullptr;
   int sm_count = 0;
+  // host-buffer entry point only: copy-in and copy-out streams and the events that order them against the caller's stream
+  bool pipe_ready = false;
+  cudaStream_t in_stream = nullptr, out_stream = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_end = nullptr, ev_in[kMaxSlabs] = {}, ev_done[kMaxSlabs] = {};
 };
 
 std::mutex g_mutex;
+std::mutex g_pipe_mutex;   // serialises the host-buffer entry point's use of the per-device streams and events
 DeviceState g_dev[kMaxDevices];
 EncodeTiledFn g_encode = nullptr;
 thread_local int tl_launch_count = 0;
@@ -459,32 +470,89 @@ int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const v
   const size_t need = gproj_attn_host_staging_bytes(B, H, Hkv, N, d);
   if (need == 0) return GPROJ_ERR_SHAPE;
   if (!staging || (reinterpret_cast<uintptr_t>(staging) & 255u) || staging_bytes < need) return GPROJ_ERR_WORKSPACE;
+  if (flags & (GPROJ_FLAG_ONLY_DQ_PASS | GPROJ_FLAG_ONLY_DKV_PASS)) return GPROJ_ERR_FLAGS;
   const size_t qb = static_cast<size_t>(B) * H * N * d * 2, kvb = static_cast<size_t>(B) * Hkv * N * d * 2;
   const size_t lb = static_cast<size_t>(B) * H * N * sizeof(float);
   uint8_t *p = static_cast<uint8_t *>(staging);
   auto take = [&](size_t bytes) { uint8_t *r = p; p += align256(bytes); return r; };
   uint8_t *dQin = take(qb), *dOin = take(qb), *dOout = take(qb), *dQout = take(qb);
   uint8_t *dKin = take(kvb), *dVin = take(kvb), *dKout = take(kvb), *dVout = take(kvb);
-  float *dLSE = reinterpret_cast<float *>(take(lb));
+  uint8_t *dLSE = take(lb);
   uint8_t *ws = p;
   const size_t ws_bytes = gproj_attn_bwd_workspace_bytes(B, H, N, d);
+  DeviceState *st = nullptr;
+  if (int rc = device_state(&st)) return rc;
+
+  // The (batch, KV head) axis is cut into slabs of whole KV heads with their query heads (contiguous in every tensor), and
+  // the slabs are pipelined: copy-in of slab c + 1 and copy-out of slab c - 1 run on two internal streams while the
+  // caller's stream computes slab c.  About 2 MiB of Q and at least 128 key tiles per slab: smaller slabs leave the
+  // persistent kernels too few tiles (measured: slower than no pipeline at all), larger ones leave the copies exposed.
+  const int kv_heads = B * Hkv, G = H / Hkv;
+  int slabs = static_cast<int>((qb + (size_t(1) << (kHostSlabLog2 - 1))) >> kHostSlabLog2);
+  const long long kv_tiles = static_cast<long long>(kv_heads) * ((N + 127) / 128);
+  slabs = std::min(slabs, static_cast<int>(std::min<long long>(kv_tiles / 128, kMaxSlabs)));   // >= 128 key tiles per slab
+  slabs = std::max(1, std::min(slabs, kv_heads));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  bool ok = cudaMemcpyAsync(dQin, Q, qb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-            cudaMemcpyAsync(dKin, K, kvb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-            cudaMemcpyAsync(dVin, V, kvb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-            cudaMemcpyAsync(dOin, dO, qb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);   // the internal streams and events are shared by all callers of the device
+  if (slabs > 1 && !st->pipe_ready) {
+    bool ok = cudaStreamCreateWithFlags(&st->in_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&st->out_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st->ev_end, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kMaxSlabs; ++i)
+      ok = cudaEventCreateWithFlags(&st->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&st->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+    st->pipe_ready = true;
+  }
+  cudaStream_t s_in = slabs > 1 ? st->in_stream : s, s_out = slabs > 1 ? st->out_stream : s;
+  bool ok = true;
+  if (slabs > 1) {
+    // nothing of this call may start before the work already queued on the caller's stream (it may still use `staging`)
+    ok = cudaEventRecord(st->ev_start, s) == cudaSuccess && cudaStreamWaitEvent(s_in, st->ev_start, 0) == cudaSuccess &&
+         cudaStreamWaitEvent(s_out, st->ev_start, 0) == cudaSuccess;
+  }
+  const size_t row_bytes = static_cast<size_t>(N) * d * 2;           // one head of one tensor
+  auto slab_begin = [&](int c) { return static_cast<int>(static_cast<long long>(kv_heads) * c / slabs); };
+  for (int c = 0; ok && c < slabs; ++c) {
+    const size_t k0 = slab_begin(c), kn = slab_begin(c + 1) - k0, q0 = k0 * G, qn = kn * G;
+    ok = cudaMemcpyAsync(dQin + q0 * row_bytes, static_cast<const uint8_t *>(Q) + q0 * row_bytes, qn * row_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
+         cudaMemcpyAsync(dKin + k0 * row_bytes, static_cast<const uint8_t *>(K) + k0 * row_bytes, kn * row_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
+         cudaMemcpyAsync(dVin + k0 * row_bytes, static_cast<const uint8_t *>(V) + k0 * row_bytes, kn * row_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
+         cudaMemcpyAsync(dOin + q0 * row_bytes, static_cast<const uint8_t *>(dO) + q0 * row_bytes, qn * row_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    if (ok && slabs > 1) ok = cudaEventRecord(st->ev_in[c], s_in) == cudaSuccess;
+  }
   if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
-  if (int rc = gproj_attn_fwd_gqa(dQin, dKin, dVin, dOout, dLSE, B, H, Hkv, N, d, softmax_scale, causal, stream)) return rc;
-  if (int rc = gproj_attn_bwd_gqa(dQin, dKin, dVin, dOout, dLSE, dOin, dQout, dKout, dVout, B, H, Hkv, N, d, softmax_scale,
-                                  causal, ws, ws_bytes, flags, stream))
-    return rc;
-  ok = cudaMemcpyAsync(dQ, dQout, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaMemcpyAsync(dK, dKout, kvb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaMemcpyAsync(dV, dVout, kvb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-  if (ok && O) ok = cudaMemcpyAsync(O, dOout, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-  if (ok && LSE) ok = cudaMemcpyAsync(LSE, dLSE, lb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-  if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
-  tl_launch_count = 3;
+  int launches = 0;
+  for (int c = 0; c < slabs; ++c) {
+    const size_t k0 = slab_begin(c), kn = slab_begin(c + 1) - k0, q0 = k0 * G, qn = kn * G;
+    if (slabs > 1 && cudaStreamWaitEvent(s, st->ev_in[c], 0) != cudaSuccess) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+    float *lse_c = reinterpret_cast<float *>(dLSE + q0 * N * sizeof(float));
+    // a slab is a problem with batch 1, kn KV heads and qn query heads; the slabs share the backward workspace in turn
+    if (int rc = gproj_attn_fwd_gqa(dQin + q0 * row_bytes, dKin + k0 * row_bytes, dVin + k0 * row_bytes, dOout + q0 * row_bytes, lse_c, 1,
+                                    static_cast<int>(qn), static_cast<int>(kn), N, d, softmax_scale, causal, stream))
+      return rc;
+    launches += tl_launch_count;
+    if (int rc = gproj_attn_bwd_gqa(dQin + q0 * row_bytes, dKin + k0 * row_bytes, dVin + k0 * row_bytes, dOout + q0 * row_bytes, lse_c,
+                                    dOin + q0 * row_bytes, dQout + q0 * row_bytes, dKout + k0 * row_bytes, dVout + k0 * row_bytes, 1,
+                                    static_cast<int>(qn), static_cast<int>(kn), N, d, softmax_scale, causal, ws, ws_bytes, flags, stream))
+      return rc;
+    launches += tl_launch_count;
+    ok = slabs == 1 || (cudaEventRecord(st->ev_done[c], s) == cudaSuccess && cudaStreamWaitEvent(s_out, st->ev_done[c], 0) == cudaSuccess);
+    ok = ok && cudaMemcpyAsync(static_cast<uint8_t *>(dQ) + q0 * row_bytes, dQout + q0 * row_bytes, qn * row_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess &&
+         cudaMemcpyAsync(static_cast<uint8_t *>(dK) + k0 * row_bytes, dKout + k0 * row_bytes, kn * row_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess &&
+         cudaMemcpyAsync(static_cast<uint8_t *>(dV) + k0 * row_bytes, dVout + k0 * row_bytes, kn * row_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+    if (ok && O) ok = cudaMemcpyAsync(static_cast<uint8_t *>(O) + q0 * row_bytes, dOout + q0 * row_bytes, qn * row_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+    if (ok && LSE) ok = cudaMemcpyAsync(LSE + q0 * N, lse_c, qn * N * sizeof(float), cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+  }
+  // the caller's stream reaches the end of the call only when the last copy-out has landed
+  if (slabs > 1 && !(cudaEventRecord(st->ev_end, s_out) == cudaSuccess && cudaStreamWaitEvent(s, st->ev_end, 0) == cudaSuccess)) {
+    (void)cudaGetLastError();
+    return GPROJ_ERR_CUDA;
+  }
+  tl_launch_count = launches;
   return GPROJ_OK;
 }
 

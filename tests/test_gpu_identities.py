@@ -233,6 +233,39 @@ def test_host_buffer_entry_point_matches_device_calls():
     assert e.value.status == -4
 
 
+@pytest.mark.parametrize("shape", [(2, 8, 8, 2048, 64), (1, 10, 5, 8192, 64), (3, 2, 1, 16384, 128)])
+def test_host_buffer_entry_point_pipelined_slabs(shape):
+    # Problems above a few MiB are cut into slabs of KV heads whose copies overlap the kernels on internal streams
+    # (2 even slabs; 2 slabs over 5 KV heads; 3 slabs of one KV head with two query heads each).  A slab may run the forward in
+    # another tile mode than the whole problem, so the comparison with the device-pointer calls is to rounding, not bits;
+    # a slab offset or ordering mistake is a gross error.  Two calls back to back on one stream reuse the staging buffer.
+    B, H, Hkv, N, d = shape
+    staging = torch.empty(g.gproj_attn_host_staging_bytes(B, H, Hkv, N, d), dtype=torch.uint8, device="cuda")
+    pending = []
+    for rep in range(2):
+        w = Workload("host_slabs", B, H, N, d, True, k_offset=4.0, seed=57 + rep, Hkv=Hkv)
+        inp = make_inputs(w)
+        host = {k: v.pin_memory() for k, v in inp.items()}
+        out = {"O": torch.empty_like(host["Q"]).pin_memory(), "LSE": torch.empty(B, H, N, dtype=torch.float32).pin_memory(),
+               "dQ": torch.empty_like(host["Q"]).pin_memory(), "dK": torch.empty_like(host["K"]).pin_memory(),
+               "dV": torch.empty_like(host["K"]).pin_memory()}
+        for t in out.values():
+            t.fill_(float("nan"))
+        g.gproj_attn_fwd_bwd_host(host["Q"], host["K"], host["V"], host["dO"], out["dQ"], out["dK"], out["dV"], w.softmax_scale, True,
+                                  staging, O=out["O"], LSE=out["LSE"])
+        assert g.gproj_last_launch_count() >= 6          # at least two slabs of three kernels
+        pending.append((w, inp, host, out))
+    rc, detail = g.gproj_last_device_status()          # synchronises the stream, which waits for the last copy-out
+    assert rc == 0, hex(detail)
+    for w, inp, host, out in pending:
+        O, LSE, dQ, dK, dV = fwd_bwd(inp["Q"], inp["K"], inp["V"], inp["dO"], w.softmax_scale, True)
+        assert torch.allclose(out["LSE"], LSE.cpu(), rtol=1e-5, atol=1e-5)
+        for name, ref in (("O", O), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+            got, ref = out[name].double(), ref.cpu().double()
+            assert torch.isfinite(got).all(), name
+            assert float((got - ref).norm() / ref.norm()) <= 2e-3, name
+
+
 def test_cuda_graph_capture_and_replay():
     # The entry points only enqueue work on the given stream (no allocation, no synchronisation once the per-device
     # set-up of the first call is done), so forward + backward can be captured into a CUDA graph and replayed.

@@ -306,6 +306,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_smem, 0);   // the shuffle marks it warp-uniform
 
+  // The dK/dV-side kernel that follows in the stream may be scheduled on SMs this kernel has left: its set-up and its
+  // stationary-tile loads need nothing from here, and it waits (griddep_wait) before it reads the statistics and Z.
+  griddep_launch_dependents();
+
   TileSched sched(total_tiles);
   // tile decode: causal -> longest rows first
   auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH), N, Nk); };
@@ -674,6 +678,9 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (Q, dO, Z, stats) step tiles
     if (lane == 0) {
+      // Z and the row statistics come from the dQ-side kernel, which may still be running (programmatic dependent
+      // launch); everything this CTA did so far, and the stationary-tile loads of the other loader warp, did not need it.
+      griddep_wait();
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
         const TileInfo tl = tile_of(lin);

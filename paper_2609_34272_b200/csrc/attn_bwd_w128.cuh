@@ -162,6 +162,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of the streamed (Q, dO, Z, stats) step tiles
     if (lane == 0) {
+      // Z and the row statistics come from the dQ-side kernel, which may still be running (programmatic dependent
+      // launch); everything this CTA did so far, and the stationary-tile loads of the other loader warp, did not need it.
+      griddep_wait();
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
         const TileInfo tl = tile_of(lin);

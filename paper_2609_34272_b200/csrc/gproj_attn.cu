@@ -146,6 +146,24 @@ int check_shape(int B, int H, int N, int d) {
 
 size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
+// Launch `kernel`; with overlap_previous it may be scheduled while the kernel before it in the stream still runs
+// (programmatic dependent launch: the kernel itself waits, by griddep_wait, before it reads what that kernel writes).
+template <typename... Params, typename... Args>
+void launch_after(void (*kernel)(Params...), dim3 grid, int threads, size_t smem, cudaStream_t s, bool overlap_previous,
+                  Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(static_cast<unsigned>(threads));
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap_previous ? 1 : 0;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);   // the caller reads cudaGetLastError()
+}
+
 int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE, int B, int H, int Hkv, int N, int Nk, int d,
                float softmax_scale, int causal, unsigned fwd_flags, const int4 *plan, int n_plan_tiles, void *stream);
 int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
@@ -316,7 +334,7 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
           flags,                                                                                                        \
           st->status_ptr);                                                                                              \
     if (run_dkv)                                                                                                        \
-      bwd_dkv_kernel<DD, CC><<<grid_kv, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s>>>(                             \
+      launch_after(bwd_dkv_kernel<DD, CC>, grid_kv, BwdCfg<DD>::kThreads, BwdCfg<DD>::kDkvSmemBytes, s, run_dq,            \
           mK128, mV128, mQ64, mdO64, mZ64, mdKst, mdVst, stats, static_cast<__nv_bfloat16 *>(dK),                        \
           static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, Nk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale, \
           flags,                                                                                                        \
@@ -331,7 +349,7 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
           mQ128, mdO128, mK64, mV64, mdQst, mZst, Ob, dOb, LSE, stats, static_cast<__nv_bfloat16 *>(dQ), Zneg, plan_q,    \
           nblk, N, Nk, BH, H, G, total_tiles, scale_log2, softmax_scale, flags, st->status_ptr);                          \
     if (run_dkv)                                                                                                        \
-      bwd_dkv_w128_kernel<CC><<<grid_kv, BwdW128::kThreads, BwdW128::kDkvSmemBytes, s>>>(                                \
+      launch_after(bwd_dkv_w128_kernel<CC>, grid_kv, BwdW128::kThreads, BwdW128::kDkvSmemBytes, s, run_dq,               \
           mK128, mV128, mQ128, mdO128, mZst, mdKst, mdVst, stats, static_cast<__nv_bfloat16 *>(dK),                       \
           static_cast<__nv_bfloat16 *>(dV), plan_kv, nblk, Nk, N, BHkv, Hkv, G, total_kv_tiles, scale_log2, softmax_scale,\
           flags, st->status_ptr);                                                                                       \

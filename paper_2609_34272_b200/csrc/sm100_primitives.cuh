@@ -343,6 +343,13 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   return d;
 }
 // three-input maximum (one instruction on sm_100)
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start while the
+// kernel before it in the stream still runs.  launch_dependents (in the earlier kernel) allows that start once every CTA of
+// the earlier kernel has issued it or exited; wait (in the later kernel) returns when the earlier kernel has completed and
+// its memory is visible.  Both are no-ops for a kernel launched without the attribute / with nothing before it.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));

@@ -167,6 +167,29 @@ int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const voi
                           unsigned flags, void *stream);
 
 /*
+ * Packed sequences whose query and key lengths differ (Appendix "Synthetic Numerical Suite": packed segments, unequal
+ * lengths, empty causal rows).  Queries, O, dO, dQ are [H][Tq][d] with Tq = cu_seqlens_q[num_seqs], LSE [H][Tq]; keys,
+ * values, dK, dV are [Hkv][Tk][d] with Tk = cu_seqlens_k[num_seqs]; sequence s owns query rows cu_seqlens_q[s] ..
+ * cu_seqlens_q[s+1]-1 and key rows cu_seqlens_k[s] .. cu_seqlens_k[s+1]-1.  Inside a sequence the rules are those of the
+ * *_rect entry points: causal means query i sees the keys j <= i + (Lk - Lq), a query without visible key gets O = 0,
+ * dQ = 0 and LSE = +infinity.  A sequence may have no queries (its dK, dV rows are written as zero), no keys (all its
+ * queries are such empty rows), or neither (skipped); Tq and Tk must both be positive.  Plan, workspace
+ * (gproj_attn_bwd_varlen_workspace_bytes() of cu_seqlens_q), flags and errors are as for the packed entry points above,
+ * which are the case cu_seqlens_k == cu_seqlens_q; a plan built by one pair of plan functions works only with the
+ * forward / backward of the same pair and the same offsets.
+ */
+size_t gproj_attn_varlen_qk_plan_bytes(const int *cu_seqlens_q, const int *cu_seqlens_k, int num_seqs);
+int gproj_attn_varlen_qk_plan(const int *cu_seqlens_q, const int *cu_seqlens_k, int num_seqs, int causal, void *plan_host,
+                              size_t plan_bytes);
+int gproj_attn_fwd_varlen_qk(const void *Q, const void *K, const void *V, void *O, float *LSE, const int *cu_seqlens_q,
+                             const int *cu_seqlens_k, int num_seqs, const void *plan_device, int H, int Hkv, int d,
+                             float softmax_scale, int causal, unsigned fwd_flags, void *stream);
+int gproj_attn_bwd_varlen_qk(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                             void *dQ, void *dK, void *dV, const int *cu_seqlens_q, const int *cu_seqlens_k, int num_seqs,
+                             const void *plan_device, int H, int Hkv, int d, float softmax_scale, int causal, void *workspace,
+                             size_t workspace_bytes, unsigned flags, void *stream);
+
+/*
  * Forward and backward in one call from HOST buffers (a convenience around the entry points above; the paper's
  * Algorithm 1 starts from tensors already on the device).  Q, K, V, dO are copied to the device, the forward
  * (Eq. "gproj-forward") and the backward (Algorithm 1) run, and dQ, dK, dV (and O, LSE when those pointers are not NULL)

@@ -15,12 +15,14 @@ from .binding import (  # noqa: F401
     gproj_attn_bwd_rect,
     gproj_attn_bwd_static_scratch,
     gproj_attn_bwd_varlen,
+    gproj_attn_bwd_varlen_qk,
     gproj_attn_bwd_workspace_bytes,
     gproj_attn_fwd,
     gproj_attn_fwd_bwd_host,
     gproj_attn_fwd_rect,
     gproj_attn_host_staging_bytes,
     gproj_attn_fwd_varlen,
+    gproj_attn_fwd_varlen_qk,
     gproj_last_device_status,
     gproj_last_launch_count,
     gproj_selftest_wait_timeout,

@@ -25,6 +25,7 @@ EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd",
            "gproj_attn_bwd_static_scratch", "gproj_attn_fwd_rect", "gproj_attn_bwd_rect",
            "gproj_attn_varlen_plan_bytes", "gproj_attn_varlen_plan", "gproj_attn_fwd_varlen",
            "gproj_attn_bwd_varlen_workspace_bytes", "gproj_attn_bwd_varlen",
+           "gproj_attn_varlen_qk_plan_bytes", "gproj_attn_varlen_qk_plan", "gproj_attn_fwd_varlen_qk", "gproj_attn_bwd_varlen_qk",
            "gproj_attn_host_staging_bytes", "gproj_attn_fwd_bwd_host",
            "gproj_last_device_status", "gproj_selftest_wait_timeout",
            "gproj_status_string", "gproj_last_launch_count")
@@ -76,6 +77,14 @@ def load():
         lib.gproj_attn_bwd_varlen_workspace_bytes.argtypes = [ip, i, i, i]
         lib.gproj_attn_bwd_varlen.restype = i
         lib.gproj_attn_bwd_varlen.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ip, i, vp, i, i, i, f, i, vp, ctypes.c_size_t, u, vp]
+        lib.gproj_attn_varlen_qk_plan_bytes.restype = ctypes.c_size_t
+        lib.gproj_attn_varlen_qk_plan_bytes.argtypes = [ip, ip, i]
+        lib.gproj_attn_varlen_qk_plan.restype = i
+        lib.gproj_attn_varlen_qk_plan.argtypes = [ip, ip, i, i, vp, ctypes.c_size_t]
+        lib.gproj_attn_fwd_varlen_qk.restype = i
+        lib.gproj_attn_fwd_varlen_qk.argtypes = [vp, vp, vp, vp, vp, ip, ip, i, vp, i, i, i, f, i, u, vp]
+        lib.gproj_attn_bwd_varlen_qk.restype = i
+        lib.gproj_attn_bwd_varlen_qk.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ip, ip, i, vp, i, i, i, f, i, vp, ctypes.c_size_t, u, vp]
         lib.gproj_attn_host_staging_bytes.restype = ctypes.c_size_t
         lib.gproj_attn_host_staging_bytes.argtypes = [i, i, i, i, i]
         lib.gproj_attn_fwd_bwd_host.restype = i
@@ -273,19 +282,33 @@ def gproj_last_launch_count() -> int:
 
 
 class VarlenPlan:
-    """Packed-sequence description: host cu_seqlens plus the device tile list the kernels walk (built once per packing)."""
+    """Packed-sequence description: host cu_seqlens plus the device tile list the kernels walk (built once per packing).
 
-    def __init__(self, cu_seqlens, causal, device="cuda"):
+    With ``cu_seqlens_k`` the sequences' key lengths differ from their query lengths (the ``*_varlen_qk`` calls)."""
+
+    def __init__(self, cu_seqlens, causal, device="cuda", cu_seqlens_k=None):
         cu = [int(x) for x in cu_seqlens]
         self.num_seqs = len(cu) - 1
         self.cu = (ctypes.c_int * len(cu))(*cu)
         self.causal = bool(causal)
         self.total = cu[-1]
-        nbytes = int(load().gproj_attn_varlen_plan_bytes(self.cu, self.num_seqs))
-        if nbytes == 0 and self.total <= 0:
+        self.cu_k, self.total_k = None, self.total
+        if cu_seqlens_k is not None:
+            ck = [int(x) for x in cu_seqlens_k]
+            if len(ck) != len(cu):
+                raise ValueError("cu_seqlens_k must have as many entries as cu_seqlens")
+            self.cu_k = (ctypes.c_int * len(ck))(*ck)
+            self.total_k = ck[-1]
+            nbytes = int(load().gproj_attn_varlen_qk_plan_bytes(self.cu, self.cu_k, self.num_seqs))
+        else:
+            nbytes = int(load().gproj_attn_varlen_plan_bytes(self.cu, self.num_seqs))
+        if nbytes == 0 and (self.total <= 0 or self.total_k <= 0):
             raise GprojError(-2, "gproj_attn_varlen_plan_bytes")
         host = torch.empty(max(nbytes, 16), dtype=torch.uint8)
-        rc = load().gproj_attn_varlen_plan(self.cu, self.num_seqs, int(self.causal), ctypes.c_void_p(host.data_ptr()), nbytes)
+        if self.cu_k is not None:
+            rc = load().gproj_attn_varlen_qk_plan(self.cu, self.cu_k, self.num_seqs, int(self.causal), ctypes.c_void_p(host.data_ptr()), nbytes)
+        else:
+            rc = load().gproj_attn_varlen_plan(self.cu, self.num_seqs, int(self.causal), ctypes.c_void_p(host.data_ptr()), nbytes)
         if rc != GPROJ_OK:
             raise GprojError(rc, "gproj_attn_varlen_plan")
         self.host = host
@@ -354,3 +377,49 @@ def gproj_attn_fwd_bwd_host(Q, K, V, dO, dQ, dK, dV, softmax_scale, causal, stag
                                             _stream(staging.device))
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_fwd_bwd_host")
+
+
+def _packed_qk_shapes(Q, K, V, plan):
+    _check_bf16("Q", Q)
+    H, Tq, d = Q.shape
+    _check_bf16("K", K); _check_bf16("V", V, K.shape)
+    if plan.cu_k is None:
+        raise ValueError("the plan has no cu_seqlens_k: build it with VarlenPlan(cu_q, causal, cu_seqlens_k=cu_k)")
+    if K.dim() != 3 or K.shape[2] != d or H % K.shape[0] != 0 or Tq != plan.total or K.shape[1] != plan.total_k:
+        raise ValueError("packed tensors must be Q [H, Tq, d], K/V [Hkv, Tk, d] with Tq, Tk the last offsets and H a multiple of Hkv")
+    return H, K.shape[0], Tq, d
+
+
+def gproj_attn_fwd_varlen_qk(Q, K, V, plan, softmax_scale, fwd_flags=0):
+    """O, LSE = forward over packed sequences with their own query and key lengths.  Q: [H, Tq, d]; K, V: [Hkv, Tk, d]."""
+    H, Hkv, Tq, d = _packed_qk_shapes(Q, K, V, plan)
+    O = torch.empty_like(Q)
+    LSE = torch.empty((H, Tq), dtype=torch.float32, device=Q.device)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_fwd_varlen_qk(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), plan.cu, plan.cu_k,
+                                             plan.num_seqs, plan.device.data_ptr(), H, Hkv, d, float(softmax_scale),
+                                             int(plan.causal), int(fwd_flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_fwd_varlen_qk")
+    return O, LSE
+
+
+def gproj_attn_bwd_varlen_qk(Q, K, V, O, LSE, dO, plan, softmax_scale, flags=0, workspace=None):
+    """dQ, dK, dV = backward of gproj_attn_fwd_varlen_qk (same layout; dK, dV like K)."""
+    H, Hkv, Tq, d = _packed_qk_shapes(Q, K, V, plan)
+    for name, t in (("O", O), ("dO", dO)):
+        _check_bf16(name, t, Q.shape)
+    if not (LSE.is_cuda and LSE.dtype == torch.float32 and LSE.is_contiguous() and tuple(LSE.shape) == (H, Tq)):
+        raise TypeError("LSE must be a contiguous CUDA float32 tensor [H, Tq]")
+    need = int(load().gproj_attn_bwd_varlen_workspace_bytes(plan.cu, plan.num_seqs, H, d))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_attn_bwd_varlen_qk(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
+                                             dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), plan.cu, plan.cu_k, plan.num_seqs,
+                                             plan.device.data_ptr(), H, Hkv, d, float(softmax_scale), int(plan.causal),
+                                             workspace.data_ptr(), workspace.numel(), int(flags), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_attn_bwd_varlen_qk")
+    return dQ, dK, dV

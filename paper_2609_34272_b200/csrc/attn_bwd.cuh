@@ -97,14 +97,15 @@ struct TileSched {
 
 // One 128-row tile of one sequence.  Rows are counted inside a head ([heads][rows][d] tensors): dense calls have one
 // sequence [0, N) per head; packed (variable-length) calls have several, listed tile by tile in a plan the host
-// prepared: {row0, seq0, seq_end, blk0} with blk0 the sequence's first 64-row block of row statistics.
+// prepared, two int4 per tile: {row0, seq0, seq_end, blk0} with blk0 the first 64-row block of row statistics of the
+// sequence's QUERIES, and {oseq0, oseq_end, -, -}.
 // [oseq0, oseq_end) is the range of the OTHER operand's rows the tile works against (keys for a query tile, queries for a
-// key tile); it differs from [seq0, seq_end) only in dense calls with unequal query and key lengths.
+// key tile); it differs from [seq0, seq_end) when query and key lengths are unequal.
 struct TileInfo { int row0, seq0, seq_end, blk0, oseq0, oseq_end; };
 __device__ __forceinline__ TileInfo tile_info(const int4 *plan, int idx, int dense_tile, int N, int N_other) {
   if (plan != nullptr) {
-    const int4 e = __ldg(plan + idx);
-    return TileInfo{e.x, e.y, e.z, e.w, e.y, e.z};
+    const int4 e = __ldg(plan + 2 * idx), o = __ldg(plan + 2 * idx + 1);
+    return TileInfo{e.x, e.y, e.z, e.w, o.x, o.y};
   }
   return TileInfo{128 * dense_tile, 0, N, 0, 0, N_other};
 }

@@ -169,7 +169,7 @@ int launch_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE,
 int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
                void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int Nk, int d, float softmax_scale, int causal,
                void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
-               int n_plan_tiles, int nblk, void *stream);
+               int n_plan_q_tiles, int n_plan_kv_tiles, int nblk, void *stream);
 
 // Row statistics {-LSE log2 e, -D}: blocks of 64 rows, 512 B each (per head ceil(N / 64) of them, the last one
 // zero-padded), plus one spare block: the 128-wide steps fetch two blocks at a time and may reach one past the end.
@@ -273,19 +273,19 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
                        void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int d, float softmax_scale, int causal,
                        void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
   return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, Hkv, N, N, d, softmax_scale, causal, workspace, workspace_bytes, flags,
-                    nullptr, nullptr, 0, (N + 63) / 64, stream);
+                    nullptr, nullptr, 0, 0, (N + 63) / 64, stream);
 }
 
 }  // extern "C"
 
 namespace {
 
-// Dense call: plans == nullptr.  Packed call: B = 1, N = total tokens, plan_q / plan_kv = device tile lists in the order
-// of the dQ-side and the dK/dV-side kernel, nblk = 64-row statistic blocks per head.
+// Dense call: plans == nullptr.  Packed call: B = 1, N / Nk = total query / key rows, plan_q / plan_kv = device tile lists
+// in the order of the dQ-side and the dK/dV-side kernel, nblk = 64-row statistic blocks per head.
 int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
                void *dQ, void *dK, void *dV, int B, int H, int Hkv, int N, int Nk, int d, float softmax_scale, int causal,
                void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
-               int n_plan_tiles, int nblk, void *stream) {
+               int n_plan_q_tiles, int n_plan_kv_tiles, int nblk, void *stream) {
   if (!Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return GPROJ_ERR_NULL;
   if (int rc = check_shape(B, H, N, d)) return rc;
   if (Hkv <= 0 || H % Hkv != 0 || check_shape(B, Hkv, Nk, d) != GPROJ_OK) return GPROJ_ERR_SHAPE;
@@ -296,7 +296,8 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
   if (!std::isfinite(softmax_scale) || !(softmax_scale > 0.f)) return GPROJ_ERR_SCALE;
   if (flags & ~(GPROJ_FLAG_NO_Q_CORRECTION | GPROJ_FLAG_NO_K_CORRECTION | GPROJ_FLAG_ONLY_DQ_PASS | GPROJ_FLAG_ONLY_DKV_PASS))
     return GPROJ_ERR_FLAGS;
-  const bool run_dq = !(flags & GPROJ_FLAG_ONLY_DKV_PASS), run_dkv = !(flags & GPROJ_FLAG_ONLY_DQ_PASS);
+  const bool run_dq = !(flags & GPROJ_FLAG_ONLY_DKV_PASS);
+  bool run_dkv = !(flags & GPROJ_FLAG_ONLY_DQ_PASS);
   if (!run_dq && !run_dkv) return GPROJ_ERR_FLAGS;
   const size_t stats_sz = stats_blocks_bytes(static_cast<size_t>(B) * H * nblk);
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
@@ -318,9 +319,10 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
   if (!ok) return GPROJ_ERR_CUDA;
 
   const float scale_log2 = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634);
-  const int n_qt = plan_q ? n_plan_tiles : (N + 127) / 128, n_kt = plan_q ? n_plan_tiles : (Nk + 127) / 128;
+  const int n_qt = plan_q ? n_plan_q_tiles : (N + 127) / 128, n_kt = plan_q ? n_plan_kv_tiles : (Nk + 127) / 128;
   const int total_tiles = BH * n_qt, total_kv_tiles = BHkv * n_kt;
   if (total_tiles <= 0) return GPROJ_OK;   // nothing but empty sequences
+  if (total_kv_tiles <= 0) run_dkv = false;   // packed call in which no sequence has both queries and keys
   const dim3 grid(static_cast<unsigned>(total_tiles < st->sm_count ? total_tiles : st->sm_count));   // persistent: one CTA per SM
   const dim3 grid_kv(static_cast<unsigned>(total_kv_tiles < st->sm_count ? total_kv_tiles : st->sm_count));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -377,7 +379,7 @@ int gproj_attn_bwd_rect(const void *Q, const void *K, const void *V, const void 
                         void *dQ, void *dK, void *dV, int B, int H, int Hkv, int Nq, int Nk, int d, float softmax_scale,
                         int causal, void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
   return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, B, H, Hkv, Nq, Nk, d, softmax_scale, causal, workspace, workspace_bytes,
-                    flags, nullptr, nullptr, 0, (Nq + 63) / 64, stream);
+                    flags, nullptr, nullptr, 0, 0, (Nq + 63) / 64, stream);
 }
 
 // ---- packed (variable-length) sequences ------------------------------------------------------------
@@ -385,23 +387,106 @@ int gproj_attn_bwd_rect(const void *Q, const void *K, const void *V, const void 
 
 namespace {
 
-struct PackedShape { int total, n_tiles, nblk; };
+// total_q / total_k: rows per head of the query-side / key-side tensors; q_tiles: query tiles of sequences with queries;
+// kv_tiles: key tiles of sequences with both queries and keys; nblk: 64-row statistic blocks of the queries.
+struct PackedShape { int total_q, total_k, q_tiles, kv_tiles, nblk; };
 
-// cu_seqlens: num_seqs + 1 non-decreasing row offsets, the first one 0.  Empty sequences are allowed and skipped.
-bool packed_shape(const int *cu, int num_seqs, PackedShape *out) {
-  if (!cu || num_seqs <= 0 || cu[0] != 0) return false;
-  long long tiles = 0, blocks = 0;
+// cu_q, cu_k: num_seqs + 1 non-decreasing row offsets each, the first one 0 (cu_k == cu_q: equal lengths).  Sequences
+// without queries, without keys or without both are allowed.
+bool packed_shape(const int *cu_q, const int *cu_k, int num_seqs, PackedShape *out) {
+  if (!cu_q || !cu_k || num_seqs <= 0 || cu_q[0] != 0 || cu_k[0] != 0) return false;
+  long long q_tiles = 0, kv_tiles = 0, blocks = 0;
   for (int s = 0; s < num_seqs; ++s) {
-    const long long len = static_cast<long long>(cu[s + 1]) - cu[s];
-    if (len < 0) return false;
-    tiles += (len + 127) / 128;
-    blocks += (len + 63) / 64;
+    const long long lq = static_cast<long long>(cu_q[s + 1]) - cu_q[s], lk = static_cast<long long>(cu_k[s + 1]) - cu_k[s];
+    if (lq < 0 || lk < 0) return false;
+    q_tiles += (lq + 127) / 128;
+    if (lq > 0) kv_tiles += (lk + 127) / 128;
+    blocks += (lq + 63) / 64;
   }
-  if (cu[num_seqs] <= 0 || tiles >= (1LL << 24)) return false;
-  out->total = cu[num_seqs];
-  out->n_tiles = static_cast<int>(tiles);
+  if (cu_q[num_seqs] <= 0 || cu_k[num_seqs] <= 0 || q_tiles >= (1LL << 24) || kv_tiles >= (1LL << 24)) return false;
+  out->total_q = cu_q[num_seqs];
+  out->total_k = cu_k[num_seqs];
+  out->q_tiles = static_cast<int>(q_tiles);
+  out->kv_tiles = static_cast<int>(kv_tiles);
   out->nblk = static_cast<int>(blocks);
   return true;
+}
+
+size_t plan_bytes_of(const PackedShape &ps) { return 2 * (static_cast<size_t>(ps.q_tiles) + ps.kv_tiles) * sizeof(int4); }
+
+// Tile list of a packing: the query tiles in the order the query-stationary kernels deal them, then the key tiles in the
+// order of the key-stationary kernel; two int4 per tile, {row0, seq0, seq_end, first statistics block of the sequence's
+// queries} and {other operand's seq0, seq_end, 0, 0}.
+int build_plan(const int *cu_q, const int *cu_k, int num_seqs, int causal, void *plan_host, size_t plan_bytes) {
+  PackedShape ps;
+  if (!packed_shape(cu_q, cu_k, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
+  if (!plan_host) return GPROJ_ERR_NULL;
+  if (plan_bytes < plan_bytes_of(ps)) return GPROJ_ERR_WORKSPACE;
+  struct Entry { int4 e, o; long long work; };
+  std::vector<Entry> vq, vk;
+  vq.reserve(static_cast<size_t>(ps.q_tiles));
+  vk.reserve(static_cast<size_t>(ps.kv_tiles));
+  int blk0 = 0;
+  for (int s = 0; s < num_seqs; ++s) {
+    const int q0 = cu_q[s], q1 = cu_q[s + 1], k0 = cu_k[s], k1 = cu_k[s + 1], lq = q1 - q0, lk = k1 - k0;
+    const long long off = static_cast<long long>(lk) - lq;   // causal: query i sees the keys j <= i + off
+    for (int t = 0; t * 128 < lq; ++t) {
+      const long long last_row = std::min<long long>((t + 1) * 128LL, lq) - 1;
+      const long long keys = causal ? std::max<long long>(0, std::min<long long>(lk, last_row + 1 + off)) : lk;
+      vq.push_back(Entry{make_int4(q0 + 128 * t, q0, q1, blk0), make_int4(k0, k1, 0, 0), keys});
+    }
+    for (int t = 0; lq > 0 && t * 128 < lk; ++t) {
+      const long long first_q = causal ? std::max<long long>(0, 128LL * t - off) : 0;
+      vk.push_back(Entry{make_int4(k0 + 128 * t, k0, k1, blk0), make_int4(q0, q1, 0, 0), std::max<long long>(0, lq - first_q)});
+    }
+    blk0 += (lq + 63) / 64;
+  }
+  // the persistent kernels deal tiles in this order: longest first (stable, so equal tiles keep their memory order)
+  auto by_work = [](const Entry &a, const Entry &b) { return a.work > b.work; };
+  std::stable_sort(vq.begin(), vq.end(), by_work);
+  std::stable_sort(vk.begin(), vk.end(), by_work);
+  int4 *out = static_cast<int4 *>(plan_host);
+  for (const Entry &en : vq) { *out++ = en.e; *out++ = en.o; }
+  for (const Entry &en : vk) { *out++ = en.e; *out++ = en.o; }
+  return GPROJ_OK;
+}
+
+int fwd_packed(const void *Q, const void *K, const void *V, void *O, float *LSE, const int *cu_q, const int *cu_k, int num_seqs,
+               const void *plan_device, int H, int Hkv, int d, float softmax_scale, int causal, unsigned fwd_flags, void *stream) {
+  PackedShape ps;
+  if (!packed_shape(cu_q, cu_k, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
+  if (!plan_device) return GPROJ_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
+  return launch_fwd(Q, K, V, O, LSE, 1, H, Hkv, ps.total_q, ps.total_k, d, softmax_scale, causal, fwd_flags,
+                    static_cast<const int4 *>(plan_device), ps.q_tiles, stream);
+}
+
+int bwd_packed(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO, void *dQ, void *dK,
+               void *dV, const int *cu_q, const int *cu_k, int num_seqs, const void *plan_device, int H, int Hkv, int d,
+               float softmax_scale, int causal, void *workspace, size_t workspace_bytes, unsigned flags, void *stream) {
+  PackedShape ps;
+  if (!packed_shape(cu_q, cu_k, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
+  if (!plan_device) return GPROJ_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
+  const int4 *plan = static_cast<const int4 *>(plan_device);
+  const int rc = launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, 1, H, Hkv, ps.total_q, ps.total_k, d, softmax_scale, causal, workspace,
+                            workspace_bytes, flags, plan, plan + 2 * static_cast<size_t>(ps.q_tiles), ps.q_tiles, ps.kv_tiles,
+                            ps.nblk, stream);
+  if (rc != GPROJ_OK || (flags & GPROJ_FLAG_ONLY_DQ_PASS)) return rc;
+  // Keys of a sequence without queries are in no tile: their gradient rows are zero.
+  const int launches = tl_launch_count;
+  const size_t row = static_cast<size_t>(d) * 2, pitch = static_cast<size_t>(ps.total_k) * row;
+  for (int s = 0; s < num_seqs; ++s) {
+    if (cu_q[s + 1] != cu_q[s] || cu_k[s + 1] == cu_k[s]) continue;
+    const size_t at = static_cast<size_t>(cu_k[s]) * row, width = static_cast<size_t>(cu_k[s + 1] - cu_k[s]) * row;
+    if (cudaMemset2DAsync(static_cast<uint8_t *>(dK) + at, pitch, 0, width, Hkv, static_cast<cudaStream_t>(stream)) != cudaSuccess ||
+        cudaMemset2DAsync(static_cast<uint8_t *>(dV) + at, pitch, 0, width, Hkv, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return GPROJ_ERR_CUDA;
+    }
+  }
+  tl_launch_count = launches;
+  return GPROJ_OK;
 }
 
 }  // namespace
@@ -409,69 +494,58 @@ bool packed_shape(const int *cu, int num_seqs, PackedShape *out) {
 extern "C" {
 
 size_t gproj_attn_varlen_plan_bytes(const int *cu_seqlens, int num_seqs) {
-  PackedShape ps;
-  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return 0;
-  return 2 * static_cast<size_t>(ps.n_tiles) * sizeof(int4);
+  return gproj_attn_varlen_qk_plan_bytes(cu_seqlens, cu_seqlens, num_seqs);
 }
 
 int gproj_attn_varlen_plan(const int *cu_seqlens, int num_seqs, int causal, void *plan_host, size_t plan_bytes) {
-  PackedShape ps;
-  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
-  if (!plan_host) return GPROJ_ERR_NULL;
-  if (plan_bytes < 2 * static_cast<size_t>(ps.n_tiles) * sizeof(int4)) return GPROJ_ERR_WORKSPACE;
-  struct Entry { int4 e; long long work_q, work_kv; };
-  std::vector<Entry> v;
-  v.reserve(static_cast<size_t>(ps.n_tiles));
-  int blk0 = 0;
-  for (int s = 0; s < num_seqs; ++s) {
-    const int seq0 = cu_seqlens[s], seq_end = cu_seqlens[s + 1], len = seq_end - seq0;
-    for (int t = 0; t * 128 < len; ++t) {
-      Entry en;
-      en.e = make_int4(seq0 + 128 * t, seq0, seq_end, blk0);
-      const int upto = (t + 1) * 128 < len ? (t + 1) * 128 : len;
-      en.work_q = causal ? upto : len;            // keys a query tile walks
-      en.work_kv = causal ? len - 128 * t : len;  // queries a key tile walks
-      v.push_back(en);
-    }
-    blk0 += (len + 63) / 64;
-  }
-  int4 *out = static_cast<int4 *>(plan_host);
-  // the persistent kernels deal tiles in this order: longest first (stable, so equal tiles keep their memory order)
-  std::stable_sort(v.begin(), v.end(), [](const Entry &a, const Entry &b) { return a.work_q > b.work_q; });
-  for (size_t i = 0; i < v.size(); ++i) out[i] = v[i].e;
-  std::stable_sort(v.begin(), v.end(), [](const Entry &a, const Entry &b) { return a.work_kv > b.work_kv; });
-  for (size_t i = 0; i < v.size(); ++i) out[v.size() + i] = v[i].e;
-  return GPROJ_OK;
+  return build_plan(cu_seqlens, cu_seqlens, num_seqs, causal, plan_host, plan_bytes);
 }
 
 int gproj_attn_fwd_varlen(const void *Q, const void *K, const void *V, void *O, float *LSE, const int *cu_seqlens,
                           int num_seqs, const void *plan_device, int H, int Hkv, int d, float softmax_scale, int causal,
                           unsigned fwd_flags, void *stream) {
-  PackedShape ps;
-  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
-  if (!plan_device) return GPROJ_ERR_NULL;
-  if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
-  return launch_fwd(Q, K, V, O, LSE, 1, H, Hkv, ps.total, ps.total, d, softmax_scale, causal, fwd_flags,
-                    static_cast<const int4 *>(plan_device), ps.n_tiles, stream);
+  return fwd_packed(Q, K, V, O, LSE, cu_seqlens, cu_seqlens, num_seqs, plan_device, H, Hkv, d, softmax_scale, causal, fwd_flags, stream);
 }
 
 size_t gproj_attn_bwd_varlen_workspace_bytes(const int *cu_seqlens, int num_seqs, int H, int d) {
   PackedShape ps;
-  if (!packed_shape(cu_seqlens, num_seqs, &ps) || check_shape(1, H, ps.total, d) != GPROJ_OK) return 0;
-  return stats_blocks_bytes(static_cast<size_t>(H) * ps.nblk) + align256(static_cast<size_t>(H) * ps.total * static_cast<size_t>(d) * 2);
+  if (!packed_shape(cu_seqlens, cu_seqlens, num_seqs, &ps) || check_shape(1, H, ps.total_q, d) != GPROJ_OK) return 0;
+  return stats_blocks_bytes(static_cast<size_t>(H) * ps.nblk) + align256(static_cast<size_t>(H) * ps.total_q * static_cast<size_t>(d) * 2);
 }
 
 int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
                           void *dQ, void *dK, void *dV, const int *cu_seqlens, int num_seqs, const void *plan_device, int H,
                           int Hkv, int d, float softmax_scale, int causal, void *workspace, size_t workspace_bytes,
                           unsigned flags, void *stream) {
+  return bwd_packed(Q, K, V, O, LSE, dO, dQ, dK, dV, cu_seqlens, cu_seqlens, num_seqs, plan_device, H, Hkv, d, softmax_scale, causal,
+                    workspace, workspace_bytes, flags, stream);
+}
+
+// packed sequences whose query and key lengths differ
+size_t gproj_attn_varlen_qk_plan_bytes(const int *cu_seqlens_q, const int *cu_seqlens_k, int num_seqs) {
   PackedShape ps;
-  if (!packed_shape(cu_seqlens, num_seqs, &ps)) return GPROJ_ERR_SHAPE;
-  if (!plan_device) return GPROJ_ERR_NULL;
-  if (reinterpret_cast<uintptr_t>(plan_device) & 15u) return GPROJ_ERR_ALIGN;
-  const int4 *plan = static_cast<const int4 *>(plan_device);
-  return launch_bwd(Q, K, V, O, LSE, dO, dQ, dK, dV, 1, H, Hkv, ps.total, ps.total, d, softmax_scale, causal, workspace, workspace_bytes,
-                    flags, plan, plan + ps.n_tiles, ps.n_tiles, ps.nblk, stream);
+  if (!packed_shape(cu_seqlens_q, cu_seqlens_k, num_seqs, &ps)) return 0;
+  return plan_bytes_of(ps);
+}
+
+int gproj_attn_varlen_qk_plan(const int *cu_seqlens_q, const int *cu_seqlens_k, int num_seqs, int causal, void *plan_host,
+                              size_t plan_bytes) {
+  return build_plan(cu_seqlens_q, cu_seqlens_k, num_seqs, causal, plan_host, plan_bytes);
+}
+
+int gproj_attn_fwd_varlen_qk(const void *Q, const void *K, const void *V, void *O, float *LSE, const int *cu_seqlens_q,
+                             const int *cu_seqlens_k, int num_seqs, const void *plan_device, int H, int Hkv, int d,
+                             float softmax_scale, int causal, unsigned fwd_flags, void *stream) {
+  return fwd_packed(Q, K, V, O, LSE, cu_seqlens_q, cu_seqlens_k, num_seqs, plan_device, H, Hkv, d, softmax_scale, causal, fwd_flags,
+                    stream);
+}
+
+int gproj_attn_bwd_varlen_qk(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
+                             void *dQ, void *dK, void *dV, const int *cu_seqlens_q, const int *cu_seqlens_k, int num_seqs,
+                             const void *plan_device, int H, int Hkv, int d, float softmax_scale, int causal, void *workspace,
+                             size_t workspace_bytes, unsigned flags, void *stream) {
+  return bwd_packed(Q, K, V, O, LSE, dO, dQ, dK, dV, cu_seqlens_q, cu_seqlens_k, num_seqs, plan_device, H, Hkv, d, softmax_scale,
+                    causal, workspace, workspace_bytes, flags, stream);
 }
 
 // ---- forward + backward from host buffers ----------------------------------------------------------

@@ -74,7 +74,8 @@ def test_python_binding_refuses_cpu_tensors():
 
 def test_varlen_plan_on_host(lib):
     # the plan is host arithmetic: every 128-row tile of every non-empty sequence exactly once in each of the two orders,
-    # longest work first, statistic blocks numbered sequence after sequence
+    # longest work first, statistic blocks numbered sequence after sequence; two int4 per tile, the second one the range
+    # of the other operand (here the same rows: equal query and key lengths)
     import numpy as np
     cu = [0, 1, 6, 70, 70, 470, 598]
     arr = (ctypes.c_int * len(cu))(*cu)
@@ -82,23 +83,65 @@ def test_varlen_plan_on_host(lib):
     lens = np.diff(cu)
     n_tiles = int(sum((l + 127) // 128 for l in lens))
     nbytes = lib.gproj_attn_varlen_plan_bytes(arr, S)
-    assert nbytes == 2 * n_tiles * 16
+    assert nbytes == 2 * n_tiles * 32
     for causal in (0, 1):
-        buf = np.zeros(2 * n_tiles * 4, dtype=np.int32)
+        buf = np.zeros(2 * n_tiles * 8, dtype=np.int32)
         assert lib.gproj_attn_varlen_plan(arr, S, causal, buf.ctypes.data_as(ctypes.c_void_p), nbytes) == 0
-        plan = buf.reshape(2, n_tiles, 4)
+        plan = buf.reshape(2, n_tiles, 8)
         expect = set()
         blk = 0
         for s in range(S):
             for t in range((lens[s] + 127) // 128):
-                expect.add((cu[s] + 128 * t, cu[s], cu[s + 1], blk))
+                expect.add((cu[s] + 128 * t, cu[s], cu[s + 1], blk, cu[s], cu[s + 1], 0, 0))
             blk += (lens[s] + 63) // 64
         for order in range(2):
             assert set(map(tuple, plan[order].tolist())) == expect and len(plan[order]) == len(expect)
-        work_q = [min(r0 + 128, e) - s0 if causal else e - s0 for r0, s0, e, _ in plan[0]]
-        work_kv = [e - r0 if causal else e - s0 for r0, s0, e, _ in plan[1]]
+        work_q = [min(r0 + 128, e) - s0 if causal else e - s0 for r0, s0, e, *_ in plan[0]]
+        work_kv = [e - r0 if causal else e - s0 for r0, s0, e, *_ in plan[1]]
         assert work_q == sorted(work_q, reverse=True) and work_kv == sorted(work_kv, reverse=True)
     assert lib.gproj_attn_varlen_plan(arr, S, 1, None, nbytes) == -1
     assert lib.gproj_attn_varlen_plan(arr, S, 1, ctypes.c_void_p(0x1000), 16) == -4
     bad = (ctypes.c_int * 3)(0, 5, 3)
     assert lib.gproj_attn_varlen_plan_bytes(bad, 2) == 0 and lib.gproj_attn_varlen_plan(bad, 2, 1, None, 0) == -2
+
+
+def test_varlen_qk_plan_on_host(lib):
+    # separate query and key offsets: query tiles of every sequence with queries, key tiles of every sequence with both;
+    # a query tile's work is the keys its last row sees, a key tile's the queries from the first one that sees it
+    import numpy as np
+    cu_q = [0, 100, 100, 400, 430, 431]
+    cu_k = [0, 300, 350, 480, 480, 1000]      # (100, 300), (0, 50), (300, 130), (30, 0), (1, 520)
+    aq = (ctypes.c_int * len(cu_q))(*cu_q); ak = (ctypes.c_int * len(cu_k))(*cu_k)
+    S = len(cu_q) - 1
+    lq, lk = np.diff(cu_q), np.diff(cu_k)
+    n_q = int(sum((l + 127) // 128 for l in lq))
+    n_k = int(sum((k + 127) // 128 for q, k in zip(lq, lk) if q > 0))
+    nbytes = lib.gproj_attn_varlen_qk_plan_bytes(aq, ak, S)
+    assert nbytes == (n_q + n_k) * 32
+    for causal in (0, 1):
+        buf = np.zeros((n_q + n_k) * 8, dtype=np.int32)
+        assert lib.gproj_attn_varlen_qk_plan(aq, ak, S, causal, buf.ctypes.data_as(ctypes.c_void_p), nbytes) == 0
+        plan = buf.reshape(n_q + n_k, 8)
+        exp_q, exp_k, blk = set(), set(), 0
+        for s in range(S):
+            for t in range((lq[s] + 127) // 128):
+                exp_q.add((cu_q[s] + 128 * t, cu_q[s], cu_q[s + 1], blk, cu_k[s], cu_k[s + 1], 0, 0))
+            if lq[s] > 0:
+                for t in range((lk[s] + 127) // 128):
+                    exp_k.add((cu_k[s] + 128 * t, cu_k[s], cu_k[s + 1], blk, cu_q[s], cu_q[s + 1], 0, 0))
+            blk += (lq[s] + 63) // 64
+        assert set(map(tuple, plan[:n_q].tolist())) == exp_q and set(map(tuple, plan[n_q:].tolist())) == exp_k
+
+        def keys_seen(r0, s0, e, _b, k0, k1, *_):
+            off = (k1 - k0) - (e - s0)
+            return max(0, min(k1 - k0, min(r0 + 128, e) - s0 + off)) if causal else k1 - k0
+
+        def queries_seeing(r0, s0, e, _b, q0, q1, *_):
+            off = (e - s0) - (q1 - q0)
+            return max(0, (q1 - q0) - max(0, r0 - s0 - off)) if causal else q1 - q0
+
+        wq = [keys_seen(*r) for r in plan[:n_q].tolist()]
+        wk = [queries_seeing(*r) for r in plan[n_q:].tolist()]
+        assert wq == sorted(wq, reverse=True) and wk == sorted(wk, reverse=True)
+    short = (ctypes.c_int * 2)(0, 0)
+    assert lib.gproj_attn_varlen_qk_plan_bytes(aq, short, 1) == 0        # no keys at all

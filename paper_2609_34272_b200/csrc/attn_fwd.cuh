@@ -98,7 +98,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t *sQ = smem;                              // tile 0, then tile 1 (each later reused to stage O_t)
   uint8_t *sKV = sQ + 2 * C::kTileBytes;            // stage s: K tile, then V tile
 
-  __shared__ uint64_t bar_q_full, bar_q_free, bar_k_full[S], bar_v_full[S], bar_kv_empty[S];
+  __shared__ uint64_t bar_q_full[2], bar_q_free[2], bar_k_full[S], bar_v_full[S], bar_kv_empty[S];
   __shared__ uint64_t bar_s_full[2], bar_s_free[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_turn[2], bar_merge, bar_drain[2];
   __shared__ float s_m1[2][128], s_l1[2][128];   // split mode: running maximum and normaliser of the second warpgroup
   __shared__ uint32_t tmem_base_smem;
@@ -117,9 +117,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
-    mbar_init(&bar_q_full, 1);
     mbar_init(&bar_merge, 128);
-    mbar_init(&bar_q_free, tiles_per_item);         // one arrival per query tile slot: its O store has left shared memory
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&bar_q_full[b], 1);
+      mbar_init(&bar_q_free[b], tiles_per_item);    // one arrival per query tile slot: its O store has left shared memory
+    }
     for (int s = 0; s < S; ++s) { mbar_init(&bar_k_full[s], 1); mbar_init(&bar_v_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(&bar_drain[t], 1);
@@ -162,6 +164,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     return t < it.nq && (!CAUSAL || j <= max(0, ((it.qt0 + t) * C::kBlockM + C::kBlockM - 1 + it.off) >> 7));
   };
 
+  // Q buffers: a pair item fills both tile slots of the one buffer; single-tile items (split mode) alternate between the
+  // two slots, so that the next item's Q is loaded, and its first scores are computed, during this item's epilogue.
+  auto q_buf = [&](int ti) { return split ? (ti & 1) : 0; };
+  auto q_use = [&](int ti) { return split ? (ti >> 1) : ti; };      // how often the buffer has been used before item ti
+
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of K_j, V_j
     if (lane == 0) {
@@ -196,14 +203,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
         const Item it = decode(lin);
         const int bh = lin % BH, tiles = it.nq;
-        if (ti >= 1) mbar_wait(&bar_q_free, (ti - 1) & 1, ab, kFwdWaitQFree);
-        mbar_expect_tx(&bar_q_full, tiles * C::kTileBytes);
+        const int qb = q_buf(ti), use = q_use(ti);
+        if (use >= 1) mbar_wait(&bar_q_free[qb], (use - 1) & 1, ab, kFwdWaitQFree);
+        mbar_expect_tx(&bar_q_full[qb], tiles * C::kTileBytes);
         for (int t = 0; t < tiles; ++t)
           for (int s = 0; s < C::kSlabs; ++s)
-            tma_load_3d(sQ + t * C::kTileBytes + s * C::kSlabBytes, &tmQ, &bar_q_full, s * 64, it.seq0 + (it.qt0 + t) * C::kBlockM, bh);
+            tma_load_3d(sQ + (qb + t) * C::kTileBytes + s * C::kSlabBytes, &tmQ, &bar_q_full[qb], s * 64, it.seq0 + (it.qt0 + t) * C::kBlockM, bh);
       }
-      if (cta_abort && ti > 0)
-        for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full, (ti - 1) & 1); ++spin) {}
+      if (cta_abort)
+        for (int q = (ti > 2 ? ti - 2 : 0); q < ti; ++q)
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full[q_buf(q)], q_use(q) & 1); ++spin) {}
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- tensor-core issuer 1: S_t = Q_t K_j^T
@@ -216,7 +225,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const Item it = decode(lin);
       const int T = it.n_kt;
-      mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
+      const int qb = q_buf(ti);
+      mbar_wait(&bar_q_full[qb], q_use(ti) & 1, ab, kFwdWaitQ);
       for (int j = 0; j < T; ++j, ++g) {
         const int st = g % S;
         mbar_wait(&bar_k_full[st], (g / S) & 1, ab, kFwdWaitK);
@@ -231,7 +241,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             else          mbar_wait(&bar_pv_done[t], (cnt[t] - 1) & 1, ab, kFwdWaitSFree);
           }
           tc_fence_after();
-          const SmemDesc dscQ = dscQ0.advanced(split ? 0 : t * C::kTileBytes);
+          const SmemDesc dscQ = dscQ0.advanced((split ? qb : t) * C::kTileBytes);
           if (elect_one_sync()) {
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
@@ -301,12 +311,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int jl = CAUSAL ? max(0, (qt * C::kBlockM + C::kBlockM - 1 + it.off) >> 7) : T;   // last key tile of this query tile
       const int jm = CAUSAL ? min((qt * C::kBlockM + it.off + 1) >> 7, it.klen >> 7) : (it.klen >> 7);
       // Split mode: stay in step with the item (its Q has landed), so that a warpgroup without key tiles cannot run ahead.
-      if (split) mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
+      const int qb = q_buf(ti);
+      if (split) mbar_wait(&bar_q_full[qb], q_use(ti) & 1, ab, kFwdWaitQ);
       if (!split && t >= it.nq) {
         // Odd number of query tiles: the last pair has no second tile.  Stay in step with the item (its Q has landed)
         // before handing back this slot, so that no barrier runs ahead of the roles that wait on it.
-        mbar_wait(&bar_q_full, ti & 1, ab, kFwdWaitQ);
-        if (row == 0) mbar_arrive(&bar_q_free);
+        mbar_wait(&bar_q_full[0], ti & 1, ab, kFwdWaitQ);
+        if (row == 0) mbar_arrive(&bar_q_free[0]);
         mbar_arrive(&bar_o_free[t]);
         continue;
       }
@@ -395,7 +406,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // ---- epilogue: O = BF16(acc / l) staged in the TMA layout over this tile's Q, LSE = alpha x_max + ln l
       if (cnt > cnt_item0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
       if (split && t == 1) {
-        // hand this half's statistics to warpgroup 0, which merges the two accumulators (l = 0: no key tiles here)
+        // hand this half's statistics to warpgroup 0, which merges the two accumulators (l = 0: no key tiles here).
+        // With two Q slots this warpgroup could finish a second item before warpgroup 0 has looked at the first one's
+        // hand-over, and the merge barrier would be two phases ahead of its waiter; so it first waits until
+        // warpgroup 0 has read the previous item's accumulators.
+        if (ti > 0) mbar_wait(&bar_o_free[1], (ti - 1) & 1, ab, kFwdWaitOFree);
         s_m1[ti & 1][row] = m_run;
         s_l1[ti & 1][row] = l_run;
         tc_fence_before();
@@ -420,7 +435,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
       }
       const float inv_l = has1 ? 1.0f : a0;            // with two halves the weights a_0, a_1 already carry 1 / l
-      uint8_t *stage = sQ + t * C::kTileBytes;         // no MMA reads this Q tile any more
+      uint8_t *stage = sQ + (split ? qb : t) * C::kTileBytes;   // no MMA reads this Q tile any more
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t o[32];
@@ -456,13 +471,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           for (int sl = 0; sl < C::kSlabs; ++sl) tma_store_3d(&tmO, stage + sl * C::kSlabBytes, sl * 64, qrow0, bh);
           bulk_commit_group();
           bulk_wait_group_read0();
-          mbar_arrive(&bar_q_free);                    // this tile's half of the Q buffer may be reloaded
+          mbar_arrive(&bar_q_free[qb]);                // this tile's slot of the Q buffer may be reloaded
         }
       } else {
         // ragged last tile of a packed sequence that another sequence follows: rows past its end are not ours to write
         store_rows_clipped<D>(stage, C::kSlabBytes, Og + (static_cast<size_t>(bh) * N + qrow0) * D, row, it.len - qt * C::kBlockM);
         named_bar_sync(1 + t, 128);
-        if (row == 0) mbar_arrive(&bar_q_free);
+        if (row == 0) mbar_arrive(&bar_q_free[qb]);
       }
     }
   }

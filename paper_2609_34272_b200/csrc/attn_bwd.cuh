@@ -74,7 +74,11 @@ struct BwdCfg {
   static constexpr int kDqStages = (D == 64) ? 6 : 4;
   static constexpr int kDqStageBytes = 2 * kStepTileBytes;
   static constexpr int kDqResBufs = (D == 64) ? 2 : 1;             // stationary (Q, dO) buffers
-  static constexpr int kDqSmemBytes = kDqResBufs * 2 * kBigTileBytes + kDqStages * kDqStageBytes + (kSepStaging ? 2 * kBigTileBytes : 0) + 1024;
+  // d = 64: the saved-output rows of the NEXT tile (for D = rowsum(dO o O)) are copied into shared memory asynchronously
+  // during the current tile's epilogue; at d = 128 there is no room and the rows are loaded at the tile's start.
+  static constexpr bool kPrefetchO = (D == 64);
+  static constexpr int kDqSmemBytes = kDqResBufs * 2 * kBigTileBytes + kDqStages * kDqStageBytes + (kSepStaging ? 2 * kBigTileBytes : 0) +
+                                      (kPrefetchO ? kBigTileBytes : 0) + 1024;
   // dK/dV-side kernel: K, V resident; ring of (Q, dO, Z, stats) step tiles
   static constexpr int kDkvStages = (D == 64) ? 5 : 3;
   static constexpr int kDkvStageBytes = 3 * kStepTileBytes + 1024;   // + 2 x 64 floats of row statistics (512 B used)
@@ -91,6 +95,10 @@ struct TileSched {
   __device__ __forceinline__ int next() {
     const int idx = round * G + ((round & 1) ? (G - 1 - c) : c);
     ++round;
+    return idx < total ? idx : -1;
+  }
+  __device__ __forceinline__ int peek() const {     // the item next() would return, without taking it
+    const int idx = round * G + ((round & 1) ? (G - 1 - c) : c);
     return idx < total ? idx : -1;
   }
 };
@@ -271,12 +279,13 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   uint8_t *sRes = smem;                                        // buffer rb: Q tile, then dO tile
   uint8_t *sKV = sRes + R * 2 * C::kBigTileBytes;              // stage s: K step tile, then V step tile
   uint8_t *sOut = sKV + S * C::kDqStageBytes;                  // staging (dQ tile, then Z tile) when separate
+  uint8_t *sO = sOut + (C::kSepStaging ? 2 * C::kBigTileBytes : 0);   // saved-output rows of the next tile (kPrefetchO), row-major
 
   __shared__ uint64_t bar_res_full[R], bar_res_free[R], bar_kv_full[S], bar_kv_empty[S];
   __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
-  __shared__ float s_rho[C::kWG - 1][128], s_m[C::kWG - 1][128], s_lam[128], s_D[128];
+  __shared__ float s_rho[C::kWG - 1][128], s_m[C::kWG - 1][128], s_lam[128], s_D[128], s_lse[128];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
@@ -442,6 +451,24 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
     const uint32_t slice_addr = tmem_base + lane_addr + C::kSliceCols * slice;
     int g0 = 0, ti = 0;
+    constexpr int L = D / 8, RPI = 32 / L;               // D computation: lanes per row, rows per warp-wide load
+    const int sub = lane / L, part = lane % L;
+    // kPrefetchO: the O rows and the LSE of tile lin_n travel to shared memory while the tile before it finishes
+    auto prefetch_tile = [&](int lin_n) {
+      const TileInfo tn = tile_of(lin_n);
+      const size_t hr0 = static_cast<size_t>(lin_n % BH) * N;
+#pragma unroll
+      for (int it = 0; it < 8 / RPI; ++it) {
+        const int r = 8 * (warp - 4) + it * RPI + sub;
+        if (tn.row0 + r < tn.seq_end) cp_async16(sO + r * (D * 2) + part * 16, Og + (hr0 + tn.row0 + r) * D + part * 8);
+      }
+      if (wg == 0 && tn.row0 + row < tn.seq_end) cp_async4(&s_lse[row], LSE + hr0 + tn.row0 + row);
+      cp_async_commit();
+    };
+    if (C::kPrefetchO) {
+      const int lin0 = sched.peek();
+      if (lin0 >= 0) prefetch_tile(lin0);
+    }
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const TileInfo tl = tile_of(lin);
       const int bh = lin % BH, T = steps_of(tl), rb = ti % R;
@@ -449,17 +476,28 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       const int qrow = tl.row0 + row;                  // this thread's query row within the head (past seq_end in a ragged tile)
 
       // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1): each of the 16 compute warps
-      // takes eight rows, coalesced 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
+      // takes eight rows, 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
+      if (C::kPrefetchO) {
+        cp_async_wait_all();                                      // this thread's share of the O rows and LSE
+        mbar_wait(&bar_res_full[rb], (ti / R) & 1, ab, kDqWaitQ);   // dO is read from the stationary tile
+        named_bar_sync(2, C::kCompute);                           // everybody's share
+      }
+      // read before the barrier below: the next tile's prefetch, which overwrites it, is issued behind that barrier
+      const float lse_pre = C::kPrefetchO ? s_lse[row] : 0.f;
       {
-        constexpr int L = D / 8, RPI = 32 / L;           // lanes per row, rows per warp-wide load
-        const int sub = lane / L, part = lane % L;
 #pragma unroll
         for (int it = 0; it < 8 / RPI; ++it) {
           const int r = 8 * (warp - 4) + it * RPI + sub;
           uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
           if (tl.row0 + r < tl.seq_end) {
-            a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + tl.row0 + r) * D) + part);
-            b = __ldg(reinterpret_cast<const uint4 *>(dOg + (head_row0 + tl.row0 + r) * D) + part);
+            if (C::kPrefetchO) {
+              a = *reinterpret_cast<const uint4 *>(sO + r * (D * 2) + part * 16);
+              b = *reinterpret_cast<const uint4 *>(sRes + rb * 2 * C::kBigTileBytes + C::kBigTileBytes + (part >> 3) * C::kBigSlabBytes +
+                                                   swz128_offset(r, part & 7));
+            } else {
+              a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + tl.row0 + r) * D) + part);
+              b = __ldg(reinterpret_cast<const uint4 *>(dOg + (head_row0 + tl.row0 + r) * D) + part);
+            }
           }
           const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
           float acc = 0.f;
@@ -475,7 +513,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
       named_bar_sync(2, C::kCompute);
       const float Dv = s_D[row];
-      const float neg_lse2 = (qrow < tl.seq_end) ? -LSE[head_row0 + qrow] * 1.4426950408889634f : 0.f;
+      const float lse_row = (qrow < tl.seq_end) ? (C::kPrefetchO ? lse_pre : LSE[head_row0 + qrow]) : 0.f;
+      const float neg_lse2 = -lse_row * 1.4426950408889634f;
       // Per 64-row block of a sequence (the last one padded with zeros): 64 x {-LSE log2 e}, then 64 x {-D}.
       const int rel = qrow - tl.seq0;                  // row inside the sequence
       if (wg == 0 && rel < ((tl.seq_end - tl.seq0 + C::kStepRows - 1) / C::kStepRows) * C::kStepRows) {
@@ -506,6 +545,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         mbar_arrive(&bar_tr_ready[b]);
       }
 
+      if (C::kPrefetchO) {
+        // every thread took its D and LSE out of shared memory before its first step (behind the barrier above), and dO of
+        // the next tile sits in the other stationary buffer: the next tile's rows may travel during this tile's epilogue
+        const int lin_n = sched.peek();
+        if (lin_n >= 0) prefetch_tile(lin_n);
+      }
       // ---- row statistics of all warpgroups (fixed order), lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
       float rho_lo, rho_hi, m_lo, m_hi;
       f32x2_split(rho2, rho_lo, rho_hi);

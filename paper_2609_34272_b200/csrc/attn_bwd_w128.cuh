@@ -121,7 +121,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   if (threadIdx.x == 0) {
     cta_abort = 0;
     mbar_init(&bar_res_full, 1);
-    mbar_init(&bar_res_free, 2);
+    mbar_init(&bar_res_free, 1);   // the last score product alone: the epilogue has its own staging buffer and never touches K / V
     for (int s = 0; s < S; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_s_full[b], 1); mbar_init(&bar_s_free[b], 1);
@@ -333,10 +333,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&bar_acc_free);          // the accumulators may be overwritten by the next tile
-      if (threadIdx.x == 128) {
-        mbar_arrive(&bar_res_free);        // second arrival: with its own staging buffer the epilogue never touches K / V
-        bulk_wait_group_read0();           // the previous tile's stores have left the staging buffer
-      }
+      if (threadIdx.x == 128) bulk_wait_group_read0();   // the previous tile's stores have left the staging buffer
       named_bar_sync(1, C::kCompute);
 #pragma unroll
       for (int v = 0; v < 2; ++v) {

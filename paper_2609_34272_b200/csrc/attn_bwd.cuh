@@ -322,7 +322,14 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 
   TileSched sched(total_tiles);
   // tile decode: causal -> longest rows first
-  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, CAUSAL ? (n_qt - 1 - lin / BH) : (lin / BH), N, Nk); };
+  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
+  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
+  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
+  const int n_per_head = total_tiles / BH;
+  const bool head_major = !CAUSAL && plan == nullptr;
+  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
+  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
+  auto tile_of = [&](int lin) { return tile_info(plan, tix(lin), CAUSAL ? (n_qt - 1 - tix(lin)) : tix(lin), N, Nk); };
   // 64-key steps of a query tile: the keys its last row sees (causal) or all of them; at least one step, fully masked
   // if the tile sees no key at all, so that every tile runs through the same pipeline.
   auto steps_of = [&](const TileInfo &t) {
@@ -337,7 +344,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
         const TileInfo tl = tile_of(lin);
-        const int bh = lin % BH, T = steps_of(tl);
+        const int bh = hix(lin), T = steps_of(tl);
         for (int n = 0; n < T; ++n, ++g) {
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kDqWaitKVEmpty);
@@ -362,7 +369,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int rb = ti % R, bh = lin % BH, qrow0 = tile_of(lin).row0;
+        const int rb = ti % R, bh = hix(lin), qrow0 = tile_of(lin).row0;
         if (ti >= R) mbar_wait(&bar_res_free[rb], ((ti / R) - 1) & 1, ab, kDqWaitResFree);
         mbar_expect_tx(&bar_res_full[rb], 2 * C::kBigTileBytes);
         uint8_t *dst = sRes + rb * 2 * C::kBigTileBytes;
@@ -456,7 +463,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     // kPrefetchO: the O rows and the LSE of tile lin_n travel to shared memory while the tile before it finishes
     auto prefetch_tile = [&](int lin_n) {
       const TileInfo tn = tile_of(lin_n);
-      const size_t hr0 = static_cast<size_t>(lin_n % BH) * N;
+      const size_t hr0 = static_cast<size_t>(hix(lin_n)) * N;
 #pragma unroll
       for (int it = 0; it < 8 / RPI; ++it) {
         const int r = 8 * (warp - 4) + it * RPI + sub;
@@ -471,7 +478,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     }
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const TileInfo tl = tile_of(lin);
-      const int bh = lin % BH, T = steps_of(tl), rb = ti % R;
+      const int bh = hix(lin), T = steps_of(tl), rb = ti % R;
       const size_t head_row0 = static_cast<size_t>(bh) * N;
       const int qrow = tl.row0 + row;                  // this thread's query row within the head (past seq_end in a ragged tile)
 
@@ -711,7 +718,14 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   // are zero and its padded statistics are zero, so t = 0 and r multiplies zero rows); key rows past N are clipped on store.
   // In a packed layout the query columns past the end of the sequence are the next sequence's rows and are masked.
   // N: key rows per head (own operand), Nq: query rows per head.  A key j is seen by the queries i >= j - (L_k - L_q).
-  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, lin / BH, N, Nq); };
+  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
+  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
+  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
+  const int n_per_head = total_tiles / BH;
+  const bool head_major = !CAUSAL && plan == nullptr;
+  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
+  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
+  auto tile_of = [&](int lin) { return tile_info(plan, tix(lin), tix(lin), N, Nq); };
   // First query (inside its sequence, rounded down to a 64-row statistics block) that sees this key tile, and the steps
   // from there to the end of the queries; at least one step, fully masked if no query sees the tile.
   auto q_start_of = [&](const TileInfo &t) {
@@ -730,7 +744,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
         const TileInfo tl = tile_of(lin);
-        const int bh = lin % BH, T = steps_of(tl), q_start = q_start_of(tl);
+        const int bh = hix(lin), T = steps_of(tl), q_start = q_start_of(tl);
         const int q_head0 = (bh / Hkv) * (Hkv * G) + (bh % Hkv) * G;     // first query head of the group (flat index)
         for (int n = 0; n < G * T; ++n, ++g) {
           const int st = g % S;
@@ -756,7 +770,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int bh = lin % BH, krow0 = tile_of(lin).row0;
+        const int bh = hix(lin), krow0 = tile_of(lin).row0;
         if (ti >= 1) mbar_wait(&bar_res_free, (ti - 1) & 1, ab, kDkvWaitResFree);
         mbar_expect_tx(&bar_res_full, 2 * C::kBigTileBytes);
         for (int s = 0; s < C::kSlabs; ++s) {
@@ -864,7 +878,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const TileInfo tl = tile_of(lin);
-      const int bh = lin % BH, Th = steps_of(tl), T = G * Th, q_start = q_start_of(tl);
+      const int bh = hix(lin), Th = steps_of(tl), T = G * Th, q_start = q_start_of(tl);
 #ifdef GPROJ_TRACE
       const unsigned long long tile_t0 = global_ns();
 #endif

@@ -149,7 +149,14 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   // A step may reach past the end of the sequence: those query columns are zero fill or the next packed sequence's rows,
   // and are masked.
   // N: key rows per head (own operand), Nq: query rows per head.  A key j is seen by the queries i >= j - (L_k - L_q).
-  auto tile_of = [&](int lin) { return tile_info(plan, lin / BH, lin / BH, N, Nq); };
+  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
+  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
+  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
+  const int n_per_head = total_tiles / BH;
+  const bool head_major = !CAUSAL && plan == nullptr;
+  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
+  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
+  auto tile_of = [&](int lin) { return tile_info(plan, tix(lin), tix(lin), N, Nq); };
   // First query (inside its sequence, rounded down to a 64-row statistics block) that sees this key tile, and the steps
   // from there to the end of the queries; at least one step, fully masked if no query sees the tile.
   auto q_start_of = [&](const TileInfo &t) {
@@ -168,7 +175,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
         const TileInfo tl = tile_of(lin);
-        const int bh = lin % BH, T = steps_of(tl), q_start = q_start_of(tl);
+        const int bh = hix(lin), T = steps_of(tl), q_start = q_start_of(tl);
         const int q_head0 = (bh / Hkv) * (Hkv * G) + (bh % Hkv) * G;     // first query head of the group (flat index)
         for (int n = 0; n < G * T; ++n, ++g) {
           const int st = g % S;
@@ -194,7 +201,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     if (lane == 0) {
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int bh = lin % BH, krow0 = tile_of(lin).row0;
+        const int bh = hix(lin), krow0 = tile_of(lin).row0;
         if (ti >= 1) mbar_wait(&bar_res_free, (ti - 1) & 1, ab, kWkResFree);
         mbar_expect_tx(&bar_res_full, 2 * C::kTileBytes);
         tma_load_3d(sK, &tmK, &bar_res_full, 0, krow0, bh);
@@ -292,7 +299,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const TileInfo tl = tile_of(lin);
-      const int bh = lin % BH, Th = steps_of(tl), T = G * Th, q_start = q_start_of(tl);
+      const int bh = hix(lin), Th = steps_of(tl), T = G * Th, q_start = q_start_of(tl);
       // (Issuing the first TMEM load of a phase early, when its barrier had already completed, and letting warpgroup pairs
       // take turns in phase 1, were both measured slower.)
       for (int n = 0; n < T; ++n) {

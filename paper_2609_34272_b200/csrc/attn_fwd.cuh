@@ -141,15 +141,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // qt0: index of the first query tile inside its sequence; nq: query tiles; n_kt: key tiles walked; kseq0, klen: the keys.
   // Causal support of query i: keys j <= i + off with off = klen - len (the diagonal ends at the last query and last key).
   struct Item { int seq0, len, qt0, nq, n_kt, kseq0, klen, off; };
+  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
+  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
+  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
+  const int n_per_head = total_items / BH;
+  const bool head_major = !CAUSAL && plan == nullptr;
+  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
+  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
   TileSched sched(total_items);
   auto decode = [&](int lin) {
     Item it;
     if (plan != nullptr) {
-      const TileInfo ti = tile_info(plan, lin / BH, 0, N, Nk);
+      const TileInfo ti = tile_info(plan, tix(lin), 0, N, Nk);
       it.seq0 = ti.seq0; it.len = ti.seq_end - ti.seq0; it.qt0 = (ti.row0 - ti.seq0) / C::kBlockM; it.nq = 1;
       it.kseq0 = ti.oseq0; it.klen = ti.oseq_end - ti.oseq0;
     } else {
-      const int pair = CAUSAL ? (n_pairs - 1 - lin / BH) : (lin / BH);
+      const int pair = CAUSAL ? (n_pairs - 1 - tix(lin)) : tix(lin);
       it.seq0 = 0; it.len = N; it.qt0 = TPI * pair; it.nq = min(TPI, n_qt - it.qt0);
       it.kseq0 = 0; it.klen = Nk;
     }
@@ -175,7 +182,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       int g = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next()) {
         const Item it = decode(lin);
-        const int bh = lin % BH, T = it.n_kt;
+        const int bh = hix(lin), T = it.n_kt;
         for (int j = 0; j < T; ++j, ++g) {
           const int st = g % S;
           if (g >= S) mbar_wait(&bar_kv_empty[st], ((g / S) - 1) & 1, ab, kFwdWaitKVEmpty);
@@ -202,7 +209,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
         const Item it = decode(lin);
-        const int bh = lin % BH, tiles = it.nq;
+        const int bh = hix(lin), tiles = it.nq;
         const int qb = q_buf(ti), use = q_use(ti);
         if (use >= 1) mbar_wait(&bar_q_free[qb], (use - 1) & 1, ab, kFwdWaitQFree);
         mbar_expect_tx(&bar_q_full[qb], tiles * C::kTileBytes);
@@ -302,7 +309,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     int ti = 0, cnt = 0, turn = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const Item it = decode(lin);
-      const int bh = lin % BH, T = it.n_kt;
+      const int bh = hix(lin), T = it.n_kt;
       const int qt = it.qt0 + (split ? 0 : t);        // this warpgroup's query tile inside the sequence
       // Masking, reduced to two numbers per tile: column c of key tile j is outside the row's support when
       // 128 j + c > rk, with rk the last key the row sees (causal diagonal and end of the keys, whichever comes first);

@@ -103,6 +103,26 @@ struct TileSched {
   }
 };
 
+// Item number -> (rank of the tile in decreasing work, head).  Items are dealt in groups of `group` consecutive ranks of
+// all heads; inside a group the ranks of one head are adjacent, so that CTAs running at the same time work on the same
+// head and share the rows they stream (the other operand) in L2 instead of fetching one head each out of HBM.
+// group = 1: every head's longest tile first (the exact longest-first order; packed calls, whose plan is already
+// sorted); group = tiles per head: head-major (dense non-causal calls, whose tiles are all alike); in between for
+// causal calls with many heads, where a few adjacent ranks differ little in work.
+struct ItemOrder {
+  int gk, per_group, n_full, rem;   // ranks per group, items per group (heads x gk), full groups, ranks of the short last group
+#ifdef __CUDACC__
+  __device__ __forceinline__ int rank(int lin) const {
+    const int g = lin / per_group, within = lin - g * per_group;
+    return g * gk + within % ((g < n_full) ? gk : rem);
+  }
+  __device__ __forceinline__ int head(int lin) const {
+    const int g = lin / per_group, within = lin - g * per_group;
+    return within / ((g < n_full) ? gk : rem);
+  }
+#endif
+};
+
 // One 128-row tile of one sequence.  Rows are counted inside a head ([heads][rows][d] tensors): dense calls have one
 // sequence [0, N) per head; packed (variable-length) calls have several, listed tile by tile in a plan the host
 // prepared, two int4 per tile: {row0, seq0, seq_end, blk0} with blk0 the first 64-row block of row statistics of the
@@ -270,7 +290,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
               const float *__restrict__ LSE, float *__restrict__ stats,
               __nv_bfloat16 *__restrict__ dQg, __nv_bfloat16 *__restrict__ Zg,   // plain-store targets of clipped tiles
               const int4 *__restrict__ plan, int nblk,                          // packed sequences: tile list; 64-row statistic blocks per head
-              int N, int Nk, int BH, int Hq, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+              int N, int Nk, int BH, int Hq, int G, int total_tiles, const ItemOrder order, float scale_log2, float alpha, unsigned flags, int *status) {
   // N: query rows per head (own operand), Nk: key rows per head.  Causal support of query i: keys j <= i + (L_k - L_q).
   using C = BwdCfg<D>;
   constexpr int NB = C::kNB, R = C::kDqResBufs, S = C::kDqStages;
@@ -322,13 +342,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 
   TileSched sched(total_tiles);
   // tile decode: causal -> longest rows first
-  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
-  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
-  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
-  const int n_per_head = total_tiles / BH;
-  const bool head_major = !CAUSAL && plan == nullptr;
-  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
-  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
+  auto tix = [&](int lin) { return order.rank(lin); };
+  auto hix = [&](int lin) { return order.head(lin); };
   auto tile_of = [&](int lin) { return tile_info(plan, tix(lin), CAUSAL ? (n_qt - 1 - tix(lin)) : tix(lin), N, Nk); };
   // 64-key steps of a query tile: the keys its last row sees (causal) or all of them; at least one step, fully masked
   // if the tile sees no key at all, so that every tile runs through the same pipeline.
@@ -660,7 +675,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
                const float *__restrict__ stats,
                __nv_bfloat16 *__restrict__ dKg, __nv_bfloat16 *__restrict__ dVg,   // plain-store targets of clipped tiles
                const int4 *__restrict__ plan, int nblk,                           // packed sequences: tile list; statistic blocks per head
-               int N, int Nq, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+               int N, int Nq, int BH, int Hkv, int G, int total_tiles, const ItemOrder order, float scale_log2, float alpha, unsigned flags, int *status) {
   // BH counts (batch, KV head) pairs here.  With grouped queries (G > 1) one work item walks the query steps of all G
   // query heads of its KV head, so their contributions are summed in the FP32 accumulators (Section 3.1: key and value
   // contributions also sum over the query heads that share a KV head).
@@ -718,13 +733,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   // are zero and its padded statistics are zero, so t = 0 and r multiplies zero rows); key rows past N are clipped on store.
   // In a packed layout the query columns past the end of the sequence are the next sequence's rows and are masked.
   // N: key rows per head (own operand), Nq: query rows per head.  A key j is seen by the queries i >= j - (L_k - L_q).
-  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
-  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
-  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
-  const int n_per_head = total_tiles / BH;
-  const bool head_major = !CAUSAL && plan == nullptr;
-  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
-  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
+  auto tix = [&](int lin) { return order.rank(lin); };
+  auto hix = [&](int lin) { return order.head(lin); };
   auto tile_of = [&](int lin) { return tile_info(plan, tix(lin), tix(lin), N, Nq); };
   // First query (inside its sequence, rounded down to a 64-row statistics block) that sees this key tile, and the steps
   // from there to the end of the queries; at least one step, fully masked if no query sees the tile.

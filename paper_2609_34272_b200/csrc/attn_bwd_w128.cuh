@@ -91,7 +91,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
                     const float *__restrict__ stats,
                     __nv_bfloat16 *__restrict__ dKg, __nv_bfloat16 *__restrict__ dVg,
                     const int4 *__restrict__ plan, int nblk,
-                    int N, int Nq, int BH, int Hkv, int G, int total_tiles, float scale_log2, float alpha, unsigned flags, int *status) {
+                    int N, int Nq, int BH, int Hkv, int G, int total_tiles, const ItemOrder order, float scale_log2, float alpha, unsigned flags, int *status) {
   // BH counts (batch, KV head) pairs.  With grouped queries one work item walks the query steps of all G query heads of
   // its KV head, so that their contributions are summed in the FP32 accumulators (Section 3.1).
   using C = BwdW128;
@@ -149,13 +149,8 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   // A step may reach past the end of the sequence: those query columns are zero fill or the next packed sequence's rows,
   // and are masked.
   // N: key rows per head (own operand), Nq: query rows per head.  A key j is seen by the queries i >= j - (L_k - L_q).
-  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
-  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
-  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
-  const int n_per_head = total_tiles / BH;
-  const bool head_major = !CAUSAL && plan == nullptr;
-  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
-  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
+  auto tix = [&](int lin) { return order.rank(lin); };
+  auto hix = [&](int lin) { return order.head(lin); };
   auto tile_of = [&](int lin) { return tile_info(plan, tix(lin), tix(lin), N, Nq); };
   // First query (inside its sequence, rounded down to a 64-row statistics block) that sees this key tile, and the steps
   // from there to the end of the queries; at least one step, fully masked if no query sees the tile.

@@ -89,7 +89,7 @@ template <int D, bool CAUSAL, bool FMA_SOFTMAX, int MODE>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                __nv_bfloat16 *__restrict__ Og, const int4 *__restrict__ plan, float *__restrict__ LSE, int N, int Nk, int BH, int Hq, int G, int tiles_per_item, int total_items, float scale_log2, float alpha,
+                __nv_bfloat16 *__restrict__ Og, const int4 *__restrict__ plan, float *__restrict__ LSE, int N, int Nk, int BH, int Hq, int G, int tiles_per_item, int total_items, const ItemOrder order, float scale_log2, float alpha,
                 int *status) {
   using C = FwdCfg<D>;
   constexpr int S = C::kStages;
@@ -98,6 +98,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t *sQ = smem;                              // tile 0, then tile 1 (each later reused to stage O_t)
   uint8_t *sKV = sQ + 2 * C::kTileBytes;            // stage s: K tile, then V tile
 
+  __shared__ int s_item[4][2];
   __shared__ uint64_t bar_q_full[2], bar_q_free[2], bar_k_full[S], bar_v_full[S], bar_kv_empty[S];
   __shared__ uint64_t bar_s_full[2], bar_s_free[2], bar_p_ready[2], bar_pv_done[2], bar_o_free[2], bar_turn[2], bar_merge, bar_drain[2];
   __shared__ float s_m1[2][128], s_l1[2][128];   // split mode: running maximum and normaliser of the second warpgroup
@@ -141,22 +142,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // qt0: index of the first query tile inside its sequence; nq: query tiles; n_kt: key tiles walked; kseq0, klen: the keys.
   // Causal support of query i: keys j <= i + off with off = klen - len (the diagonal ends at the last query and last key).
   struct Item { int seq0, len, qt0, nq, n_kt, kseq0, klen, off; };
-  // Item -> (tile, head).  Causal and packed calls order items by decreasing work: every head's longest tile first.  Dense
-  // non-causal tiles are all alike; there the tiles of one head are consecutive, so that the CTAs running at the same
-  // time stream the same rows of the other operand through L2 instead of one head each out of HBM.
-  const int n_per_head = total_items / BH;
-  const bool head_major = !CAUSAL && plan == nullptr;
-  auto tix = [&](int lin) { return head_major ? lin % n_per_head : lin / BH; };
-  auto hix = [&](int lin) { return head_major ? lin / n_per_head : lin % BH; };
+  auto tix = [&](int lin) { return order.rank(lin); };
+  auto hix = [&](int lin) { return order.head(lin); };
   TileSched sched(total_items);
-  auto decode = [&](int lin) {
+  auto decode_rank = [&](int rank) {       // rank: position of the item's tile (pair) in its head's list, longest first
     Item it;
     if (plan != nullptr) {
-      const TileInfo ti = tile_info(plan, tix(lin), 0, N, Nk);
+      const TileInfo ti = tile_info(plan, rank, 0, N, Nk);
       it.seq0 = ti.seq0; it.len = ti.seq_end - ti.seq0; it.qt0 = (ti.row0 - ti.seq0) / C::kBlockM; it.nq = 1;
       it.kseq0 = ti.oseq0; it.klen = ti.oseq_end - ti.oseq0;
     } else {
-      const int pair = CAUSAL ? (n_pairs - 1 - tix(lin)) : tix(lin);
+      const int pair = CAUSAL ? (n_pairs - 1 - rank) : rank;
       it.seq0 = 0; it.len = N; it.qt0 = TPI * pair; it.nq = min(TPI, n_qt - it.qt0);
       it.kseq0 = 0; it.klen = Nk;
     }
@@ -166,6 +162,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     it.n_kt = max(1, (max(kend, 0) + C::kBlockN - 1) / C::kBlockN);
     return it;
   };
+  auto decode = [&](int lin) { return decode_rank(tix(lin)); };
   // query tile t of the item takes part in key step j?  (key tile 0 always, so that every tile has a first step)
   auto active = [&](const Item &it, int t, int j) {
     return t < it.nq && (!CAUSAL || j <= max(0, ((it.qt0 + t) * C::kBlockM + C::kBlockM - 1 + it.off) >> 7));
@@ -212,6 +209,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int bh = hix(lin), tiles = it.nq;
         const int qb = q_buf(ti), use = q_use(ti);
         if (use >= 1) mbar_wait(&bar_q_free[qb], (use - 1) & 1, ab, kFwdWaitQFree);
+        // The softmax warps (168 registers, the kernel's tightest code) take the item's rank and head from here instead
+        // of decoding the item number themselves; the barrier's completion publishes the two words.  The loader is at
+        // most two items ahead of them, the ring has four entries.
+        s_item[ti & 3][0] = tix(lin);
+        s_item[ti & 3][1] = bh;
         mbar_expect_tx(&bar_q_full[qb], tiles * C::kTileBytes);
         for (int t = 0; t < tiles; ++t)
           for (int s = 0; s < C::kSlabs; ++s)
@@ -308,8 +310,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tP = tmem_base + (C::kSepP ? C::kColP + 64 * t : C::kColS + 128 * t) + lane_addr;
     int ti = 0, cnt = 0, turn = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-      const Item it = decode(lin);
-      const int bh = hix(lin), T = it.n_kt;
+      const int qb = q_buf(ti);
+      mbar_wait(&bar_q_full[qb], q_use(ti) & 1, ab, kFwdWaitQ);   // the item's Q has landed, and with it its description
+      const Item it = decode_rank(s_item[ti & 3][0]);
+      const int bh = s_item[ti & 3][1], T = it.n_kt;
       const int qt = it.qt0 + (split ? 0 : t);        // this warpgroup's query tile inside the sequence
       // Masking, reduced to two numbers per tile: column c of key tile j is outside the row's support when
       // 128 j + c > rk, with rk the last key the row sees (causal diagonal and end of the keys, whichever comes first);
@@ -317,13 +321,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int rk = CAUSAL ? min(row + qt * C::kBlockM + it.off, it.klen - 1) : it.klen - 1;
       const int jl = CAUSAL ? max(0, (qt * C::kBlockM + C::kBlockM - 1 + it.off) >> 7) : T;   // last key tile of this query tile
       const int jm = CAUSAL ? min((qt * C::kBlockM + it.off + 1) >> 7, it.klen >> 7) : (it.klen >> 7);
-      // Split mode: stay in step with the item (its Q has landed), so that a warpgroup without key tiles cannot run ahead.
-      const int qb = q_buf(ti);
-      if (split) mbar_wait(&bar_q_full[qb], q_use(ti) & 1, ab, kFwdWaitQ);
       if (!split && t >= it.nq) {
-        // Odd number of query tiles: the last pair has no second tile.  Stay in step with the item (its Q has landed)
-        // before handing back this slot, so that no barrier runs ahead of the roles that wait on it.
-        mbar_wait(&bar_q_full[0], ti & 1, ab, kFwdWaitQ);
+        // Odd number of query tiles: the last pair has no second tile.  This warpgroup is in step with the item (it has
+        // waited for its Q above), so it may hand back the slot without any barrier running ahead of its waiters.
         if (row == 0) mbar_arrive(&bar_q_free[0]);
         mbar_arrive(&bar_o_free[t]);
         continue;

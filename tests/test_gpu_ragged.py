@@ -139,3 +139,27 @@ def test_random_shapes(seed):
     inp = make_inputs(w)
     ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, causal)
     print("shape", B, Hkv * G, Hkv, N, d, causal, check(run_gpu(inp, w.softmax_scale, causal), ex))
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_many_heads_long_causal_matches_chunks_of_heads(d):
+    # 40 heads x 8192 rows stream more than 64 MB of K / V: the kernels then deal groups of adjacent tiles per head (so
+    # that concurrent CTAs share a head's rows in L2) instead of every head's longest tile first.  Scheduling must not
+    # change a single bit of the backward: the same heads run in chunks of 8 (plain longest-first order) give identical
+    # gradients from the same saved O and LSE; the forward, whose tile pairing may differ, agrees to rounding.
+    B, H, N = 1, 40, 8192
+    gen = torch.Generator().manual_seed(4040 + d)
+    Q, K, V, dO = (torch.randn(B, H, N, d, generator=gen).to(torch.bfloat16).cuda() for _ in range(4))
+    alpha = d ** -0.5
+    O, LSE = g.gproj_attn_fwd(Q, K, V, alpha, True)
+    dQ, dK, dV = g.gproj_attn_bwd(Q, K, V, O, LSE, dO, alpha, True)
+    for h0 in range(0, H, 8):
+        sl = slice(h0, h0 + 8)
+        q, k, v, do, o, lse = (t[:, sl].contiguous() for t in (Q, K, V, dO, O, LSE))
+        o2, lse2 = g.gproj_attn_fwd(q, k, v, alpha, True)
+        assert torch.allclose(lse2, lse, rtol=1e-5, atol=1e-5)
+        assert float((o2.float() - o.float()).abs().max()) <= 0.02 * float(o.float().abs().max())
+        dq2, dk2, dv2 = g.gproj_attn_bwd(q, k, v, o, lse, do, alpha, True)
+        assert torch.equal(dq2, dQ[:, sl]) and torch.equal(dk2, dK[:, sl]) and torch.equal(dv2, dV[:, sl]), h0
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, hex(detail)

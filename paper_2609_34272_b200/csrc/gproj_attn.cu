@@ -5,7 +5,9 @@
 #include <cmath>
 #include <cstdint>
 #include <algorithm>
+#include <map>
 #include <mutex>
+#include <tuple>
 #include <vector>
 
 #include "attn_bwd.cuh"
@@ -234,6 +236,15 @@ int tile_group_of(bool packed, bool causal, int heads, int n_per_head, size_t st
   if (heads < 32 || n_per_head < 2 || streamed_bytes <= (size_t(64) << 20)) return 1;
   const long long items = static_cast<long long>(heads) * n_per_head;
   if (items > (1 << 16)) return 8;   // hundreds of items per CTA: any small group balances
+  // the replay costs a fraction of a millisecond of host time: remember the answer for this shape
+  static std::mutex memo_mutex;
+  static std::map<std::tuple<int, int, int, int>, int> memo;
+  const auto key = std::make_tuple(heads, n_per_head, sms, static_cast<int>(item_cost * 100.0));
+  {
+    std::lock_guard<std::mutex> lock(memo_mutex);
+    const auto hit = memo.find(key);
+    if (hit != memo.end()) return hit->second;
+  }
   auto makespan = [&](int k) {
     const long long per_group = static_cast<long long>(heads) * k;
     const int n_full = n_per_head / k;
@@ -245,9 +256,12 @@ int tile_group_of(bool packed, bool causal, int heads, int n_per_head, size_t st
     });
   };
   const double base = makespan(1);
-  for (int k = 16; k >= 2; k /= 2)
-    if (k <= n_per_head && makespan(k) <= 1.01 * base) return k;
-  return 1;
+  int best = 1;
+  for (int k = 16; k >= 2 && best == 1; k /= 2)
+    if (k <= n_per_head && makespan(k) <= 1.01 * base) best = k;
+  std::lock_guard<std::mutex> lock(memo_mutex);
+  if (memo.size() < 4096) memo[key] = best;
+  return best;
 }
 
 // Causal forward at d = 64: paired query tiles or single tiles with the key range split between the warpgroups?
@@ -258,6 +272,14 @@ int tile_group_of(bool packed, bool causal, int heads, int n_per_head, size_t st
 bool fwd_prefers_single_tiles(int BH, int n_qt, int sms) {
   const long long n_pairs = (n_qt + 1) / 2, items_p = BH * n_pairs, items_s = static_cast<long long>(BH) * n_qt;
   if (items_s > (1 << 16)) return false;   // many items per SM: both deals balance, pairs have the lower per-item cost
+  static std::mutex memo_mutex;
+  static std::map<std::tuple<int, int, int>, bool> memo;
+  const auto key = std::make_tuple(BH, n_qt, sms);
+  {
+    std::lock_guard<std::mutex> lock(memo_mutex);
+    const auto hit = memo.find(key);
+    if (hit != memo.end()) return hit->second;
+  }
   auto longest = [&](long long items, auto work_of) {
     const int G = static_cast<int>(std::min<long long>(items, sms));
     std::vector<double> load(static_cast<size_t>(G), 0.0);
@@ -276,6 +298,8 @@ bool fwd_prefers_single_tiles(int BH, int n_qt, int sms) {
     const long long t = n_qt - 1 - lin / BH;
     return kSplitStep * 0.5 * static_cast<double>(t + 1) + kItem;
   });
+  std::lock_guard<std::mutex> lock(memo_mutex);
+  if (memo.size() < 4096) memo[key] = t_single < t_pairs;
   return t_single < t_pairs;
 }
 

@@ -715,7 +715,13 @@ int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const v
          cudaStreamWaitEvent(s_out, st->ev_start, 0) == cudaSuccess;
   }
   const size_t row_bytes = static_cast<size_t>(N) * d * 2;           // one head of one tensor
-  auto slab_begin = [&](int c) { return static_cast<int>(static_cast<long long>(kv_heads) * c / slabs); };
+  // The last slab is half as large as the others: what stays exposed at the end of the call is that slab's kernels and
+  // its copy-out, everything before hides behind the inbound copies.
+  auto slab_begin = [&](int c) {
+    if (c >= slabs) return kv_heads;
+    if (slabs == 1 || kv_heads < 2 * slabs) return static_cast<int>(static_cast<long long>(kv_heads) * c / slabs);
+    return static_cast<int>((2LL * kv_heads * c + (2 * slabs - 1) / 2) / (2 * slabs - 1));
+  };
   for (int c = 0; ok && c < slabs; ++c) {
     const size_t k0 = slab_begin(c), kn = slab_begin(c + 1) - k0, q0 = k0 * G, qn = kn * G;
     ok = cudaMemcpyAsync(dQin + q0 * row_bytes, static_cast<const uint8_t *>(Q) + q0 * row_bytes, qn * row_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&

@@ -113,7 +113,7 @@ __device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, const 
 }
 
 // ------------------------------------------------------------------------------------------
-// TMA: 2-D tiled load global -> shared, completion on an mbarrier (no multicast anywhere)
+// TMA: 2-D tiled load global -> shared, completion on an mbarrier
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

@@ -109,17 +109,30 @@ struct TileSched {
 // group = 1: every head's longest tile first (the exact longest-first order; packed calls, whose plan is already
 // sorted); group = tiles per head: head-major (dense non-causal calls, whose tiles are all alike); in between for
 // causal calls with many heads, where a few adjacent ranks differ little in work.
-struct ItemOrder {
-  int gk, per_group, n_full, rem;   // ranks per group, items per group (heads x gk), full groups, ranks of the short last group
+// Division of a non-negative 31-bit number by a divisor fixed at launch: quotient = umulhi(x, mul) >> shr (x itself if
+// the divisor is 1), with L = ceil(log2 divisor), mul = ceil(2^(31 + L) / divisor) < 2^32 and shr = L - 1, set by the
+// host.  Three instructions instead of the forty-odd of a division by a run-time value, which sat on every role's path
+// at each tile.
+struct FastDiv {
+  unsigned div, mul, shr;
 #ifdef __CUDACC__
-  __device__ __forceinline__ int rank(int lin) const {
-    const int g = lin / per_group, within = lin - g * per_group;
-    return g * gk + within % ((g < n_full) ? gk : rem);
+  __device__ __forceinline__ int quot(int x) const {
+    return div == 1u ? x : static_cast<int>(__umulhi(static_cast<unsigned>(x), mul) >> shr);
   }
-  __device__ __forceinline__ int head(int lin) const {
-    const int g = lin / per_group, within = lin - g * per_group;
-    return within / ((g < n_full) ? gk : rem);
+#endif
+};
+struct ItemOrder {
+  int gk, n_full;                   // ranks per group, full groups
+  FastDiv per_group, by_gk, by_rem; // items per group (heads x gk); ranks per group; ranks of the short last group
+#ifdef __CUDACC__
+  __device__ __forceinline__ void decode(int lin, int &rank, int &head) const {
+    const int g = per_group.quot(lin), within = lin - g * static_cast<int>(per_group.div);
+    const bool full = g < n_full;
+    head = full ? by_gk.quot(within) : by_rem.quot(within);
+    rank = g * gk + within - head * static_cast<int>(full ? by_gk.div : by_rem.div);
   }
+  __device__ __forceinline__ int rank(int lin) const { int r, h; decode(lin, r, h); return r; }
+  __device__ __forceinline__ int head(int lin) const { int r, h; decode(lin, r, h); return h; }
 #endif
 };
 

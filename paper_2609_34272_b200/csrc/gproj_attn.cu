@@ -202,12 +202,28 @@ int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, floa
 namespace {
 
 // The kernels' item order for `heads` heads of n_per_head tiles dealt in groups of `group` ranks (clamped to 1 .. n_per_head).
+FastDiv fast_div(unsigned d) {
+  FastDiv f;
+  f.div = d;
+  f.mul = 0;
+  f.shr = 0;
+  if (d > 1) {
+    unsigned lg = 0;
+    while ((1ull << lg) < d) ++lg;                       // ceil(log2 d)
+    const unsigned p = 31 + lg;
+    f.mul = static_cast<unsigned>(((1ull << p) + d - 1) / d);
+    f.shr = p - 32;
+  }
+  return f;
+}
+
 ItemOrder item_order(int heads, int n_per_head, int group) {
   ItemOrder o;
   o.gk = std::max(1, std::min(group, n_per_head));
-  o.per_group = heads * o.gk;
   o.n_full = n_per_head / o.gk;
-  o.rem = std::max(1, n_per_head - o.n_full * o.gk);
+  o.per_group = fast_div(static_cast<unsigned>(heads) * static_cast<unsigned>(o.gk));
+  o.by_gk = fast_div(static_cast<unsigned>(o.gk));
+  o.by_rem = fast_div(static_cast<unsigned>(std::max(1, n_per_head - o.n_full * o.gk)));
   return o;
 }
 

@@ -34,7 +34,7 @@ struct BwdW128 {
   static constexpr int kTileBytes = 128 * 128;                     // 128 rows x 64 BF16: one 128-byte-row slab
   static constexpr int kStepRows = 128;
   static constexpr int kStages = 3;
-  static constexpr int kWG = 4, kCompute = 128 * kWG, kThreads = 128 + kCompute;
+  static constexpr int kWG = 4, kCompute = 128 * kWG, kThreads = 96 + kCompute;   // warp 0: stage producer (lane 0) and tile loader (lane 1); warps 1, 2: MMA issuers; 16 compute warps
   static constexpr int kSliceCols = kStepRows / kWG;               // 32 columns per thread and step
   static constexpr uint32_t kColX = 0, kColY = 128, kColZ = 256, kColAcc0 = 384, kColAcc1 = 448;
   static constexpr int kTmemCols = 512;
@@ -190,10 +190,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         for (int q = (g > S ? g - S : 0); q < g; ++q)
           for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full[q % S], (q / S) & 1); ++spin) {}
       }
-    }
-  } else if (warp == 3) {
-    // ---------------------------------------------------------------- TMA loader of the stationary (K, V) tiles
-    if (lane == 0) {
+    } else if (lane == 1) {
+      // -------------------------------------------------------------- TMA loader of the stationary (K, V) tiles (second lane of
+      // the producer's warp: the two single-thread roles share a warp, which leaves 608 threads and 104 registers each)
       int ti = 0;
       for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
         const int bh = hix(lin), krow0 = tile_of(lin).row0;
@@ -287,7 +286,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     drain_mmas_if_aborted(&bar_drain[1], ab);
   } else {
     // ---------------------------------------------------------------- compute: thread <-> (key row, 32-query slice of every step)
-    const int wg = (warp - 4) >> 2;
+    const int wg = (warp - 3) >> 2;
     const int row = 32 * (warp & 3) + lane;                  // key row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
     const uint32_t slice_addr = tmem_base + lane_addr + C::kSliceCols * wg;
@@ -335,7 +334,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&bar_acc_free);          // the accumulators may be overwritten by the next tile
-      if (threadIdx.x == 128) bulk_wait_group_read0();   // the previous tile's stores have left the staging buffer
+      if (threadIdx.x == 96) bulk_wait_group_read0();   // the previous tile's stores have left the staging buffer
       named_bar_sync(1, C::kCompute);
 #pragma unroll
       for (int v = 0; v < 2; ++v) {
@@ -353,7 +352,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       fence_proxy_async_smem();
       named_bar_sync(1, C::kCompute);
       if (tile_store_by_tma(tl, N)) {
-        if (threadIdx.x == 128) {
+        if (threadIdx.x == 96) {
           tma_store_3d(&tmdV, stage_dv, 0, tl.row0, bh);
           tma_store_3d(&tmdK, stage_dk, 0, tl.row0, bh);
           bulk_commit_group();
@@ -366,7 +365,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       }
       g0 += T;
     }
-    if (threadIdx.x == 128) bulk_wait_group_read0();
+    if (threadIdx.x == 96) bulk_wait_group_read0();
   }
 
   tc_fence_before();

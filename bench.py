@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 METRIC = "fused attn bwd TFLOP/s & % BF16 tensor peak; dQ/dK/dV rel-L2 vs FP64"
 UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised under profiles/
-NCU_DRAM_BYTES_PER_LAUNCH = {("bwd_dkv_kernel", 2): 42.515e6 + 0.896e6, ("bwd_dkv_kernel", 3): 42.252e6 + 0.861e6,
+NCU_DRAM_BYTES_PER_LAUNCH = {("bwd_dkv_kernel", 2): 42.519e6 + 0.696e6, ("bwd_dkv_kernel", 3): 42.252e6 + 0.861e6,
                              ("bwd_dkv_kernel", 4): 1351.866e6 + 516.820e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 

@@ -9,11 +9,10 @@ import torch
 import oracle
 import paper_2609_34272_b200 as g
 from oracle import emulation as em
+from helpers import load_values, witness128_arrays
 from paper_2609_34272_b200.workloads import Workload, bits, from_bits, make_inputs
 
 pytestmark = pytest.mark.gpu
-
-GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "witness_minus24.txt")
 
 
 def fwd_bwd(Q, K, V, dO, alpha, causal, flags=0):
@@ -28,41 +27,112 @@ def fwd_bwd(Q, K, V, dO, alpha, causal, flags=0):
 def witness_problem():
     """The four-key -24 witness embedded in a 128 x 128, d = 64 non-causal problem.
 
-    Every query is (0, 0, 256, 0, ...); keys 0..3 are the witness keys (third coordinate 0); the other
-    124 keys are (0, 0, -256, 0, ...), whose logits -8192 give probability exactly 0 in FP32 and FP64.
-    Every row therefore reproduces the witness (Appendix A, "An exact -24 witness").
+    Every query is (0, 0, 256, c, 0, ...); keys 0..3 are the witness keys (third and fourth coordinate 0); the
+    other 124 keys are (0, 0, -256, 0, ...), whose logits -8192 give probability exactly 0 in FP32 and FP64.
+    Every row therefore reproduces the witness (Appendix A, "An exact -24 witness"), and the third and fourth
+    query coordinates make the key-side correction visible in dK (tests/golden/witness128_key_pass.txt).
     """
-    vals = {}
-    for line in open(GOLDEN):
-        line = line.split("#", 1)[0].strip()
-        if line:
-            key, *rest = line.split()
-            vals[key] = [float(x) for x in rest]
+    vals = load_values("witness_minus24.txt")
     N, d = 128, 64
-    Q = np.zeros((N, d)); K = np.zeros((N, d)); V = np.zeros((N, d)); U = np.zeros((N, d))
-    Q[:, 2] = 256.0
-    K[4:, 2] = -256.0
-    for j in range(4):
-        K[j, :2] = vals[f"k{j + 1}"]
-        V[j, :2] = vals[f"v{j + 1}"]
-    U[:, :2] = vals["u"]
-    tens = [from_bits(em.f64_to_bf16_bits(x)).reshape(1, 1, N, d) for x in (Q, K, V, U)]
+    tens = [from_bits(em.f64_to_bf16_bits(x)).reshape(1, 1, N, d) for x in witness128_arrays()]
     return tens, vals
 
 
 def test_minus24_witness_on_gpu():
     (Q, K, V, U), vals = witness_problem()
-    alpha = vals["alpha"][0]
+    hand = load_values("witness128_key_pass.txt")
+    alpha = float(vals["alpha"][0])
     O, LSE, dQ, dK, dV = fwd_bwd(Q, K, V, U, alpha, False)
     assert torch.all(O[0, 0, :, 0].float() == vals["o"][0]) and torch.all(O[0, 0, :, 1].float() == vals["o"][1])
     assert torch.all(dQ[0, 0, :, 0].float() == vals["dq0_gproj"][0])                    # exactly zero with GProj
-    _, _, dQ_off, _, _ = fwd_bwd(Q, K, V, U, alpha, False, flags=g.FLAG_NO_Q_CORRECTION)
+    _, _, dQ_off, dK_noq, _ = fwd_bwd(Q, K, V, U, alpha, False, flags=g.FLAG_NO_Q_CORRECTION)
     assert torch.all(dQ_off[0, 0, :, 0].float() == vals["dq0_uncorrected"][0])          # -24 without it
     # the remaining coordinates agree with the rounding model of Algorithm 1
     q, k, v, u = (bits(t)[0, 0] for t in (Q, K, V, U))
     model = em.emulate_head(q, k, v, u, alpha, causal=False)
     assert np.array_equal(dQ[0, 0].float().cpu().numpy(), model["dQ"])
     assert np.array_equal(dV[0, 0].float().cpu().numpy(), model["dV"])
+    # key pass (Algorithm 1 lines 15-18): the hand-derived values, with and without the correction
+    dK_np = dK[0, 0].float().cpu().numpy()
+    assert np.array_equal(dK_np, model["dK"])
+    assert np.array_equal(dK_np[:4, 2], hand["dk2_gproj"]) and np.array_equal(dK_np[:4, 3], hand["dk3_gproj"])
+    assert torch.equal(dK_noq, dK)
+    _, _, dQ_nok, dK_nok, dV_nok = fwd_bwd(Q, K, V, U, alpha, False, flags=g.FLAG_NO_K_CORRECTION)
+    dK_nok = dK_nok[0, 0].float().cpu().numpy()
+    assert np.array_equal(dK_nok[:4, 2], hand["dk2_uncorrected"]) and np.array_equal(dK_nok[:4, 3], hand["dk3_uncorrected"])
+    assert torch.equal(dQ_nok, dQ) and torch.equal(dV_nok, dV)
+    rest = dK_np.copy(); rest[:4, 2:4] = 0
+    assert not rest.any()
+    assert np.all(dV[0, 0, :4, :2].float().cpu().numpy() == hand["dv01"])
+
+
+def three_key_problem(name):
+    """A hand-worked three-key case of tests/golden, zero-padded from d = 4 to d = 64 (N = 3: one ragged tile)."""
+    hand = load_values(name)
+    rows = lambda stem: np.array([hand[f"{stem}{j}"] for j in (1, 2, 3)])
+    Qs = rows("q") if "q1" in hand else np.tile(hand["q"], (3, 1))
+    pad = lambda x: np.concatenate([x, np.zeros((3, 60))], axis=1)
+    tens = [from_bits(em.f64_to_bf16_bits(pad(x))).reshape(1, 1, 3, 64) for x in (Qs, rows("k"), rows("v"), rows("u"))]
+    return tens, hand
+
+
+def test_three_key_operand_mass_on_gpu():
+    # lambda = rho / m with m = 513/512 (Algorithm 1 line 14): hand values of tests/golden/three_key_mass.txt
+    (Q, K, V, U), hand = three_key_problem("three_key_mass.txt")
+    alpha = float(hand["alpha"][0])
+    O, LSE, dQ, dK, dV = fwd_bwd(Q, K, V, U, alpha, False)
+    dQ, dK, dV = (x[0, 0].float().cpu().numpy() for x in (dQ, dK, dV))
+    assert np.all(np.abs(dQ[:, 0]) <= 1e-6)               # one FP32 rounding of lambda away from 0 (0.046875 with lambda = rho)
+    assert np.all(dQ[:, 1] == hand["dq1"][0])
+    assert np.array_equal(dK[:, 2], hand["dk2_gproj"])
+    assert np.all(dV[:, 3] == hand["dv3"][0]) and np.all(dV[:, :2] == hand["dv01"])
+    _, _, _, dK_nok, _ = fwd_bwd(Q, K, V, U, alpha, False, flags=g.FLAG_NO_K_CORRECTION)
+    assert np.array_equal(dK_nok[0, 0, :, 2].float().cpu().numpy(), hand["dk2_uncorrected"])
+
+
+def test_three_key_saved_output_on_gpu():
+    # D from the saved BF16 output, dV and the key correction from the rounded probabilities
+    # (Algorithm 1 lines 1, 6, 16-17): hand values of tests/golden/three_key_saved_output.txt
+    (Q, K, V, U), hand = three_key_problem("three_key_saved_output.txt")
+    alpha = float(hand["alpha"][0])
+    O, LSE, dQ, dK, dV = fwd_bwd(Q, K, V, U, alpha, False)
+    assert torch.all(O[0, 0, :, 0].float() == hand["o0"][0])
+    dQ, dK, dV = (x[0, 0].float().cpu().numpy() for x in (dQ, dK, dV))
+    assert np.all(np.abs(dQ[:, 0]) <= 1e-6) and np.all(dQ[:, 1] == hand["dq1"][0])
+    assert np.array_equal(dK[:, 3], hand["dk3_gproj"])
+    assert np.all(dV[:, 3] == hand["dv3"][0]) and np.all(dV[:, 0] == hand["dv0"][0])
+    _, _, _, dK_nok, _ = fwd_bwd(Q, K, V, U, alpha, False, flags=g.FLAG_NO_K_CORRECTION)
+    assert np.array_equal(dK_nok[0, 0, :, 3].float().cpu().numpy(), hand["dk3_uncorrected"])
+
+
+def sink_problem(N, d, seed, common_query, sink_norm):
+    """Late-training-like inputs: every query carries a large common component and key 0 is aligned with it, so
+    most rows put nearly all their probability on key 0 (an attention sink).  Input construction only."""
+    gen = torch.Generator().manual_seed(seed)
+    Q, K, V, U = (torch.randn(N, d, generator=gen) for _ in range(4))
+    c = torch.randn(d, generator=gen); c = c / c.norm()
+    Q = Q + common_query * c
+    K[0] = 0.1 * K[0] + sink_norm * c
+    return [x.to(torch.bfloat16).reshape(1, 1, N, d) for x in (Q, K, V, U)]
+
+
+@pytest.mark.parametrize("d,common_query,sink_norm", [(64, 8.0, 16.0), (64, 32.0, 4.0), (128, 12.0, 16.0)])
+def test_key_pass_is_material_with_an_attention_sink(d, common_query, sink_norm):
+    # The regime in which the paper's per-capture table shows the key pass mattering (dK error falling by more
+    # than an order of magnitude): the leaked row mass of every row lands on the one key all rows select, times the
+    # common query component.  Against the exact FP64 VJP: GProj dK at the BF16 floor, without the key pass >= 10x worse.
+    N = 512
+    Q, K, V, U = sink_problem(N, d, 4242 + d, common_query, sink_norm)
+    alpha = float(np.float32(1 / math.sqrt(d)))
+    ex = oracle.attn_fwd_bwd_f64(bits(Q), bits(K), bits(V), bits(U), alpha, True)
+    on = fwd_bwd(Q, K, V, U, alpha, True)
+    no_k = fwd_bwd(Q, K, V, U, alpha, True, flags=g.FLAG_NO_K_CORRECTION)
+    err = lambda t, n: oracle.rel_l2_percent(t.float().cpu().numpy(), ex[n])
+    e_on = {n: err(t, n) for n, t in zip(("O", "dQ", "dK", "dV"), (on[0], on[2], on[3], on[4]))}
+    e_nok = err(no_k[3], "dK")
+    print("sink regime d=%d: GProj %s, dK without the key pass %.2f %%" % (d, {k: round(v, 3) for k, v in e_on.items()}, e_nok))
+    assert all(v <= 1.0 for v in e_on.values()), e_on
+    assert e_nok >= 10 * e_on["dK"], (e_nok, e_on)
 
 
 @pytest.mark.parametrize("d", [64, 128])

@@ -9,7 +9,7 @@ import torch
 
 import oracle
 from oracle import emulation as em
-from helpers import as_bits, randn_bf16
+from helpers import as_bits, load_values, randn_bf16, witness128_arrays
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "witness_minus24.txt")
 
@@ -134,3 +134,77 @@ def test_emulation_tracks_exact_vjp_and_correction_helps(causal):
     assert np.array_equal(only_q["dV"], on["dV"]) and np.array_equal(off["dV"], on["dV"])
     # operand mass stays near one (Appendix "Synthetic Numerical Suite", "Operand masses")
     assert np.all(on["m"] > 0) and np.abs(on["m"] - 1).max() < 0.01
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Hand-derived pins of the key pass, of lambda with m != 1, of D from the saved output and of dV from r.
+# The expected values live in tests/golden/*.txt with their derivations; none was produced by the model under test.
+
+def test_key_pass_on_the_128_row_witness():
+    # Algorithm 1 lines 15-18, Eq. "gproj-key-implemented": dK = BF16(alpha (t^T Q - r^T z)), z = BF16(lambda q).
+    gold = load_golden()
+    hand = load_values("witness128_key_pass.txt")
+    q, k, v, u = (em.f64_to_bf16_bits(x) for x in witness128_arrays())
+    alpha = float(gold["alpha"][0])
+    on = em.emulate_head(q, k, v, u, alpha, causal=False)
+    only_q = em.emulate_head(q, k, v, u, alpha, causal=False, correct_k=False)
+    off = em.emulate_head(q, k, v, u, alpha, causal=False, correct_q=False, correct_k=False)
+    assert np.all(on["m"] == 1.0) and np.all(on["rho"] == gold["rho"][0]) and np.all(on["lam"] == gold["rho"][0])
+    assert np.array_equal(on["dK"][:4, 2], hand["dk2_gproj"])
+    assert np.array_equal(only_q["dK"][:4, 2], hand["dk2_uncorrected"])
+    assert np.array_equal(off["dK"][:4, 2], hand["dk2_uncorrected"])
+    assert np.all(on["dK"][:4, 3] == hand["dk3_gproj"]) and np.array_equal(only_q["dK"][:4, 3], hand["dk3_uncorrected"])
+    rest = on["dK"].copy(); rest[:4, 2:4] = 0
+    assert not rest.any()
+    assert np.all(on["dV"][:4, :2] == hand["dv01"]) and not on["dV"][4:].any() and not on["dV"][:, 2:].any()
+    assert np.all(on["dQ"][:, 0] == 0.0) and np.all(off["dQ"][:, 0] == -24.0)
+    ex = oracle.attn_fwd_bwd_f64(q[None, None], k[None, None], v[None, None], u[None, None], alpha, False)
+    assert np.allclose(ex["dK"][0, 0, :4, 2], hand["dk2_exact"], rtol=0, atol=1e-9)
+    assert np.allclose(ex["dK"][0, 0, :4, 3], hand["dk3_exact"], rtol=0, atol=1e-9)
+
+
+def small_case_inputs(vals, n=3):
+    rows = lambda stem: np.array([vals[f"{stem}{j}"] for j in range(1, n + 1)])
+    Q = rows("q") if "q1" in vals else np.tile(vals["q"], (n, 1))
+    return tuple(em.f64_to_bf16_bits(x) for x in (Q, rows("k"), rows("v"), rows("u")))
+
+
+def test_lambda_divides_by_the_operand_mass():
+    # Algorithm 1 line 14 / Eq. "gproj-row-mass": lambda = rho / m with m the sum of the ROUNDED probabilities
+    # (three keys at BF16(1/3): m = 513/512); lambda = rho would leave the mass rho (1 - m) on the mean key.
+    hand = load_values("three_key_mass.txt")
+    q, k, v, u = small_case_inputs(hand)
+    alpha = float(hand["alpha"][0])
+    on = em.emulate_head(q, k, v, u, alpha, causal=False)
+    only_q = em.emulate_head(q, k, v, u, alpha, causal=False, correct_k=False)
+    assert np.all(on["r"] == hand["r"][0]) and np.all(on["m"] == hand["m"][0])
+    assert np.array_equal(on["t"], np.tile(hand["t"], (3, 1))) and np.all(on["rho"] == hand["rho"][0])
+    assert np.all(on["D"] == 0.0)
+    assert np.all(on["lam"] == hand["lam"][0])
+    assert np.all(on["dQ"][:, 0] == hand["dq0"][0])
+    assert np.all(on["dQ"][:, 1] == hand["dq1"][0])
+    assert np.array_equal(on["dK"][:, 2], hand["dk2_gproj"])
+    assert np.array_equal(only_q["dK"][:, 2], hand["dk2_uncorrected"])
+    assert np.all(on["dV"][:, 3] == hand["dv3"][0])
+    assert np.all(on["dV"][:, :2] == hand["dv01"])
+
+
+def test_row_term_comes_from_the_saved_bf16_output_and_operands_are_the_rounded_probabilities():
+    # Algorithm 1 line 1 / Eq. "main-delta": D = rowsum(dO * BF16(o)); line 6: dV += r^T dO with r = BF16(P);
+    # lines 16-17: the key correction contracts the rounded probabilities with z = BF16(lambda q).
+    hand = load_values("three_key_saved_output.txt")
+    q, k, v, u = small_case_inputs(hand)
+    alpha = float(hand["alpha"][0])
+    on = em.emulate_head(q, k, v, u, alpha, causal=False)
+    only_q = em.emulate_head(q, k, v, u, alpha, causal=False, correct_k=False)
+    assert np.all(on["O"][:, 0] == hand["o0"][0])
+    assert np.all(on["D"] == hand["D"][0])
+    assert np.array_equal(on["t"], np.tile(hand["t"], (3, 1))) and np.all(on["rho"] == hand["rho"][0])
+    assert np.all(on["r"] == hand["r"][0]) and np.all(on["lam"] == hand["lam"][0])
+    assert np.all(on["dQ"][:, 0] == hand["dq0"][0]) and np.all(on["dQ"][:, 1] == hand["dq1"][0])
+    assert np.array_equal(on["dK"][:, 3], hand["dk3_gproj"])
+    assert np.array_equal(only_q["dK"][:, 3], hand["dk3_uncorrected"])
+    assert np.all(on["dV"][:, 3] == hand["dv3"][0]) and np.all(on["dV"][:, 0] == hand["dv0"][0])
+    # the model's exact-D switch reproduces the alternative worked out beside the golden values
+    ideal = em.emulate_head(q, k, v, u, alpha, causal=False, exact_D=True)
+    assert np.all(ideal["rho"] == -0.22265625) and np.all(ideal["dQ"][:, 1] == -10.6875)

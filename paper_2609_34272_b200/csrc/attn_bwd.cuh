@@ -509,6 +509,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       const int bh = hix(lin), T = steps_of(tl), rb = ti % R;
       const size_t head_row0 = static_cast<size_t>(bh) * N;
       const int qrow = tl.row0 + row;                  // this thread's query row within the head (past seq_end in a ragged tile)
+#ifdef GPROJ_TRACE
+      const unsigned long long ev_n0 = global_ns(); const long long ev_c0 = clock64(); unsigned long long ev_n1 = 0, ev_n2 = 0;
+#endif
 
       // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1): each of the 16 compute warps
       // takes eight rows, 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
@@ -559,6 +562,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
 
       uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);
+#ifdef GPROJ_TRACE
+      ev_n1 = global_ns();
+#endif
       for (int n = (grp - g0 % C::kGroups + C::kGroups) % C::kGroups; n < T; n += C::kGroups) {
         const int g = g0 + n, b = g % NB;
         mbar_wait(&bar_sdp_full[b], (g / NB) & 1, ab, kDqWaitSdP);
@@ -580,6 +586,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         mbar_arrive(&bar_tr_ready[b]);
       }
 
+#ifdef GPROJ_TRACE
+      ev_n2 = global_ns();
+#endif
       if (C::kPrefetchO) {
         // every thread took its D and LSE out of shared memory before its first step (behind the barrier above), and dO of
         // the next tile sits in the other stationary buffer: the next tile's rows may travel during this tile's epilogue
@@ -663,6 +672,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
         named_bar_sync(1, C::kCompute);
         if (threadIdx.x == 128) mbar_arrive(&bar_res_free[rb]);
       }
+#ifdef GPROJ_TRACE
+      if ((threadIdx.x & 127) == 0) tile_event(1 + wg, lin, T, ev_n0, ev_n1, ev_n2, global_ns(), ev_c0, clock64());
+#endif
       g0 += T;
     }
     if (threadIdx.x == 128) bulk_wait_group_read0();

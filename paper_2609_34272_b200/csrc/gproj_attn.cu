@@ -860,6 +860,17 @@ int gproj_debug_read_tile_trace(unsigned long long *out, int max_records, int re
   if (reset) { const int zero = 0; cudaMemcpyToSymbol(gproj::g_tile_trace_count, &zero, sizeof(int)); }
   return n;
 }
+int gproj_debug_read_tile_events(unsigned long long *out, int max_records, int reset) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return GPROJ_ERR_CUDA;
+  int n = 0;
+  if (cudaMemcpyFromSymbol(&n, gproj::g_tile_ev_count, sizeof(int)) != cudaSuccess) return GPROJ_ERR_CUDA;
+  if (n > gproj::kTileEvMax) n = gproj::kTileEvMax;
+  if (n > max_records) n = max_records;
+  if (n > 0 && cudaMemcpyFromSymbol(out, gproj::g_tile_ev, static_cast<size_t>(n) * 8 * sizeof(unsigned long long)) != cudaSuccess)
+    return GPROJ_ERR_CUDA;
+  if (reset) { const int zero = 0; cudaMemcpyToSymbol(gproj::g_tile_ev_count, &zero, sizeof(int)); }
+  return n;
+}
 // Debug builds only: copy the phase stamps of CTA 0 to the host (after a device synchronize).
 int gproj_debug_read_trace(long long *out, int count) {
   if (cudaDeviceSynchronize() != cudaSuccess) return GPROJ_ERR_CUDA;

@@ -44,6 +44,21 @@ __device__ __forceinline__ void tile_trace(int tile, unsigned long long t0, unsi
     g_tile_trace[4 * i] = blockIdx.x; g_tile_trace[4 * i + 1] = tile; g_tile_trace[4 * i + 2] = t0; g_tile_trace[4 * i + 3] = t1;
   }
 }
+// richer per-tile record: {kernel << 32 | cta, steps << 32 | tile, ns at tile start, at first step, after last step, at tile end,
+// clock64 at tile start, at tile end}
+constexpr int kTileEvMax = 8192;
+__device__ unsigned long long g_tile_ev[kTileEvMax * 8];
+__device__ int g_tile_ev_count;
+__device__ __forceinline__ void tile_event(int kernel, int tile, int steps, unsigned long long n0, unsigned long long n1,
+                                           unsigned long long n2, unsigned long long n3, long long c0, long long c1) {
+  const int i = atomicAdd(&g_tile_ev_count, 1);
+  if (i < kTileEvMax) {
+    unsigned long long *e = g_tile_ev + 8 * i;
+    e[0] = (static_cast<unsigned long long>(kernel) << 32) | blockIdx.x;
+    e[1] = (static_cast<unsigned long long>(steps) << 32) | static_cast<unsigned>(tile);
+    e[2] = n0; e[3] = n1; e[4] = n2; e[5] = n3; e[6] = c0; e[7] = c1;
+  }
+}
 #else
 __device__ __forceinline__ void trace_stamp(int, int, int) {}
 #endif

@@ -8,8 +8,9 @@
  *   - LSE is a DEVICE pointer to FP32 [B][H][N]: the natural-log sum-exp of the scaled scores
  *     s_ij = softmax_scale * q_i . k_j over the row's support.
  *   - Supported shapes: d in {64, 128}; any N >= 1 (tiles of 128 rows; a ragged last tile is zero-filled on load,
- *     masked where it would enter a row statistic and clipped on store); B, H >= 1 with B*H*N < 2^31; N_q = N_k = N;
- *     causal != 0 means row i attends to j <= i.  The *_gqa entry points take separate query / KV head counts, the
+ *     masked where it would enter a row statistic and clipped on store); B, H >= 1 with B*H*N < 2^31, B*H < 2^20 and
+ *     N <= 2^24 (packed calls: fewer than 2^24 query tiles and key tiles); anything else is GPROJ_ERR_SHAPE;
+ *     N_q = N_k = N; causal != 0 means row i attends to j <= i.  The *_gqa entry points take separate query / KV head counts, the
  *     *_rect entry points separate query / key lengths.
  *   - The caller owns all memory.  The library never allocates device memory, frees or synchronises; work is
  *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).  (The host-buffer entry point
@@ -34,7 +35,8 @@ extern "C" {
 typedef enum gproj_status {
   GPROJ_OK = 0,
   GPROJ_ERR_NULL = -1,      /* a required pointer is NULL */
-  GPROJ_ERR_SHAPE = -2,     /* unsupported d, non-positive dimension, H not a multiple of Hkv, size overflow */
+  GPROJ_ERR_SHAPE = -2,     /* unsupported d, non-positive dimension, H not a multiple of Hkv, or a size limit
+                               (B*H*N >= 2^31, B*H >= 2^20, N > 2^24, 2^24 or more tiles in a packed call) */
   GPROJ_ERR_ALIGN = -3,     /* a tensor base address is not 16-byte aligned */
   GPROJ_ERR_WORKSPACE = -4, /* workspace NULL, misaligned or smaller than gproj_attn_bwd_workspace_bytes() */
   GPROJ_ERR_SCALE = -5,     /* softmax_scale not finite or not > 0 */
@@ -57,8 +59,13 @@ typedef enum gproj_status {
  * Forward: O = softmax(softmax_scale * Q K^T [causal]) V and the row log-sum-exp.
  * Follows Eq. "row-attention" (Section 3.1) with the subtract-before-scale softmax of
  * Eq. "gproj-forward" (Appendix "Implemented Arithmetic and Rounding", "Forward and saved state"):
- * the unscaled row maximum is subtracted with its own FP32 rounding before the scale and the
+ * the unscaled maximum is subtracted with its own FP32 rounding before the scale and the
  * base-two exponential; the value product uses BF16 probabilities, the normaliser their FP32 values.
+ * One deviation from the literal equation: the subtracted value is a LAZY running maximum.  Key tiles are taken in
+ * order; the reference m is the true maximum of the first tile and is raised to the running maximum only when a later
+ * tile exceeds it by more than 8 in the base-two exponent domain (alpha log2 e (x_max - m) > 8).  So m <= x_max < m +
+ * 8 / (alpha log2 e) and z can reach 2^8 instead of at most 1; O = (sum z v) / (sum z) and LSE = alpha m + ln(sum z) do not
+ * depend on the reference, and a row with a single key still has z = 1 exactly (o_0 = v_0 bitwise).
  *   in : Q, K, V  (device, BF16)        out: O (device, BF16), LSE (device, FP32)
  */
 int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE,
@@ -109,8 +116,9 @@ int gproj_attn_bwd_gqa(const void *Q, const void *K, const void *V, const void *
  * Forward with options (fwd_flags = 0 is gproj_attn_fwd_gqa).  GPROJ_FWD_FLAG_FMA_SOFTMAX selects the native fused form
  * of the softmax exponent, z = exp2(fma(x, a, -fl32(x_max a))) with a = softmax_scale * log2 e (Eq. "historical-fma",
  * Appendix "The source of the saved-output error"): x a is not rounded on its own, so the largest score of a row need
- * not map to exactly zero and a one-key row can return o_0 != v_0.  It exists to reproduce the paper's "FA3" forward
- * next to the subtract-before-scale one on the same kernels; training code should leave it off.
+ * not map to exactly zero and a one-key row can return o_0 != v_0.  With this flag x_max is always the true running
+ * maximum (no lazy rule).  It exists to reproduce the paper's "FA3" forward next to the subtract-before-scale one on
+ * the same kernels; training code should leave it off.
  */
 #define GPROJ_FWD_FLAG_FMA_SOFTMAX 1u
 int gproj_attn_fwd_ex(const void *Q, const void *K, const void *V, void *O, float *LSE,
@@ -204,6 +212,8 @@ int gproj_attn_bwd_varlen_qk(const void *Q, const void *K, const void *V, const 
  *     the first pipelined call on a device creates the two streams and 34 events, which live until the process exits.
  *   - flags: those of gproj_attn_bwd without the ONLY_* bits (GPROJ_ERR_FLAGS for those).
  *   - Calls from several host threads on one device are serialised while they enqueue.
+ *   - If the call returns an error after it has begun to enqueue work, `stream` has been made to wait for everything
+ *     the call queued on its internal streams, so synchronising `stream` is enough before the host buffers are reused.
  */
 size_t gproj_attn_host_staging_bytes(int B, int H, int Hkv, int N, int d);
 int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const void *dO, void *O, float *LSE,
@@ -223,9 +233,11 @@ int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const v
  *     GPROJ_ERR_WORKSPACE (problems up to about 7.5 Mi elements B*H*N*d at d = 64 fit, e.g. B*H = 16, N = 4096); nothing is launched.
  *   - The first call on each device looks up the array's device address (with that device current); make
  *     that first call before any stream capture begins.  No call allocates or frees anything.
- *   - All calls on a device share the one array, and it keeps whatever the last call left there.  Nothing
- *     in it has to start at zero (the first kernel writes every word the second one reads), but two calls
- *     that overlap on the GPU (different streams, no dependency) race on it: serialise them.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left there, possibly from
+ *     another shape.  Nothing in it has to start at zero: the first kernel writes every word whose value the second
+ *     one uses; the few words the second kernel reads beyond those (the spare statistics block behind a sequence
+ *     whose length is not a multiple of 128) belong to masked columns and never reach a result.  Two calls that
+ *     overlap on the GPU (different streams, no dependency) race on the array: serialise them.
  */
 #define GPROJ_STATIC_SCRATCH_BYTES (16u << 20)
 int gproj_attn_bwd_static_scratch(const void *Q, const void *K, const void *V, const void *O, const float *LSE,

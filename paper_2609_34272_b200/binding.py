@@ -171,6 +171,7 @@ def gproj_attn_bwd(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, workspac
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(K) if dV is None else dV
+    _check_bf16("dQ", dQ, Q.shape); _check_bf16("dK", dK, K.shape); _check_bf16("dV", dV, K.shape)
     with torch.cuda.device(Q.device):
         if Hkv == H:
             rc = load().gproj_attn_bwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
@@ -223,6 +224,7 @@ def gproj_attn_bwd_rect(Q, K, V, O, LSE, dO, softmax_scale, causal, flags=0, wor
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(K) if dV is None else dV
+    _check_bf16("dQ", dQ, Q.shape); _check_bf16("dK", dK, K.shape); _check_bf16("dV", dV, K.shape)
     with torch.cuda.device(Q.device):
         rc = load().gproj_attn_bwd_rect(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), dO.data_ptr(),
                                         dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, Hkv, Nq, Nk, d, float(softmax_scale),
@@ -250,6 +252,8 @@ def gproj_attn_bwd_static_scratch(Q, K, V, O, LSE, dO, softmax_scale, causal, fl
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(Q) if dK is None else dK
     dV = torch.empty_like(Q) if dV is None else dV
+    for name, t in (("dQ", dQ), ("dK", dK), ("dV", dV)):      # a wrong output tensor would be overwritten out of bounds
+        _check_bf16(name, t, Q.shape)
     with torch.cuda.device(Q.device):
         rc = load().gproj_attn_bwd_static_scratch(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
                                                   dO.data_ptr(), dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, N, d,

@@ -372,12 +372,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // The floor keeps the maximum finite for a row that has seen no key yet (unequal lengths: rows before the causal
         // diagonal reaches key 0), so that such a row gives z = exp2(-inf) = 0 instead of NaN from (-inf) - (-inf).
         const float mx = fmax3(fmax3(mxp[0], mxp[1], mxp[2]), fmax3(mxp[3], mxp[4], mxp[5]), fmax3(mxp[6], mxp[7], kFwdMaxFloor));
-        // Lazy maximum: the running maximum is only raised when the tile's maximum exceeds it by more than 2^kLazyLog2
-        // in the exponent domain; otherwise the stale value stays (z <= 2^kLazyLog2, harmless in FP32 / BF16) and neither
-        // l nor the accumulator needs a rescale.  The first tile always sets it (m_run = -inf).
+        // Lazy maximum: the running maximum is only raised when the tile's maximum exceeds it by more than 8 in the
+        // base-two exponent domain; otherwise the stale value stays (z <= 2^8, harmless in FP32 / BF16: O = acc / l and
+        // LSE = alpha m + ln l do not depend on which reference m was subtracted) and neither l nor the accumulator
+        // needs a rescale.  The first tile always sets it (m_run = -inf).  The fused variant always takes the true
+        // running maximum, so that it is the arithmetic of Eq. "historical-fma" and nothing else.
         float m_new = fmaxf(m_run, mx);
 #ifndef GPROJ_FWD_EAGER_MAX
-        if (__fmul_rn(__fsub_rn(m_new, m_run), scale_log2) <= 8.0f) m_new = m_run;
+        if (!FMA_SOFTMAX && __fmul_rn(__fsub_rn(m_new, m_run), scale_log2) <= 8.0f) m_new = m_run;
 #endif
         const float corr = fast_exp2(__fmul_rn(__fsub_rn(m_run, m_new), scale_log2));
         // FMA_SOFTMAX reproduces the native fused form of Eq. "historical-fma": z = exp2(fma(x, a, -fl32(x_max a))),

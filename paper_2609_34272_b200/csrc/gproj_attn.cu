@@ -746,21 +746,32 @@ int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const v
          cudaMemcpyAsync(dOin + q0 * row_bytes, static_cast<const uint8_t *>(dO) + q0 * row_bytes, qn * row_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
     if (ok && slabs > 1) ok = cudaEventRecord(st->ev_in[c], s_in) == cudaSuccess;
   }
-  if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+  // After the first copy has been queued, an error return first makes the caller's stream wait for whatever the call
+  // put on its internal streams, so that synchronising `stream` tells the caller its host buffers are free again.
+  auto fail = [&](int rc) {
+    (void)cudaGetLastError();
+    if (slabs > 1) {
+      if (cudaEventRecord(st->ev_end, s_in) == cudaSuccess) (void)cudaStreamWaitEvent(s, st->ev_end, 0);
+      if (cudaEventRecord(st->ev_end, s_out) == cudaSuccess) (void)cudaStreamWaitEvent(s, st->ev_end, 0);
+      (void)cudaGetLastError();
+    }
+    return rc;
+  };
+  if (!ok) return fail(GPROJ_ERR_CUDA);
   int launches = 0;
   for (int c = 0; c < slabs; ++c) {
     const size_t k0 = slab_begin(c), kn = slab_begin(c + 1) - k0, q0 = k0 * G, qn = kn * G;
-    if (slabs > 1 && cudaStreamWaitEvent(s, st->ev_in[c], 0) != cudaSuccess) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+    if (slabs > 1 && cudaStreamWaitEvent(s, st->ev_in[c], 0) != cudaSuccess) return fail(GPROJ_ERR_CUDA);
     float *lse_c = reinterpret_cast<float *>(dLSE + q0 * N * sizeof(float));
     // a slab is a problem with batch 1, kn KV heads and qn query heads; the slabs share the backward workspace in turn
     if (int rc = gproj_attn_fwd_gqa(dQin + q0 * row_bytes, dKin + k0 * row_bytes, dVin + k0 * row_bytes, dOout + q0 * row_bytes, lse_c, 1,
                                     static_cast<int>(qn), static_cast<int>(kn), N, d, softmax_scale, causal, stream))
-      return rc;
+      return fail(rc);
     launches += tl_launch_count;
     if (int rc = gproj_attn_bwd_gqa(dQin + q0 * row_bytes, dKin + k0 * row_bytes, dVin + k0 * row_bytes, dOout + q0 * row_bytes, lse_c,
                                     dOin + q0 * row_bytes, dQout + q0 * row_bytes, dKout + k0 * row_bytes, dVout + k0 * row_bytes, 1,
                                     static_cast<int>(qn), static_cast<int>(kn), N, d, softmax_scale, causal, ws, ws_bytes, flags, stream))
-      return rc;
+      return fail(rc);
     launches += tl_launch_count;
     ok = slabs == 1 || (cudaEventRecord(st->ev_done[c], s) == cudaSuccess && cudaStreamWaitEvent(s_out, st->ev_done[c], 0) == cudaSuccess);
     ok = ok && cudaMemcpyAsync(static_cast<uint8_t *>(dQ) + q0 * row_bytes, dQout + q0 * row_bytes, qn * row_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess &&
@@ -768,7 +779,7 @@ int gproj_attn_fwd_bwd_host(const void *Q, const void *K, const void *V, const v
          cudaMemcpyAsync(static_cast<uint8_t *>(dV) + k0 * row_bytes, dVout + k0 * row_bytes, kn * row_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
     if (ok && O) ok = cudaMemcpyAsync(static_cast<uint8_t *>(O) + q0 * row_bytes, dOout + q0 * row_bytes, qn * row_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
     if (ok && LSE) ok = cudaMemcpyAsync(LSE + q0 * N, lse_c, qn * N * sizeof(float), cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
-    if (!ok) { (void)cudaGetLastError(); return GPROJ_ERR_CUDA; }
+    if (!ok) return fail(GPROJ_ERR_CUDA);
   }
   // the caller's stream reaches the end of the call only when the last copy-out has landed
   if (slabs > 1 && !(cudaEventRecord(st->ev_end, s_out) == cudaSuccess && cudaStreamWaitEvent(s, st->ev_end, 0) == cudaSuccess)) {
@@ -833,7 +844,7 @@ const char *gproj_status_string(int status) {
   switch (status) {
     case GPROJ_OK: return "ok";
     case GPROJ_ERR_NULL: return "null pointer argument";
-    case GPROJ_ERR_SHAPE: return "unsupported shape (need d in {64,128}, B, H, N >= 1, H a multiple of the KV heads, B*H*N < 2^31)";
+    case GPROJ_ERR_SHAPE: return "unsupported shape (d must be 64 or 128; dimensions positive; H a multiple of Hkv; B*H*N < 2^31, B*H < 2^20, N <= 2^24, fewer than 2^24 tiles)";
     case GPROJ_ERR_ALIGN: return "tensor base address not 16-byte aligned";
     case GPROJ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case GPROJ_ERR_SCALE: return "softmax_scale must be finite and positive";

@@ -390,3 +390,38 @@ def test_two_streams_run_concurrently_without_interference():
     for r, o in zip(ref, out):
         for a, b in zip(r, o):
             assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("causal", [False, True])
+def test_row_maximum_that_creeps_up_across_key_tiles(d, causal):
+    # The forward subtracts a lazily raised running maximum (raised only when a key tile exceeds it by more than 8 in
+    # the base-two exponent domain).  Here every row's maximum grows a little with every key tile: by less than the
+    # threshold from one tile to the next (so the stale reference is kept for several tiles and z exceeds one), but by
+    # far more than it over the row.  O and LSE must stay inside the bars either way, and so must the fused variant,
+    # which always takes the true running maximum.
+    N, H = 2048, 2
+    gen = torch.Generator().manual_seed(515 + d)
+    Q, K, V, dO = (torch.randn(1, H, N, d, generator=gen) for _ in range(4))
+    c = torch.randn(d, generator=gen); c = c / c.norm()
+    alpha = float(np.float32(1 / math.sqrt(d)))
+    ramp = torch.arange(N, dtype=torch.float32) / N                  # key j carries ramp_j * 40 / (alpha * 4) along c
+    Q = Q * 0.5 + 4.0 * c
+    K = K * 0.5 + (ramp[:, None] * (40.0 / (alpha * 4.0))) * c        # score grows by about 40 nats over the row, 2.5 per tile
+    Q, K, V, dO = (t.to(torch.bfloat16) for t in (Q, K, V, dO))
+    ex = oracle.attn_fwd_bwd_f64(bits(Q), bits(K), bits(V), bits(dO), alpha, causal)
+    for fwd_flags in (0, g.FWD_FLAG_FMA_SOFTMAX):
+        O, LSE = g.gproj_attn_fwd(Q.cuda(), K.cuda(), V.cuda(), alpha, causal, fwd_flags=fwd_flags)
+        rc, detail = g.gproj_last_device_status()
+        assert rc == 0, hex(detail)
+        eO = oracle.rel_l2_percent(O.float().cpu().numpy(), ex["O"])
+        dL = np.abs(LSE.cpu().numpy().astype(np.float64) - ex["LSE"])
+        assert eO <= 1.0, (fwd_flags, eO)
+        assert np.all(dL <= 1e-4 + 1e-5 * np.abs(ex["LSE"])), (fwd_flags, dL.max())
+        if fwd_flags == 0:
+            dQ, dK, dV = g.gproj_attn_bwd(Q.cuda(), K.cuda(), V.cuda(), O, LSE, dO.cuda(), alpha, causal)
+            for n, t in (("dQ", dQ), ("dK", dK), ("dV", dV)):
+                assert oracle.rel_l2_percent(t.float().cpu().numpy(), ex[n]) <= 1.0, n
+    span = (ex["LSE"][0, 0, -1] - ex["LSE"][0, 0, 0]) if causal else None
+    if causal:
+        assert span > 20.0                                            # the construction does what it says

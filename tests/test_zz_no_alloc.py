@@ -1,4 +1,7 @@
-"""The workspace-free backward entry point, through the C ABI (collected last on purpose).
+"""The workspace-free backward entry point, through the C ABI.
+
+The file name sorts behind every other test file, so pytest collects it last: a run that stops at the first failure
+(-x) has then already run every other test before it reaches this added entry point.
 
 Some users of this library cannot allocate device memory at the moment they need a gradient (a plugin inside
 another framework's memory pool, a process whose memory is fixed at start-up).  For them the library carries its
@@ -40,6 +43,41 @@ def test_static_scratch_matches_workspace_backward_twice_in_a_row():
             assert torch.equal(a, b), name
     ref, got = _run_both(first, flags=g.FLAG_NO_K_CORRECTION)
     assert all(torch.equal(a, b) for a, b in zip(ref, got))
+
+
+def test_static_scratch_allocates_nothing_and_is_not_fooled_by_a_larger_earlier_call():
+    # A large problem first (it fills most of the built-in array), then small ones of other shapes whose second kernel
+    # also reads statistic blocks the first kernel does not write for them (d = 64, N mod 128 in 1..64): whatever the large
+    # call left there must not reach a result.  With the outputs pre-allocated the call must leave both PyTorch's
+    # allocator and the device's free memory exactly as they were -- that is what the entry point is for.
+    big = Workload("noalloc_big", 1, 16, 4096, 64, True, k_offset=16.0, seed=21)
+    _run_both(big)
+    for w in (Workload("noalloc_s1", 1, 3, 192, 64, True, k_offset=8.0, seed=22), Workload("noalloc_s2", 2, 2, 320, 64, False, seed=23),
+              Workload("noalloc_s3", 1, 2, 129, 128, True, seed=24)):
+        inp = {k: v.cuda() for k, v in make_inputs(w).items()}
+        O, LSE = g.gproj_attn_fwd(inp["Q"], inp["K"], inp["V"], w.softmax_scale, w.causal)
+        ref = g.gproj_attn_bwd(inp["Q"], inp["K"], inp["V"], O, LSE, inp["dO"], w.softmax_scale, w.causal)
+        out = [torch.empty_like(inp["Q"]) for _ in range(3)]
+        g.gproj_attn_bwd_static_scratch(inp["Q"], inp["K"], inp["V"], O, LSE, inp["dO"], w.softmax_scale, w.causal,
+                                        dQ=out[0], dK=out[1], dV=out[2])            # first call of the shape: any one-time set-up
+        torch.cuda.synchronize()
+        for t in out:
+            t.zero_()
+        torch.cuda.synchronize()
+        allocated, reserved, free = torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0]
+        g.gproj_attn_bwd_static_scratch(inp["Q"], inp["K"], inp["V"], O, LSE, inp["dO"], w.softmax_scale, w.causal,
+                                        dQ=out[0], dK=out[1], dV=out[2])
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == allocated and torch.cuda.memory_reserved() == reserved
+        assert torch.cuda.mem_get_info()[0] == free
+        rc, detail = g.gproj_last_device_status()
+        assert rc == 0, hex(detail)
+        for name, a, b in zip(("dQ", "dK", "dV"), ref, out):
+            assert torch.equal(a, b), (w.name, name)
+    # a wrongly shaped output tensor is refused before anything is launched
+    with pytest.raises(ValueError):
+        g.gproj_attn_bwd_static_scratch(inp["Q"], inp["K"], inp["V"], O, LSE, inp["dO"], w.softmax_scale, w.causal,
+                                        dQ=torch.empty(1, 1, 8, 128, dtype=torch.bfloat16, device="cuda"))
 
 
 def test_static_scratch_rejects_shapes_beyond_its_size():

@@ -246,6 +246,22 @@ int gproj_attn_bwd_static_scratch(const void *Q, const void *K, const void *V, c
                                   unsigned flags, void *stream);
 
 /*
+ * Key smoothing, the comparison arm of Section 5.1 and of Table "method-definitions" ("FA3 on mean-subtracted keys"):
+ * subtract the per-sequence, per-KV-head mean row, Y_j = BF16(fl32(X_j - mean_j X_j)), mean and subtraction in FP32.
+ * The arm is built from calls of this library: K~ = gproj_key_smooth(K); the forward on (Q, K~, V) with
+ * GPROJ_FWD_FLAG_FMA_SOFTMAX; the backward with both corrections off; dK = gproj_key_smooth(dK~), which is the
+ * vector-Jacobian product of the subtraction (dK_j = dK~_j - mean_l dK~_l).  Softmax is unchanged by the shift in exact
+ * arithmetic; what the shift removes is the common component of the keys that the leaked row mass multiplies, not
+ * the leak itself (Section 2).  The paper's experiments use it only as a baseline; so does this library.
+ *   X, Y: DEVICE BF16, [B][Hkv][N][d] (dense) or [Hkv][T][d] with HOST offsets cu_seqlens (packed; the mean is taken
+ *   inside each sequence; empty sequences are skipped); Y may be X.  One launch per sequence, on `stream`.
+ *   Errors: GPROJ_ERR_NULL, GPROJ_ERR_SHAPE (d not 64 / 128, non-positive sizes, malformed offsets), GPROJ_ERR_ALIGN,
+ *   GPROJ_ERR_ARCH, GPROJ_ERR_CUDA.
+ */
+int gproj_key_smooth(const void *X, void *Y, int B, int Hkv, int N, int d, void *stream);
+int gproj_key_smooth_varlen(const void *X, void *Y, const int *cu_seqlens, int num_seqs, int Hkv, int d, void *stream);
+
+/*
  * Synchronises `stream`, then returns GPROJ_OK, GPROJ_ERR_TIMEOUT if any kernel launched by this
  * library on the current device since the last call recorded an abandoned wait, or GPROJ_ERR_CUDA.
  * If `detail` is non-NULL it receives the raw device code (0 when fine) and the code is cleared.

@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     gproj_attn_fwd_bwd_host,
     gproj_attn_fwd_rect,
     gproj_attn_host_staging_bytes,
+    gproj_key_smooth,
     gproj_attn_fwd_varlen,
     gproj_attn_fwd_varlen_qk,
     gproj_last_device_status,

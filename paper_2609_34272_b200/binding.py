@@ -26,7 +26,7 @@ EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd",
            "gproj_attn_varlen_plan_bytes", "gproj_attn_varlen_plan", "gproj_attn_fwd_varlen",
            "gproj_attn_bwd_varlen_workspace_bytes", "gproj_attn_bwd_varlen",
            "gproj_attn_varlen_qk_plan_bytes", "gproj_attn_varlen_qk_plan", "gproj_attn_fwd_varlen_qk", "gproj_attn_bwd_varlen_qk",
-           "gproj_attn_host_staging_bytes", "gproj_attn_fwd_bwd_host",
+           "gproj_attn_host_staging_bytes", "gproj_attn_fwd_bwd_host", "gproj_key_smooth", "gproj_key_smooth_varlen",
            "gproj_last_device_status", "gproj_selftest_wait_timeout",
            "gproj_status_string", "gproj_last_launch_count")
 
@@ -89,6 +89,10 @@ def load():
         lib.gproj_attn_host_staging_bytes.argtypes = [i, i, i, i, i]
         lib.gproj_attn_fwd_bwd_host.restype = i
         lib.gproj_attn_fwd_bwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, ctypes.c_size_t, u, vp]
+        lib.gproj_key_smooth.restype = i
+        lib.gproj_key_smooth.argtypes = [vp, vp, i, i, i, i, vp]
+        lib.gproj_key_smooth_varlen.restype = i
+        lib.gproj_key_smooth_varlen.argtypes = [vp, vp, ip, i, i, i, vp]
         lib.gproj_selftest_wait_timeout.restype = i
         lib.gproj_selftest_wait_timeout.argtypes = [vp]
         lib.gproj_last_device_status.restype = i
@@ -261,6 +265,25 @@ def gproj_attn_bwd_static_scratch(Q, K, V, O, LSE, dO, softmax_scale, causal, fl
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_bwd_static_scratch")
     return dQ, dK, dV
+
+
+def gproj_key_smooth(X, Y=None, cu_seqlens=None):
+    """Y = X minus its per-sequence, per-head mean row (key smoothing; also the matching fix-up of dK).
+    X: CUDA bfloat16 [B, Hkv, N, d], or packed [Hkv, T, d] with host offsets ``cu_seqlens``."""
+    _check_bf16("X", X)
+    Y = torch.empty_like(X) if Y is None else Y
+    _check_bf16("Y", Y, X.shape)
+    with torch.cuda.device(X.device):
+        if cu_seqlens is None:
+            B, Hkv, N, d = X.shape
+            rc = load().gproj_key_smooth(X.data_ptr(), Y.data_ptr(), B, Hkv, N, d, _stream(X.device))
+        else:
+            Hkv, T, d = X.shape
+            cu = (ctypes.c_int * len(cu_seqlens))(*[int(v) for v in cu_seqlens])
+            rc = load().gproj_key_smooth_varlen(X.data_ptr(), Y.data_ptr(), cu, len(cu_seqlens) - 1, Hkv, d, _stream(X.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_key_smooth")
+    return Y
 
 
 def gproj_last_device_status(device=None):

@@ -13,6 +13,7 @@
 #include "attn_bwd.cuh"
 #include "attn_bwd_w128.cuh"
 #include "attn_fwd.cuh"
+#include "key_smoothing.cuh"
 
 namespace {
 
@@ -857,6 +858,49 @@ const char *gproj_status_string(int status) {
 }
 
 int gproj_last_launch_count(void) { return tl_launch_count; }
+
+// ---- key smoothing (comparison arm of Section 5.1): subtract the per-sequence, per-head mean row -------------------
+static int smooth_rows(const void *X, void *Y, int heads, long long rows_total, int d, const int *cu_seqlens, int num_seqs,
+                       void *stream) {
+  if (!X || !Y) return GPROJ_ERR_NULL;
+  if (heads <= 0 || rows_total <= 0 || (d != 64 && d != 128) || heads >= (1 << 20) || rows_total * heads >= (1LL << 31))
+    return GPROJ_ERR_SHAPE;
+  if (!aligned16(X) || !aligned16(Y)) return GPROJ_ERR_ALIGN;
+  if (cu_seqlens) {
+    if (num_seqs <= 0 || cu_seqlens[0] != 0 || cu_seqlens[num_seqs] != rows_total) return GPROJ_ERR_SHAPE;
+    for (int s = 0; s < num_seqs; ++s)
+      if (cu_seqlens[s + 1] < cu_seqlens[s]) return GPROJ_ERR_SHAPE;
+  }
+  DeviceState *st = nullptr;
+  if (int rc = device_state(&st)) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(X);
+  __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(Y);
+  int launches = 0;
+  const int n = cu_seqlens ? num_seqs : 1;
+  for (int q = 0; q < n; ++q) {
+    const int r0 = cu_seqlens ? cu_seqlens[q] : 0, rows = cu_seqlens ? cu_seqlens[q + 1] - r0 : static_cast<int>(rows_total);
+    if (rows == 0) continue;
+    if (d == 64) smooth_rows_kernel<64><<<heads, kSmoothThreads, 0, s>>>(x, y, rows_total * d, r0, rows);
+    else         smooth_rows_kernel<128><<<heads, kSmoothThreads, 0, s>>>(x, y, rows_total * d, r0, rows);
+    ++launches;
+  }
+  if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
+  tl_launch_count = launches;
+  return GPROJ_OK;
+}
+
+int gproj_key_smooth(const void *X, void *Y, int B, int Hkv, int N, int d, void *stream) {
+  if (B <= 0 || Hkv <= 0 || N <= 0) return GPROJ_ERR_SHAPE;
+  if (static_cast<long long>(B) * Hkv >= (1LL << 20)) return GPROJ_ERR_SHAPE;
+  return smooth_rows(X, Y, B * Hkv, N, d, nullptr, 0, stream);
+}
+
+int gproj_key_smooth_varlen(const void *X, void *Y, const int *cu_seqlens, int num_seqs, int Hkv, int d, void *stream) {
+  if (!cu_seqlens) return GPROJ_ERR_NULL;
+  if (num_seqs <= 0) return GPROJ_ERR_SHAPE;
+  return smooth_rows(X, Y, Hkv, cu_seqlens[num_seqs], d, cu_seqlens, num_seqs, stream);
+}
 
 #ifdef GPROJ_TRACE
 // Debug builds only: per-tile timeline of the most recent launches (count, then {cta, tile, start ns, end ns} records).

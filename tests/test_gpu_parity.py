@@ -2,8 +2,14 @@
 
 Bar (written here, from the benchmark spec): full-tensor relative L2 error of O, dQ, dK, dV
 at most 1.0 %.  LSE is FP32 state, checked to |err| <= 1e-4 + 1e-5 |LSE| (FP32 accumulation of
-<= 32768 terms with a 2^-22 exponential).  An element-wise bound (|err| <= 3 % of the tensor's
-max magnitude) guards against a localized fault hiding in the norm.
+<= 32768 terms with a 2^-22 exponential).  An element-wise bound guards against a localized fault
+hiding in the norm; on the small shapes it is |err| <= 2^-7 |exact| + 0.05 rms(exact), on the five large
+workloads 3 % of the tensor's largest entry.  The first term is two BF16 steps of the output
+(its final cast alone may cost half a step); the second allows twenty standard deviations of the noise the BF16
+operands r, t leave in an FP32 accumulation, whose level is the 0.25 % relative L2 floor of every tensor here.
+(Rows with few contributions, the last keys of a causal head, are the noisiest relative to the tensor's rms.)
+A wrong 16-column chunk in a single row is off by about one rms and fails it; the bound is six times tighter than
+three percent of the tensor's largest entry.
 """
 import numpy as np
 import pytest
@@ -32,14 +38,19 @@ def run_gpu(inp, w, flags=0):
     return {"O": to_np(O), "LSE": LSE.cpu().numpy().astype(np.float64), "dQ": to_np(dQ), "dK": to_np(dK), "dV": to_np(dV)}
 
 
-def check(got, ex, names=("O", "dQ", "dK", "dV"), bar=REL_L2_BAR, sel=None):
+def check(got, ex, names=("O", "dQ", "dK", "dV"), bar=REL_L2_BAR, sel=None, tight=False):
     errs = {}
     for n in names:
         a = got[n] if sel is None else got[n][sel]
         e = ex[n]
         errs[n] = oracle.rel_l2_percent(a, e)
         assert errs[n] <= bar, (n, errs)
-        assert np.abs(a - e).max() <= 0.03 * np.abs(e).max(), (n, "element-wise")
+        if tight:     # the small shapes: per-element bound from the output's BF16 step and the accumulation noise
+            worst = (np.abs(a - e) / (2.0 ** -7 * np.abs(e) + 0.05 * np.sqrt(np.mean(e * e)))).max()
+            errs[n + "_elementwise"] = round(float(worst), 3)
+            assert worst <= 1.0, (n, "element-wise", worst)
+        else:         # millions of elements, rows with one to thousands of keys: 3 % of the largest entry
+            assert np.abs(a - e).max() <= 0.03 * np.abs(e).max(), (n, "element-wise")
     if "LSE" in ex:
         a = got["LSE"] if sel is None else got["LSE"][sel]
         assert np.all(np.abs(a - ex["LSE"]) <= 1e-4 + 1e-5 * np.abs(ex["LSE"]))
@@ -57,14 +68,14 @@ def test_small_shapes(B, H, N, d, causal, koff):
     w = Workload("small", B, H, N, d, causal, k_offset=koff, seed=4242 + 17 * N + d)
     inp = make_inputs(w)
     ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, causal)
-    check(run_gpu(inp, w), ex)
+    check(run_gpu(inp, w), ex, tight=True)
 
 
 def test_config1():
     w = workload(1)
     inp = make_inputs(w)
     ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, w.causal)
-    errs = check(run_gpu(inp, w), ex)
+    errs = check(run_gpu(inp, w), ex, tight=True)
     print("config 1:", errs)
 
 
@@ -97,21 +108,37 @@ def test_config3_offset_sweep():
 
 
 def test_config4_head_subset():
-    # Full-size launch; the oracle scores 4 of the 128 (batch, head) problems, one per batch index
+    # Full-size launch; the oracle scores 8 of the 128 (batch, head) problems, two per batch index
     # (each (b, h) is an independent problem).
     w = workload(4)
     inp = make_inputs(w)
-    got = run_gpu(inp, w)
-    heads = [b * w.H + h for b, h in ((0, 0), (1, 13), (2, 31), (3, 7))]
+    dev = {k: v.cuda() for k, v in inp.items()}
+    O, LSE = g.gproj_attn_fwd(dev["Q"], dev["K"], dev["V"], w.softmax_scale, w.causal)
+    dQ, dK, dV = g.gproj_attn_bwd(dev["Q"], dev["K"], dev["V"], O, LSE, dev["dO"], w.softmax_scale, w.causal)
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, (g.status_string(rc), hex(detail))
+    heads = [b * w.H + h for b, h in ((0, 0), (0, 21), (1, 13), (1, 30), (2, 31), (2, 2), (3, 7), (3, 16))]
     ex = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, w.causal, heads=heads)
-    flat = {n: v.reshape((w.B * w.H,) + v.shape[2:])[heads] for n, v in got.items()}
-    errs = check(flat, ex)
-    print("config 4 (4 heads):", errs)
+    flat = lambda t: to_np(t.reshape((w.B * w.H,) + t.shape[2:])[heads])
+    got = {"O": flat(O), "dQ": flat(dQ), "dK": flat(dK), "dV": flat(dV), "LSE": LSE.reshape(w.B * w.H, w.N)[heads].cpu().numpy().astype(np.float64)}
+    errs = check(got, ex)
+    print("config 4 (8 heads):", errs)
+    # Every one of the 128 heads: the dense non-causal launch deals its tiles head-major; scheduling must not change a
+    # bit of the backward.  The same heads run in chunks of 16 from the same saved O and LSE give identical gradients.
+    fl = lambda t: t.reshape((1, w.B * w.H) + t.shape[2:])
+    Qf, Kf, Vf, Uf, Of, Lf, dQf, dKf, dVf = (fl(t) for t in (dev["Q"], dev["K"], dev["V"], dev["dO"], O, LSE, dQ, dK, dV))
+    for h0 in range(0, w.B * w.H, 16):
+        sl = slice(h0, h0 + 16)
+        q, k, v, u, o, lse = (t[:, sl].contiguous() for t in (Qf, Kf, Vf, Uf, Of, Lf))
+        dq2, dk2, dv2 = g.gproj_attn_bwd(q, k, v, o, lse, u, w.softmax_scale, w.causal)
+        assert torch.equal(dq2, dQf[:, sl]) and torch.equal(dk2, dKf[:, sl]) and torch.equal(dv2, dVf[:, sl]), h0
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, hex(detail)
 
 
 def test_config5_sampled_rows():
     # Full-size launch; O, LSE, dQ on 64 seeded query rows per head against their full key range;
-    # dK, dV on 64 seeded key rows of one head, using FP64 forward statistics of every query row of that head.
+    # dK, dV on 64 seeded key rows of three heads, using FP64 forward statistics of every query row of those heads.
     w = workload(5)
     inp = make_inputs(w)
     got = run_gpu(inp, w)
@@ -121,12 +148,12 @@ def test_config5_sampled_rows():
         O, LSE, _, dQ = oracle.head_rows_f64(q[h], k[h], v[h], u[h], w.softmax_scale, True, rows)
         check({"O": got["O"][0, h, rows], "dQ": got["dQ"][0, h, rows], "LSE": got["LSE"][0, h, rows]},
               {"O": O, "dQ": dQ, "LSE": LSE}, names=("O", "dQ"))
-    h = 5
     allrows = np.arange(w.N, dtype=np.int32)
-    _, LSE, MUA, _ = oracle.head_rows_f64(q[h], k[h], v[h], u[h], w.softmax_scale, True, allrows)
-    keys = sample_rows(w, 64, salt=100)
-    dK, dV = oracle.head_keys_f64(q[h], k[h], v[h], u[h], w.softmax_scale, True, LSE, MUA, keys)
-    check({"dK": got["dK"][0, h, keys], "dV": got["dV"][0, h, keys]}, {"dK": dK, "dV": dV}, names=("dK", "dV"))
+    for h in (5, 0, 2):
+        _, LSE, MUA, _ = oracle.head_rows_f64(q[h], k[h], v[h], u[h], w.softmax_scale, True, allrows)
+        keys = sample_rows(w, 64, salt=100 + h)
+        dK, dV = oracle.head_keys_f64(q[h], k[h], v[h], u[h], w.softmax_scale, True, LSE, MUA, keys)
+        check({"dK": got["dK"][0, h, keys], "dV": got["dV"][0, h, keys]}, {"dK": dK, "dV": dV}, names=("dK", "dV"))
     # property that holds at any size: the exact key gradient sums to zero over keys (sum_j dS_ij = 0)
     dk = got["dK"][0]
     assert np.linalg.norm(dk.sum(axis=1)) <= 0.02 * np.linalg.norm(dk)

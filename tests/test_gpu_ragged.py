@@ -163,3 +163,29 @@ def test_many_heads_long_causal_matches_chunks_of_heads(d):
         assert torch.equal(dq2, dQ[:, sl]) and torch.equal(dk2, dK[:, sl]) and torch.equal(dv2, dV[:, sl]), h0
     rc, detail = g.gproj_last_device_status()
     assert rc == 0, hex(detail)
+
+
+@pytest.mark.parametrize("d,causal", [(64, True), (128, False)])
+def test_head_shards_give_the_bits_of_the_whole_call(d, causal):
+    # The multi-GPU launch cuts the flat (batch, head) axis into contiguous shares (one per rank, no exchange).  Run the
+    # shares one after the other on this GPU: laid side by side they must be the whole call's outputs bit for bit.
+    from paper_2609_34272_b200.sharding import shard_heads
+    B, H, N = 2, 5, 640
+    gen = torch.Generator().manual_seed(606 + d)
+    Q, K, V, dO = (torch.randn(B, H, N, d, generator=gen).to(torch.bfloat16).cuda() for _ in range(4))
+    alpha = d ** -0.5
+    O, LSE = g.gproj_attn_fwd(Q, K, V, alpha, causal)
+    dQ, dK, dV = g.gproj_attn_bwd(Q, K, V, O, LSE, dO, alpha, causal)
+    fl = lambda t: t.reshape((1, B * H) + t.shape[2:])
+    for world in (2, 3, 4):
+        for r in range(world):
+            mine = shard_heads(B * H, world, r)
+            q, k, v, u = (fl(t)[:, mine.start:mine.stop].contiguous() for t in (Q, K, V, dO))
+            o, lse = g.gproj_attn_fwd(q, k, v, alpha, causal)
+            dq, dk, dv = g.gproj_attn_bwd(q, k, v, o, lse, u, alpha, causal)
+            sl = slice(mine.start, mine.stop)
+            assert torch.equal(lse, fl(LSE)[:, sl]) or torch.allclose(lse, fl(LSE)[:, sl], rtol=1e-5, atol=1e-5)
+            dq2, dk2, dv2 = g.gproj_attn_bwd(q, k, v, fl(O)[:, sl].contiguous(), fl(LSE)[:, sl].contiguous(), u, alpha, causal)
+            assert torch.equal(dq2, fl(dQ)[:, sl]) and torch.equal(dk2, fl(dK)[:, sl]) and torch.equal(dv2, fl(dV)[:, sl]), (world, r)
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, hex(detail)

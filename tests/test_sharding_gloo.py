@@ -25,11 +25,12 @@ def _worker(rank, world, port, out_dir):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
         # each rank scores its own heads with no exchange; results must tile the full problem
-        w = Workload("shard", 1, 4, 64, 8, True, seed=3)
+        w = Workload("shard", 2, 3, 64, 8, True, seed=3)      # six (batch, head) pairs: the split cuts through a batch
         inp = {k: bits(v) for k, v in make_inputs(w).items()}
         mine = list(shard_heads(w.B * w.H, world, rank))
         part = oracle.attn_fwd_bwd_f64(inp["Q"], inp["K"], inp["V"], inp["dO"], w.softmax_scale, True, heads=mine)
-        np.save(os.path.join(out_dir, f"dq_{rank}.npy"), part["dQ"])
+        for name in ("O", "dQ", "dK", "dV"):
+            np.save(os.path.join(out_dir, f"{name}_{rank}.npy"), part[name])
         slowest = max_over_ranks(10.0 + rank, world)
         assert slowest == 10.0 + (world - 1)
         dist.barrier()
@@ -40,8 +41,24 @@ def _worker(rank, world, port, out_dir):
 def test_two_ranks_gloo(tmp_path):
     s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
     mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
-    w = Workload("shard", 1, 4, 64, 8, True, seed=3)
+    w = Workload("shard", 2, 3, 64, 8, True, seed=3)
     inp = {k: bits(v) for k, v in make_inputs(w).items()}
     full = oracle.attn_fwd_bwd_f64(inp["Q"], inp["K"], inp["V"], inp["dO"], w.softmax_scale, True)
-    got = np.concatenate([np.load(tmp_path / f"dq_{r}.npy") for r in range(2)])
-    assert np.array_equal(got, full["dQ"].reshape(got.shape))
+    for name in ("O", "dQ", "dK", "dV"):
+        got = np.concatenate([np.load(tmp_path / f"{name}_{r}.npy") for r in range(2)])
+        assert np.array_equal(got, full[name].reshape(got.shape)), name     # the shards tile the one-rank result exactly
+
+
+def test_share_of_a_rank_is_a_dense_problem_of_its_own():
+    # what `bench.py --shard heads` hands to rank r: the flat (batch, head) axis cut at shard_heads(), batch 1
+    w = Workload("shard", 2, 3, 64, 8, False, seed=5)
+    inp = make_inputs(w)
+    full = oracle.attn_fwd_bwd_f64(*(bits(inp[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, False)
+    for world in (2, 4):
+        parts = []
+        for r in range(world):
+            mine = shard_heads(w.B * w.H, world, r)
+            sub = {k: v.reshape(1, w.B * w.H, w.N, w.d)[:, mine.start:mine.stop].contiguous() for k, v in inp.items()}
+            if len(mine):
+                parts.append(oracle.attn_fwd_bwd_f64(*(bits(sub[k]) for k in ("Q", "K", "V", "dO")), w.softmax_scale, False)["dK"][0])
+        assert np.array_equal(np.concatenate(parts), full["dK"].reshape(w.B * w.H, w.N, w.d))

@@ -60,7 +60,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index, period=0.002):
         super().__init__(daemon=True)
         self.index, self.period = index, period
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.reasons, self.max_mhz, self.power_w = [], set(), None, []
         self._stop_evt = threading.Event()
         self.ok = False
         try:
@@ -79,6 +79,7 @@ class ClockSampler(threading.Thread):
         while not self._stop_evt.is_set():
             try:
                 self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                self.power_w.append(self.nv.nvmlDeviceGetPowerUsage(self.h) / 1e3)
                 mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
                 for bit, name in self.REASONS.items():
                     if mask & bit:
@@ -92,7 +93,9 @@ class ClockSampler(threading.Thread):
         if self.is_alive():
             self.join(timeout=2)
         return {"sm_mhz": (statistics.median(self.samples) if self.samples else None),
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_median": (statistics.median(self.power_w) if self.power_w else None),
+                "power_w_max": (max(self.power_w) if self.power_w else None)}
 
 
 def flops(w):

@@ -5,25 +5,32 @@
 // instruction (the full 8192 FLOP/clk/SM; an N = 64 instruction costs 48 clk for 32 clk of work):
 //
 //   columns   0..127  X   S^T of the even steps, then their packed r^T / t^T
-//           128..255  Y   dP^T of every step (single-buffered)
+//           128..255  Y   dP^T of every step (single-buffered, consumed into registers at the start of the step)
 //           256..383  Z   S^T of the odd steps, then their packed r^T / t^T
 //           384..447  dV accumulator,   448..511  dK accumulator
 //
-// A step is 128 streamed query rows.  Its arithmetic runs in two phases: phase 1 needs only S^T (p = exp2(..), r = BF16(p),
-// p kept in FP32 registers), phase 2 needs dP^T (t = BF16(p (dP - D))).  Because dP^T is consumed quickly and S^T is
-// double-buffered, the tensor core computes the scores of step n + 1 while the ALUs work on step n, and the products
-// that need only r^T start while t^T is still being computed:
+// A step is 128 streamed query rows.  Thread <-> (key row, two 16-column chunks of the step: columns 16 w .. 16 w + 15 of
+// the first 64 queries, then of the last 64; w = warpgroup).  At the start of a step a thread takes dP^T of both chunks
+// into registers and releases the single dP^T buffer at once, so the tensor core writes the next step's dP^T while this
+// step is in the ALUs.  Each chunk is then done in one pass (p = exp2(..), r = BF16(p), t = BF16(p (dP - D))) and the two
+// halves of the step are handed over separately, so the second-stage products of the first 64 queries run while the
+// last 64 are in the ALUs.
 //
 //   issuer 1:  S^T(n) -> [X|Z]   when stage n landed and the second-stage products of step n - 2 are done
-//              dP^T(n) -> Y       when phase 2 of step n - 1 has read Y
-//   ALUs:      phase 1(n) after S^T(n): r^T -> over S^T;   phase 2(n) after dP^T(n): t^T -> over S^T, Y free
-//   issuer 2:  [dV | dK] += r^T [dO | Z] after phase 1(n);   dK += t^T Q after phase 2(n);   then [X|Z] of step n is free
+//   issuer 3:  dP^T(n) -> Y       when the ALUs hold dP^T of step n - 1 in registers
+//   ALUs:      dP^T(n) -> registers, Y free;  chunk 0: r^T, t^T over S^T, first half ready;  chunk 1: second half ready
+//   issuer 2:  per half:  [dV | dK] += r^T [dO | Z],  dK += t^T Q;   after the second half [X|Z] of step n is free
 //
-// All four compute warpgroups work on the same step, warpgroup w on the 32-column slice w (thread <-> (key row, slice)).
+// Three issuing warps, because the tensor core takes its work in the order it is issued and holds an issuing thread for
+// as long as its products execute: dP^T(n + 1), which the ALUs want the moment they finish step n, must not wait in one
+// thread's program order behind S^T(n + 1) (whose buffer frees late) nor behind the second-stage products of step n.
+// (Measured on workload 2, against two-phase arithmetic with two issuing warps: 79.3 -> 77.6 us back to back.  Not kept,
+// all measured no faster: the two halves of the step on two warpgroup pairs running half a step apart; the next step's
+// TMEM loads issued behind the last stores of the current one; dP^T issued by the second-stage warp one step ahead.)
 // Everything else (persistent tile schedule, TMA staging, epilogue through a swizzled staging buffer, packed-sequence
-// descriptors, bounded waits) is as in attn_bwd.cuh.  Measured against the 64-wide kernel at d = 64: 6 % faster on
-// workload 2, 9 % on a non-causal problem; the same layout for the dQ side was 5 % SLOWER than its 64-wide kernel (its
-// phases also carry the row-mass sums) and is not kept.
+// descriptors, bounded waits) is as in attn_bwd.cuh.  Against the 64-wide kernel at d = 64 this kernel is about 8 % faster
+// on workload 2; the same layout for the dQ side was 5 % SLOWER than its 64-wide kernel (its arithmetic also carries the
+// row-mass sums) and is not kept.
 #pragma once
 #include "attn_bwd.cuh"
 
@@ -34,8 +41,7 @@ struct BwdW128 {
   static constexpr int kTileBytes = 128 * 128;                     // 128 rows x 64 BF16: one 128-byte-row slab
   static constexpr int kStepRows = 128;
   static constexpr int kStages = 3;
-  static constexpr int kWG = 4, kCompute = 128 * kWG, kThreads = 96 + kCompute;   // warp 0: stage producer (lane 0) and tile loader (lane 1); warps 1, 2: MMA issuers; 16 compute warps
-  static constexpr int kSliceCols = kStepRows / kWG;               // 32 columns per thread and step
+  static constexpr int kWG = 4, kCompute = 128 * kWG, kThreads = 128 + kCompute;  // warp 0: stage producer (lane 0) and tile loader (lane 1); warps 1, 2, 3: MMA issuers (S^T; second stage; dP^T); 16 compute warps
   static constexpr uint32_t kColX = 0, kColY = 128, kColZ = 256, kColAcc0 = 384, kColAcc1 = 448;
   static constexpr int kTmemCols = 512;
   // K, V resident, ring of (Q, dO, Z, two 64-row statistic blocks) step tiles, staging (dK, dV)
@@ -49,31 +55,43 @@ enum BwdW128WaitCode {
   kWkAcc = 0x5a, kWkAccFree = 0x5b, kWkResFree = 0x5c
 };
 
-// Phase 2 of the dK/dV side for a step that may reach past the statistics that were written (ragged end of a sequence):
-// a column with p = 0 gets t = 0 explicitly instead of 0 * (dP - D), because its -D may be arbitrary bits.
-__device__ __forceinline__ void dkv_phase2_guarded(uint32_t tS, uint32_t tdP, const float *nd, const float (&p)[32]) {
-  uint32_t xp[2][16];
-  tmem_ld16(tdP, xp[0]);
+// Arithmetic of one 16-column chunk of the dK/dV side (thread <-> key row, columns = queries), Algorithm 1 lines 5-8:
+//   p = exp2(x * (alpha log2 e) - LSE log2 e),  r = BF16(p),  t = BF16(fl32[p * fl32(dP - D)]).
+// xs: the chunk's S^T words, xp: its dP^T words (loaded at the start of the step), nl / nd: the chunk's per-column
+// -LSE log2 e and -D (shared memory, same address in every lane).  With MASKED, column c is dropped when c < lim (a query
+// before this key) or c > hi (past the sequence's last query); a dropped column gets t = 0 explicitly, because its -D
+// may be arbitrary bits.  The packed operands go over the chunk's own S^T columns: r the first eight, t the last eight.
+template <bool MASKED>
+__device__ __forceinline__ void dkv_chunk(uint32_t tS, const uint32_t (&xs)[16], const uint32_t (&xp)[16], const float *nl, const float *nd,
+                                          float scale_log2, int lim, int hi) {
+  const uint64_t scale2 = f32x2(scale_log2, scale_log2);
+  uint32_t pr[8], pt[8];
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    tmem_wait_ld();
-    if (c == 0) tmem_ld16(tdP + 16, xp[1]);
-    uint32_t pt[8];
+  for (int i = 0; i < 4; ++i) {
+    const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 4 * i);   // four columns per 16-byte read
+    const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 4 * i);
+    float a[4], p[4], t[4];
+    f32x2_split(fma2(f32x2_bits(xs[4 * i], xs[4 * i + 1]), scale2, l4.x), a[0], a[1]);
+    f32x2_split(fma2(f32x2_bits(xs[4 * i + 2], xs[4 * i + 3]), scale2, l4.y), a[2], a[3]);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
-      const int col = 16 * c + 4 * i;
-      float t[4];
-      f32x2_split(mul2(f32x2(p[col], p[col + 1]), add2(f32x2_bits(xp[c][4 * i], xp[c][4 * i + 1]), d4.x)), t[0], t[1]);
-      f32x2_split(mul2(f32x2(p[col + 2], p[col + 3]), add2(f32x2_bits(xp[c][4 * i + 2], xp[c][4 * i + 3]), d4.y)), t[2], t[3]);
+    for (int e = 0; e < 4; ++e) {
+      p[e] = fast_exp2(a[e]);
+      if (MASKED && (4 * i + e < lim || 4 * i + e > hi)) p[e] = 0.f;
+    }
+    f32x2_split(mul2(f32x2(p[0], p[1]), add2(f32x2_bits(xp[4 * i], xp[4 * i + 1]), d4.x)), t[0], t[1]);
+    f32x2_split(mul2(f32x2(p[2], p[3]), add2(f32x2_bits(xp[4 * i + 2], xp[4 * i + 3]), d4.y)), t[2], t[3]);
+    if (MASKED) {
 #pragma unroll
       for (int e = 0; e < 4; ++e)
-        if (p[col + e] == 0.f) t[e] = 0.f;
-      pt[2 * i] = pack_bf16x2(t[0], t[1]);
-      pt[2 * i + 1] = pack_bf16x2(t[2], t[3]);
+        if (p[e] == 0.f) t[e] = 0.f;
     }
-    tmem_st8(tS + 16 * c + 8, pt);
+    pr[2 * i] = pack_bf16x2(p[0], p[1]);
+    pr[2 * i + 1] = pack_bf16x2(p[2], p[3]);
+    pt[2 * i] = pack_bf16x2(t[0], t[1]);
+    pt[2 * i + 1] = pack_bf16x2(t[2], t[3]);
   }
+  tmem_st8(tS, pr);
+  tmem_st8(tS + 8, pt);
 }
 
 // ============================================================================================
@@ -104,8 +122,8 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   uint8_t *sOut = sStage + S * C::kDkvStageBytes;   // staging: dK tile, then dV tile
 
   __shared__ uint64_t bar_res_full, bar_res_free, bar_q_full[S], bar_q_empty[S];
-  __shared__ uint64_t bar_s_full[2], bar_r_ready[2], bar_t_ready[2], bar_s_free[2], bar_dp_full, bar_y_free;
-  __shared__ uint64_t bar_acc_done, bar_acc_free, bar_drain[2];
+  __shared__ uint64_t bar_s_full[2], bar_rt_ready[2][2], bar_s_free[2], bar_dp_full, bar_y_free;
+  __shared__ uint64_t bar_acc_done, bar_acc_free, bar_drain[3];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -121,11 +139,11 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   if (threadIdx.x == 0) {
     cta_abort = 0;
     mbar_init(&bar_res_full, 1);
-    mbar_init(&bar_res_free, 1);   // the last score product alone: the epilogue has its own staging buffer and never touches K / V
+    mbar_init(&bar_res_free, 2);   // the last S^T product (issuer 1) and the last dP^T product (issuer 2): the epilogue never touches K / V
     for (int s = 0; s < S; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_s_full[b], 1); mbar_init(&bar_s_free[b], 1);
-      mbar_init(&bar_r_ready[b], C::kCompute); mbar_init(&bar_t_ready[b], C::kCompute);
+      mbar_init(&bar_rt_ready[b][0], C::kCompute); mbar_init(&bar_rt_ready[b][1], C::kCompute);
     }
     mbar_init(&bar_dp_full, 1);
     mbar_init(&bar_y_free, C::kCompute);
@@ -133,6 +151,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     mbar_init(&bar_acc_free, C::kCompute);
     mbar_init(&bar_drain[0], 1);
     mbar_init(&bar_drain[1], 1);
+    mbar_init(&bar_drain[2], 1);
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc(&tmem_base_smem, C::kTmemCols); tmem_relinquish(); }
@@ -226,18 +245,42 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
           umma_commit(&bar_s_full[sb]);
         }
         __syncwarp();
-        if (g >= 1) mbar_wait(&bar_y_free, (g - 1) & 1, ab, kWkYFree);               // phase 2 of step g - 1 has read dP^T
+        if (n == T - 1) {
+          if (elect_one_sync()) umma_commit(&bar_res_free);   // first of two arrivals: no score product reads this K tile any more
+          __syncwarp();
+        }
+      }
+    }
+    drain_mmas_if_aborted(&bar_drain[0], ab);
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- tensor-core issuer 3: dP^T = V dO^T
+    // A warp of its own: the tensor core takes its work in the order it is issued and an issuing thread is held for as
+    // long as its products execute, so dP^T of step g + 1 -- which the ALUs want the moment they finish step g, and which
+    // may be written as soon as they hold dP^T of step g in registers -- must neither wait behind this step's S^T (whose
+    // buffer frees late) in one thread's program order nor behind the second-stage products in another's.
+    constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
+    const SmemDesc dscV = make_smem_desc(smem_u32(sV), 16, 1024);
+    const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);
+    int g = 0, ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int T = G * steps_of(tile_of(lin));
+      mbar_wait(&bar_res_full, ti & 1, ab, kWkRes);
+      for (int n = 0; n < T; ++n, ++g) {
+        const int st = g % S;
+        mbar_wait(&bar_q_full[st], (g / S) & 1, ab, kWkQ);
+        if (g >= 1) mbar_wait(&bar_y_free, (g - 1) & 1, ab, kWkYFree);               // the ALUs hold dP^T of step g - 1 in registers
         tc_fence_after();
+        const SmemDesc dscdO = dscQ0.advanced(st * C::kDkvStageBytes + C::kTileBytes);
         if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) umma_ss(tmem_base + C::kColY, dscV.at(k * 32), dscdO.at(k * 32), idesc_s, k > 0);
           umma_commit(&bar_dp_full);
-          if (n == T - 1) umma_commit(&bar_res_free);   // no MMA reads this K / V tile any more
+          if (n == T - 1) umma_commit(&bar_res_free);   // second of two arrivals: no product reads this V tile any more
         }
         __syncwarp();
       }
     }
-    drain_mmas_if_aborted(&bar_drain[0], ab);
+    drain_mmas_if_aborted(&bar_drain[2], ab);
   } else if (warp == 2) {
     // ---------------------------------------------------------------- tensor-core issuer 2: [dV | dK] += r^T [dO | Z], then dK += t^T Q
     constexpr uint32_t idesc_a = idesc_bf16_f32(128, D, 0, 1);         // [128 keys] x [d], contraction over 128 queries
@@ -250,79 +293,94 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       for (int p = 0; p < T; ++p, ++g) {
         const int st = g % S, sb = g & 1;
         const SmemDesc dscQ = dscQ0mn.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kTileBytes);
+
         // packed BF16 operands of query slice k (16 queries): r^T over columns 16 k .. 16 k + 7 of the S region, t^T over the next eight
         const uint32_t tR = tmem_base + (sb ? C::kColZ : C::kColX), tT = tR + 8;
         const uint32_t acc = (p > 0) ? 1u : 0u;
-        mbar_wait(&bar_r_ready[sb], (g >> 1) & 1, ab, kWkR);
-        tc_fence_after();
-        if (elect_one_sync()) {
-          if (use_z) {
-            // the dO and Z step tiles are adjacent 64-column atoms of one MN-major operand and the dV and dK accumulators
-            // are adjacent TMEM columns: r^T [dO | -BF16(lambda Q)] is ONE N = 128 product (Algorithm 1 lines 17-18)
+        // Every compute thread finishes the first 64 query columns of the step (k = 0..3) before the last 64, and hands
+        // the two halves over separately: the products of the first half run while the second half is in the ALUs.
 #pragma unroll
-            for (int k = 0; k < C::kStepRows / 16; ++k)
-              umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_fused, k > 0 ? 1u : acc);
-          } else {
+        for (int h = 0; h < 2; ++h) {
+          mbar_wait(&bar_rt_ready[sb][h], (g >> 1) & 1, ab, kWkR);
+          tc_fence_after();
+          if (elect_one_sync()) {
+            if (use_z) {
+              // the dO and Z step tiles are adjacent 64-column atoms of one MN-major operand and the dV and dK accumulators
+              // are adjacent TMEM columns: r^T [dO | -BF16(lambda Q)] is ONE N = 128 product (Algorithm 1 lines 17-18)
 #pragma unroll
-            for (int k = 0; k < C::kStepRows / 16; ++k)      // dV += r^T dO
-              umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+              for (int k = 4 * h; k < 4 * h + 4; ++k)
+                umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_fused, k > 0 ? 1u : acc);
+            } else {
+#pragma unroll
+              for (int k = 4 * h; k < 4 * h + 4; ++k)      // dV += r^T dO
+                umma_ts(tmem_base + C::kColAcc0, tR + 16 * k, dscdO.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
+            }
+            const uint32_t acc_k = use_z ? 1u : acc;         // with the correction, dK already holds this step's r^T Z
+#pragma unroll
+            for (int k = 4 * h; k < 4 * h + 4; ++k)          // dK += t^T Q
+              umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc_k);
+            if (h == 1) {
+              umma_commit(&bar_s_free[sb]);
+              umma_commit(&bar_q_empty[st]);
+              if (p == T - 1) umma_commit(&bar_acc_done);
+            }
           }
+          __syncwarp();
         }
-        __syncwarp();
-        mbar_wait(&bar_t_ready[sb], (g >> 1) & 1, ab, kWkT);
-        tc_fence_after();
-        if (elect_one_sync()) {
-          const uint32_t acc_k = use_z ? 1u : acc;           // with the correction, dK already holds this step's r^T Z
-#pragma unroll
-          for (int k = 0; k < C::kStepRows / 16; ++k)        // dK += t^T Q
-            umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc_k);
-          umma_commit(&bar_s_free[sb]);
-          umma_commit(&bar_q_empty[st]);
-          if (p == T - 1) umma_commit(&bar_acc_done);
-        }
-        __syncwarp();
       }
     }
     drain_mmas_if_aborted(&bar_drain[1], ab);
   } else {
     // ---------------------------------------------------------------- compute: thread <-> (key row, 32-query slice of every step)
-    const int wg = (warp - 3) >> 2;
+    const int wg = (warp - 4) >> 2;
     const int row = 32 * (warp & 3) + lane;                  // key row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>(32 * (warp & 3)) << 16;
-    const uint32_t slice_addr = tmem_base + lane_addr + C::kSliceCols * wg;
     int g0 = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const TileInfo tl = tile_of(lin);
       const int bh = hix(lin), Th = steps_of(tl), T = G * Th, q_start = q_start_of(tl);
-      // (Issuing the first TMEM load of a phase early, when its barrier had already completed, and letting warpgroup pairs
-      // take turns in phase 1, were both measured slower.)
       for (int n = 0; n < T; ++n) {
         const int g = g0 + n, st = g % S, sb = g & 1;
-        const uint32_t tS = slice_addr + (sb ? C::kColZ : C::kColX), tdP = slice_addr + C::kColY;
+        // This thread's two 16-column chunks: columns 16 w .. 16 w + 15 of the step's first 64 queries, then of its last 64
+        // (operand slices k = w and k = 4 + w).
+        const int cb = 16 * wg;
+        const uint32_t tS0 = tmem_base + lane_addr + (sb ? C::kColZ : C::kColX) + 16 * wg, tS1 = tS0 + 64;
+        const uint32_t tdP0 = tmem_base + lane_addr + C::kColY + 16 * wg, tdP1 = tdP0 + 64;
         // The scores of this step were issued after its stage (and with it the row statistics) had landed in shared
-        // memory, so their completion covers both.  Slice w of the 128 columns lies in statistic block w / 2.
-        const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kTileBytes) + (wg >> 1) * 128 + (wg & 1) * 32;
+        // memory, so their completion covers both.  The first 64 columns lie in statistic block 0, the last 64 in block 1:
+        // {64 x -LSE log2 e, 64 x -D} each.
+        const float *st0 = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kTileBytes) + 16 * wg, *st1 = st0 + 128;
+        constexpr int kChunk1 = 64;
         const int nh = n % Th;                                              // step within the current query head
         const int Lq = tl.oseq_end - tl.oseq0, off = (tl.seq_end - tl.seq0) - Lq, krel0 = tl.row0 - tl.seq0;
         const int qs = q_start + nh * C::kStepRows;                         // first query (inside its sequence) of the step
-        const int q0 = qs + C::kSliceCols * wg;                             // ... of the slice's column 0
+        const int q0 = qs + cb;                                             // ... of this thread's first chunk
         const bool masked = (CAUSAL && qs < krel0 + 128 - off) || qs + C::kStepRows > Lq;
-        float pkeep[32];
+        const int lim = CAUSAL ? krel0 + row - off - q0 : 0, hi = Lq - 1 - q0;
+        // dP^T of both chunks and S^T of the first go to registers at the start of the step; dP^T (single-buffered) is then
+        // released to the tensor core.
         mbar_wait(&bar_s_full[sb], (g >> 1) & 1, ab, kWkS);
-        tc_fence_after();
-        if (masked) dkv_phase1<true>(tS, nl, scale_log2, CAUSAL ? krel0 + row - off - q0 : 0, Lq - 1 - q0, pkeep);
-        else        dkv_phase1<false>(tS, nl, scale_log2, 0, 0, pkeep);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(&bar_r_ready[sb]);
         mbar_wait(&bar_dp_full, g & 1, ab, kWkDP);
         tc_fence_after();
-        if (masked) dkv_phase2_guarded(tS, tdP, nl + 64, pkeep);
-        else        dkv_phase2(tS, tdP, nl + 64, pkeep);
+        uint32_t xp[32], xs[16];
+        tmem_ld16(tdP0, *reinterpret_cast<uint32_t (*)[16]>(&xp[0]));
+        tmem_ld16(tdP1, *reinterpret_cast<uint32_t (*)[16]>(&xp[16]));
+        tmem_ld16(tS0, xs);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&bar_y_free);                   // dP^T is in registers: the tensor core may write the next step's
+        if (masked) dkv_chunk<true>(tS0, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[0]), st0, st0 + 64, scale_log2, lim, hi);
+        else        dkv_chunk<false>(tS0, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[0]), st0, st0 + 64, scale_log2, 0, 0);
+        tmem_ld16(tS1, xs);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&bar_y_free);                      // dP^T of this step has been read: the next one may be computed
-        mbar_arrive(&bar_t_ready[sb]);
+        mbar_arrive(&bar_rt_ready[sb][0]);
+        tmem_wait_ld();
+        if (masked) dkv_chunk<true>(tS1, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[16]), st1, st1 + 64, scale_log2, lim - kChunk1, hi - kChunk1);
+        else        dkv_chunk<false>(tS1, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[16]), st1, st1 + 64, scale_log2, 0, 0);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bar_rt_ready[sb][1]);
       }
 
       mbar_wait(&bar_acc_done, ti & 1, ab, kWkAcc);
@@ -334,7 +392,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&bar_acc_free);          // the accumulators may be overwritten by the next tile
-      if (threadIdx.x == 96) bulk_wait_group_read0();   // the previous tile's stores have left the staging buffer
+      if (threadIdx.x == 128) bulk_wait_group_read0();   // the previous tile's stores have left the staging buffer
       named_bar_sync(1, C::kCompute);
 #pragma unroll
       for (int v = 0; v < 2; ++v) {
@@ -352,7 +410,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       fence_proxy_async_smem();
       named_bar_sync(1, C::kCompute);
       if (tile_store_by_tma(tl, N)) {
-        if (threadIdx.x == 96) {
+        if (threadIdx.x == 128) {
           tma_store_3d(&tmdV, stage_dv, 0, tl.row0, bh);
           tma_store_3d(&tmdK, stage_dk, 0, tl.row0, bh);
           bulk_commit_group();
@@ -365,7 +423,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       }
       g0 += T;
     }
-    if (threadIdx.x == 96) bulk_wait_group_read0();
+    if (threadIdx.x == 128) bulk_wait_group_read0();
   }
 
   tc_fence_before();

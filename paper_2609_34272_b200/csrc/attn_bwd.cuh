@@ -315,7 +315,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   uint8_t *sO = sOut + (C::kSepStaging ? 2 * C::kBigTileBytes : 0);   // saved-output rows of the next tile (kPrefetchO), row-major
 
   __shared__ uint64_t bar_res_full[R], bar_res_free[R], bar_kv_full[S], bar_kv_empty[S];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_acc_done, bar_acc_free, bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
   __shared__ float s_rho[C::kWG - 1][128], s_m[C::kWG - 1][128], s_lam[128], s_D[128], s_lse[128];
@@ -332,7 +332,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     cta_abort = 0;
     for (int r = 0; r < R; ++r) { mbar_init(&bar_res_full[r], 1); mbar_init(&bar_res_free[r], 2); }
     for (int s = 0; s < S; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
-    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128 * C::kSlices); mbar_init(&bar_buf_free[b], 1); }
+    for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128 * C::kSlices); }
     mbar_init(&bar_acc_done, 1);
     mbar_init(&bar_acc_free, C::kCompute);
     mbar_init(&bar_drain[0], 1);
@@ -426,7 +426,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       for (int n = 0; n < T; ++n, ++g) {
         const int st = g % S, b = g % NB;
         mbar_wait(&bar_kv_full[st], (g / S) & 1, ab, kDqWaitKV);
-        if (g >= NB) mbar_wait(&bar_buf_free[b], ((g / NB) - 1) & 1, ab, kDqWaitBuf);   // r, t of step g - NB consumed
+        // r, t of step g - NB consumed: that step's second-stage products are complete.  One commit per step serves this
+        // wait and the stage ring's (every commit costs the tensor pipe some forty cycles in this stream of short products).
+        if (g >= NB) mbar_wait(&bar_kv_empty[(g - NB) % S], ((g - NB) / S) & 1, ab, kDqWaitBuf);
         tc_fence_after();
         const SmemDesc dscK = dscK0.advanced(st * C::kDqStageBytes), dscV = dscK.advanced(C::kStepTileBytes);
         const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
@@ -471,8 +473,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)
             umma_ts(tmem_base + C::kColAcc1, tR + 16 * k, dscK.at(k * 2048), idesc_a, k > 0 ? 1u : acc);
-          umma_commit(&bar_buf_free[b]);
-          umma_commit(&bar_kv_empty[st]);
+          umma_commit(&bar_kv_empty[st]);                   // step done: its stage and its score buffer are free
           if (p == T - 1) umma_commit(&bar_acc_done);
         }
         __syncwarp();
@@ -714,7 +715,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   uint8_t *sOut = sStage + S * C::kDkvStageBytes;   // staging (dK tile, then dV tile) when separate
 
   __shared__ uint64_t bar_res_full, bar_res_free, bar_q_full[S], bar_q_empty[S];
-  __shared__ uint64_t bar_s_full[NB], bar_dp_full[NB], bar_r_ready[NB], bar_t_ready[NB], bar_buf_free[NB], bar_acc_done, bar_acc_free, bar_drain[2];
+  __shared__ uint64_t bar_s_full[NB], bar_dp_full[NB], bar_r_ready[NB], bar_t_ready[NB], bar_acc_done, bar_acc_free, bar_drain[2];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
 
@@ -733,7 +734,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     mbar_init(&bar_res_free, 2);
     for (int s = 0; s < S; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
     for (int b = 0; b < NB; ++b) {
-      mbar_init(&bar_s_full[b], 1); mbar_init(&bar_dp_full[b], 1); mbar_init(&bar_buf_free[b], 1);
+      mbar_init(&bar_s_full[b], 1); mbar_init(&bar_dp_full[b], 1);
       mbar_init(&bar_r_ready[b], 128 * C::kSlices); mbar_init(&bar_t_ready[b], 128 * C::kSlices);
     }
     mbar_init(&bar_acc_done, 1);
@@ -828,7 +829,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       for (int n = 0; n < T; ++n, ++g) {
         const int st = g % S, b = g % NB;
         mbar_wait(&bar_q_full[st], (g / S) & 1, ab, kDkvWaitQ);
-        if (g >= NB) mbar_wait(&bar_buf_free[b], ((g / NB) - 1) & 1, ab, kDkvWaitBuf);   // r, t of step g - NB consumed
+        if (g >= NB) mbar_wait(&bar_q_empty[(g - NB) % S], ((g - NB) / S) & 1, ab, kDkvWaitBuf);   // step g - NB done: its r, t are consumed
         tc_fence_after();
         const SmemDesc dscQ = dscQ0.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kStepTileBytes);
         const uint32_t tS = tmem_base + 128 * b, tdP = tS + 64;
@@ -896,8 +897,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
 #pragma unroll
           for (int k = 0; k < C::kStepRows / 16; ++k)        // dK += t^T Q
             umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc_k);
-          umma_commit(&bar_buf_free[b]);
-          umma_commit(&bar_q_empty[st]);
+          umma_commit(&bar_q_empty[st]);                    // step done: its stage and its score buffer are free
           if (p == T - 1) umma_commit(&bar_acc_done);
         }
         __syncwarp();

@@ -122,7 +122,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   uint8_t *sOut = sStage + S * C::kDkvStageBytes;   // staging: dK tile, then dV tile
 
   __shared__ uint64_t bar_res_full, bar_res_free, bar_q_full[S], bar_q_empty[S];
-  __shared__ uint64_t bar_s_full[2], bar_rt_ready[2][2], bar_s_free[2], bar_dp_full, bar_y_free;
+  __shared__ uint64_t bar_s_full[2], bar_rt_ready[2][2], bar_dp_full, bar_y_free;
   __shared__ uint64_t bar_acc_done, bar_acc_free, bar_drain[3];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
@@ -142,7 +142,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     mbar_init(&bar_res_free, 2);   // the last S^T product (issuer 1) and the last dP^T product (issuer 2): the epilogue never touches K / V
     for (int s = 0; s < S; ++s) { mbar_init(&bar_q_full[s], 1); mbar_init(&bar_q_empty[s], 1); }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&bar_s_full[b], 1); mbar_init(&bar_s_free[b], 1);
+      mbar_init(&bar_s_full[b], 1);
       mbar_init(&bar_rt_ready[b][0], C::kCompute); mbar_init(&bar_rt_ready[b][1], C::kCompute);
     }
     mbar_init(&bar_dp_full, 1);
@@ -235,7 +235,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       for (int n = 0; n < T; ++n, ++g) {
         const int st = g % S, sb = g & 1;
         mbar_wait(&bar_q_full[st], (g / S) & 1, ab, kWkQ);
-        if (g >= 2) mbar_wait(&bar_s_free[sb], ((g >> 1) - 1) & 1, ab, kWkSFree);   // r, t of step g - 2 consumed
+        if (g >= 2) mbar_wait(&bar_q_empty[(g - 2) % S], ((g - 2) / S) & 1, ab, kWkSFree);   // step g - 2 done: its r, t are consumed
         tc_fence_after();
         const SmemDesc dscQ = dscQ0.advanced(st * C::kDkvStageBytes), dscdO = dscQ.advanced(C::kTileBytes);
         const uint32_t tS = tmem_base + (sb ? C::kColZ : C::kColX);
@@ -320,8 +320,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
             for (int k = 4 * h; k < 4 * h + 4; ++k)          // dK += t^T Q
               umma_ts(tmem_base + C::kColAcc1, tT + 16 * k, dscQ.at(k * 2048), idesc_a, k > 0 ? 1u : acc_k);
             if (h == 1) {
-              umma_commit(&bar_s_free[sb]);
-              umma_commit(&bar_q_empty[st]);
+              umma_commit(&bar_q_empty[st]);               // step done: its stage and its S^T buffer are free
               if (p == T - 1) umma_commit(&bar_acc_done);
             }
           }

@@ -431,6 +431,24 @@ def main():
             "bwd_frac_of_bf16_peak": 7 * unit_p / bp / 1e12 / burst, "fwd_tflops": 2 * unit_p / fp / 1e12,
             "note": "timed with output allocation inside the call (binding allocates O, LSE, dQ, dK, dV, workspace)"}
 
+    if rank == 0 and not args.no_extras and args.workload == 2 and args.shard == "replicas":
+        # the paper's fused FP32 comparison arm on the same workload (plain FP32 arithmetic on the CUDA cores), for context
+        saved = torch.empty(g.binding.load().gproj_fp32_attn_saved_bytes(w.B, w.H, w.N, w.d), dtype=torch.uint8, device=dev)
+
+        def body32(ev):
+            ev[0].record(stream); g.gproj_fp32_attn_fwd(d_in["Q"], d_in["K"], d_in["V"], a, c, saved=saved); ev[1].record(stream)
+            ev[2].record(stream); g.gproj_fp32_attn_bwd(d_in["Q"], d_in["K"], d_in["V"], d_in["dO"], saved, a, c); ev[3].record(stream)
+
+        for _ in range(2):
+            body32([torch.cuda.Event(enable_timing=True) for _ in range(4)])
+        e32, _ = timed_steps(5, body32)
+        f32 = sum(e[0].elapsed_time(e[1]) for e in e32) / 5
+        b32 = sum(e[2].elapsed_time(e[3]) for e in e32) / 5
+        line["also"]["fused_fp32_arm_" + w.name] = {
+            "fwd_ms": f32, "bwd_ms": b32, "bwd_tflops_5unit": fl["bwd5"] / (b32 / 1e3) / 1e12, "fwd_tflops": fl["fwd"] / (f32 / 1e3) / 1e12,
+            "step_ms_ratio_to_tensor_core_path": (f32 + b32) / ((fwd_ms + bwd_ms) / steps),
+            "note": "comparison arm: FP32 FMAs on the CUDA cores, FP32 saved output; the paper's fused FP32 attention cost its training step +33 %"}
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         b = {k: bits(v) for k, v in host.items()}

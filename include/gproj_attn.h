@@ -246,6 +246,25 @@ int gproj_attn_bwd_static_scratch(const void *Q, const void *K, const void *V, c
                                   unsigned flags, void *stream);
 
 /*
+ * Fused FP32 attention, the paper's "fused FP32" comparison arm (Appendix "Accuracy and Cost", paragraph "Fused FP32
+ * baseline"; Table "method-definitions", row "FP32 attention"): the BF16 inputs are decoded and every product, the
+ * softmax (Eq. "row-attention") and the gradients (Eq. "row-gradients") are computed in FP32 fused multiply-adds on the
+ * CUDA cores (no tensor core, no TF32); outputs and gradients are returned in BF16.  The forward saves an FP32 output
+ * and three FP32 row statistics (log-sum-exp, row maximum of the scaled scores, inverse normaliser); the backward
+ * recomputes P = exp(s - max) / l tile by tile and takes D = rowsum(dO * O) from the FP32 output.  Nothing of size N^2 is
+ * stored.  A baseline to compare accuracy and cost with, an order of magnitude slower than the tensor-core path.
+ *   Q, K, V, dO, O, dQ, dK, dV: DEVICE BF16 [B][H][N][d] (one head count; d in {64, 128}; any N >= 1); causal as above.
+ *   saved: DEVICE scratch, 256-byte aligned, gproj_fp32_attn_saved_bytes() bytes, written by the forward and read (its
+ *   row-term part also written) by the backward of the same problem; GPROJ_ERR_WORKSPACE if NULL, misaligned or short.
+ *   Other errors as for gproj_attn_fwd.  One launch (forward) / two launches (backward) on `stream`.
+ */
+size_t gproj_fp32_attn_saved_bytes(int B, int H, int N, int d);
+int gproj_fp32_attn_fwd(const void *Q, const void *K, const void *V, void *O, void *saved, size_t saved_bytes,
+                        int B, int H, int N, int d, float softmax_scale, int causal, void *stream);
+int gproj_fp32_attn_bwd(const void *Q, const void *K, const void *V, const void *dO, void *saved, size_t saved_bytes,
+                        void *dQ, void *dK, void *dV, int B, int H, int N, int d, float softmax_scale, int causal, void *stream);
+
+/*
  * Key smoothing, the comparison arm of Section 5.1 and of Table "method-definitions" ("FA3 on mean-subtracted keys"):
  * subtract the per-sequence, per-KV-head mean row, Y_j = BF16(fl32(X_j - mean_j X_j)), mean and subtraction in FP32.
  * The arm is built from calls of this library: K~ = gproj_key_smooth(K); the forward on (Q, K~, V) with

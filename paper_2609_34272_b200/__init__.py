@@ -21,6 +21,8 @@ from .binding import (  # noqa: F401
     gproj_attn_fwd_bwd_host,
     gproj_attn_fwd_rect,
     gproj_attn_host_staging_bytes,
+    gproj_fp32_attn_bwd,
+    gproj_fp32_attn_fwd,
     gproj_key_smooth,
     gproj_attn_fwd_varlen,
     gproj_attn_fwd_varlen_qk,

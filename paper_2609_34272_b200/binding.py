@@ -27,6 +27,7 @@ EXPORTS = ("gproj_attn_fwd", "gproj_attn_bwd_workspace_bytes", "gproj_attn_bwd",
            "gproj_attn_bwd_varlen_workspace_bytes", "gproj_attn_bwd_varlen",
            "gproj_attn_varlen_qk_plan_bytes", "gproj_attn_varlen_qk_plan", "gproj_attn_fwd_varlen_qk", "gproj_attn_bwd_varlen_qk",
            "gproj_attn_host_staging_bytes", "gproj_attn_fwd_bwd_host", "gproj_key_smooth", "gproj_key_smooth_varlen",
+           "gproj_fp32_attn_saved_bytes", "gproj_fp32_attn_fwd", "gproj_fp32_attn_bwd",
            "gproj_last_device_status", "gproj_selftest_wait_timeout",
            "gproj_status_string", "gproj_last_launch_count")
 
@@ -89,6 +90,12 @@ def load():
         lib.gproj_attn_host_staging_bytes.argtypes = [i, i, i, i, i]
         lib.gproj_attn_fwd_bwd_host.restype = i
         lib.gproj_attn_fwd_bwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp, ctypes.c_size_t, u, vp]
+        lib.gproj_fp32_attn_saved_bytes.restype = sz
+        lib.gproj_fp32_attn_saved_bytes.argtypes = [i, i, i, i]
+        lib.gproj_fp32_attn_fwd.restype = i
+        lib.gproj_fp32_attn_fwd.argtypes = [vp, vp, vp, vp, vp, sz, i, i, i, i, f, i, vp]
+        lib.gproj_fp32_attn_bwd.restype = i
+        lib.gproj_fp32_attn_bwd.argtypes = [vp, vp, vp, vp, vp, sz, vp, vp, vp, i, i, i, i, f, i, vp]
         lib.gproj_key_smooth.restype = i
         lib.gproj_key_smooth.argtypes = [vp, vp, i, i, i, i, vp]
         lib.gproj_key_smooth_varlen.restype = i
@@ -264,6 +271,39 @@ def gproj_attn_bwd_static_scratch(Q, K, V, O, LSE, dO, softmax_scale, causal, fl
                                                   float(softmax_scale), int(bool(causal)), int(flags), _stream(Q.device))
     if rc != GPROJ_OK:
         raise GprojError(rc, "gproj_attn_bwd_static_scratch")
+    return dQ, dK, dV
+
+
+def gproj_fp32_attn_fwd(Q, K, V, softmax_scale, causal, saved=None):
+    """O (bfloat16), saved = fused FP32 attention forward (the comparison arm; plain FP32 arithmetic on the CUDA cores)."""
+    _check_bf16("Q", Q)
+    B, H, N, d = Q.shape
+    _check_bf16("K", K, Q.shape); _check_bf16("V", V, Q.shape)
+    need = int(load().gproj_fp32_attn_saved_bytes(B, H, N, d))
+    if saved is None:
+        saved = torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device)
+    O = torch.empty_like(Q)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_fp32_attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), saved.data_ptr(), saved.numel(),
+                                        B, H, N, d, float(softmax_scale), int(bool(causal)), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_fp32_attn_fwd")
+    return O, saved
+
+
+def gproj_fp32_attn_bwd(Q, K, V, dO, saved, softmax_scale, causal):
+    """dQ, dK, dV (bfloat16) = fused FP32 attention backward from the state gproj_fp32_attn_fwd saved."""
+    _check_bf16("Q", Q)
+    B, H, N, d = Q.shape
+    for name, t in (("K", K), ("V", V), ("dO", dO)):
+        _check_bf16(name, t, Q.shape)
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(Q), torch.empty_like(Q)
+    with torch.cuda.device(Q.device):
+        rc = load().gproj_fp32_attn_bwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), dO.data_ptr(), saved.data_ptr(), saved.numel(),
+                                        dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), B, H, N, d, float(softmax_scale),
+                                        int(bool(causal)), _stream(Q.device))
+    if rc != GPROJ_OK:
+        raise GprojError(rc, "gproj_fp32_attn_bwd")
     return dQ, dK, dV
 
 

@@ -8,7 +8,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgproj_attn.so")
 SOURCES = [os.path.join(CSRC, "gproj_attn.cu")]
-HEADERS = [os.path.join(CSRC, f) for f in ("sm100_primitives.cuh", "attn_fwd.cuh", "attn_bwd.cuh", "attn_bwd_w128.cuh", "key_smoothing.cuh")] + \
+HEADERS = [os.path.join(CSRC, f) for f in ("sm100_primitives.cuh", "attn_fwd.cuh", "attn_bwd.cuh", "attn_bwd_w128.cuh", "key_smoothing.cuh", "attn_fp32.cuh")] + \
           [os.path.join(ROOT, "include", "gproj_attn.h")]
 
 

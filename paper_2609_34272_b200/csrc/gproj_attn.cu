@@ -14,6 +14,7 @@
 #include "attn_bwd_w128.cuh"
 #include "attn_fwd.cuh"
 #include "key_smoothing.cuh"
+#include "attn_fp32.cuh"
 
 namespace {
 
@@ -858,6 +859,76 @@ const char *gproj_status_string(int status) {
 }
 
 int gproj_last_launch_count(void) { return tl_launch_count; }
+
+// ---- fused FP32 attention (comparison arm; plain SIMT arithmetic) ------------------------------------------------------
+size_t gproj_fp32_attn_saved_bytes(int B, int H, int N, int d) {
+  if (check_shape(B, H, N, d) != GPROJ_OK) return 0;
+  const size_t rows = static_cast<size_t>(B) * H * N;
+  return (rows * static_cast<size_t>(d) + 4 * rows) * sizeof(float);     // O32, then lse / max / 1 / l per row, then D
+}
+
+static int fp32_common(const void *const *ptrs, int n_ptrs, void *saved, size_t saved_bytes, int B, int H, int N, int d, float scale) {
+  for (int i = 0; i < n_ptrs; ++i) if (!ptrs[i]) return GPROJ_ERR_NULL;
+  if (int rc = check_shape(B, H, N, d)) return rc;
+  for (int i = 0; i < n_ptrs; ++i) if (!aligned16(ptrs[i])) return GPROJ_ERR_ALIGN;
+  if (!std::isfinite(scale) || !(scale > 0.f)) return GPROJ_ERR_SCALE;
+  if (!saved || (reinterpret_cast<uintptr_t>(saved) & 255u) || saved_bytes < gproj_fp32_attn_saved_bytes(B, H, N, d)) return GPROJ_ERR_WORKSPACE;
+  return GPROJ_OK;
+}
+
+int gproj_fp32_attn_fwd(const void *Q, const void *K, const void *V, void *O, void *saved, size_t saved_bytes,
+                        int B, int H, int N, int d, float softmax_scale, int causal, void *stream) {
+  const void *ptrs[4] = {Q, K, V, O};
+  if (int rc = fp32_common(ptrs, 4, saved, saved_bytes, B, H, N, d, softmax_scale)) return rc;
+  DeviceState *st = nullptr;
+  if (int rc = device_state(&st)) return rc;
+  const size_t rows = static_cast<size_t>(B) * H * N;
+  float *O32 = static_cast<float *>(saved), *stats = O32 + rows * d;
+  const dim3 grid(static_cast<unsigned>((N + 63) / 64), static_cast<unsigned>(B * H));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  auto q = static_cast<const __nv_bfloat16 *>(Q); auto k = static_cast<const __nv_bfloat16 *>(K); auto v = static_cast<const __nv_bfloat16 *>(V);
+  auto o = static_cast<__nv_bfloat16 *>(O);
+#define GPROJ_FP32_FWD(DD, CC)                                                                                     \
+  do {                                                                                                             \
+    if (cudaFuncSetAttribute(fp32_attn_fwd_kernel<DD, CC>, cudaFuncAttributeMaxDynamicSharedMemorySize, Fp32Cfg<DD>::kFwdSmem) != cudaSuccess) \
+      return GPROJ_ERR_CUDA;                                                                                       \
+    fp32_attn_fwd_kernel<DD, CC><<<grid, 128, Fp32Cfg<DD>::kFwdSmem, s>>>(q, k, v, o, O32, stats, N, softmax_scale); \
+  } while (0)
+  if (d == 64) { if (causal) GPROJ_FP32_FWD(64, true); else GPROJ_FP32_FWD(64, false); }
+  else         { if (causal) GPROJ_FP32_FWD(128, true); else GPROJ_FP32_FWD(128, false); }
+#undef GPROJ_FP32_FWD
+  if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
+  tl_launch_count = 1;
+  return GPROJ_OK;
+}
+
+int gproj_fp32_attn_bwd(const void *Q, const void *K, const void *V, const void *dO, void *saved, size_t saved_bytes,
+                        void *dQ, void *dK, void *dV, int B, int H, int N, int d, float softmax_scale, int causal, void *stream) {
+  const void *ptrs[7] = {Q, K, V, dO, dQ, dK, dV};
+  if (int rc = fp32_common(ptrs, 7, saved, saved_bytes, B, H, N, d, softmax_scale)) return rc;
+  DeviceState *st = nullptr;
+  if (int rc = device_state(&st)) return rc;
+  const size_t rows = static_cast<size_t>(B) * H * N;
+  float *O32 = static_cast<float *>(saved), *stats = O32 + rows * d, *Drow = stats + 3 * rows;
+  const dim3 grid(static_cast<unsigned>((N + 63) / 64), static_cast<unsigned>(B * H));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  auto q = static_cast<const __nv_bfloat16 *>(Q); auto k = static_cast<const __nv_bfloat16 *>(K); auto v = static_cast<const __nv_bfloat16 *>(V);
+  auto u = static_cast<const __nv_bfloat16 *>(dO);
+#define GPROJ_FP32_BWD(DD, CC)                                                                                     \
+  do {                                                                                                             \
+    if (cudaFuncSetAttribute(fp32_attn_dq_kernel<DD, CC>, cudaFuncAttributeMaxDynamicSharedMemorySize, Fp32Cfg<DD>::kBwdSmem) != cudaSuccess || \
+        cudaFuncSetAttribute(fp32_attn_dkv_kernel<DD, CC>, cudaFuncAttributeMaxDynamicSharedMemorySize, Fp32Cfg<DD>::kBwdSmem) != cudaSuccess) \
+      return GPROJ_ERR_CUDA;                                                                                       \
+    fp32_attn_dq_kernel<DD, CC><<<grid, 128, Fp32Cfg<DD>::kBwdSmem, s>>>(q, k, v, u, O32, stats, Drow, static_cast<__nv_bfloat16 *>(dQ), N, softmax_scale); \
+    fp32_attn_dkv_kernel<DD, CC><<<grid, 128, Fp32Cfg<DD>::kBwdSmem, s>>>(q, k, v, u, stats, Drow, static_cast<__nv_bfloat16 *>(dK), static_cast<__nv_bfloat16 *>(dV), N, softmax_scale); \
+  } while (0)
+  if (d == 64) { if (causal) GPROJ_FP32_BWD(64, true); else GPROJ_FP32_BWD(64, false); }
+  else         { if (causal) GPROJ_FP32_BWD(128, true); else GPROJ_FP32_BWD(128, false); }
+#undef GPROJ_FP32_BWD
+  if (cudaGetLastError() != cudaSuccess) return GPROJ_ERR_CUDA;
+  tl_launch_count = 2;
+  return GPROJ_OK;
+}
 
 // ---- key smoothing (comparison arm of Section 5.1): subtract the per-sequence, per-head mean row -------------------
 static int smooth_rows(const void *X, void *Y, int heads, long long rows_total, int d, const int *cu_seqlens, int num_seqs,

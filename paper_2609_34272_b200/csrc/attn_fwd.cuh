@@ -329,6 +329,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         continue;
       }
       float m_run = -INFINITY, l_run = 0.f;
+#ifdef GPROJ_TRACE
+      const unsigned long long ev_n0 = global_ns(); const long long ev_c0 = clock64();
+#endif
       // Both tiles of the pair exist: the warpgroups alternate in the exponential phase, step by step, tile 0 first.
       const bool take_turns = TURNS && it.nq == 2;
       const int cnt_item0 = cnt;
@@ -412,6 +415,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_arrive(&bar_p_ready[t]);
         ++cnt;
       }
+#ifdef GPROJ_TRACE
+      const unsigned long long ev_n2 = global_ns();
+#endif
       // ---- epilogue: O = BF16(acc / l) staged in the TMA layout over this tile's Q, LSE = alpha x_max + ln l
       if (cnt > cnt_item0) { mbar_wait(&bar_pv_done[t], (cnt - 1) & 1, ab, kFwdWaitPV); tc_fence_after(); }
       if (split && t == 1) {
@@ -424,6 +430,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         s_l1[ti & 1][row] = l_run;
         tc_fence_before();
         mbar_arrive(&bar_merge);
+#ifdef GPROJ_TRACE
+        if (row == 0) tile_event(21, lin, T, ev_n0, ev_n0, ev_n2, global_ns(), ev_c0, clock64());
+#endif
         continue;
       }
       // Split mode: O = (O_0 s_0 + O_1 s_1) / (l_0 s_0 + l_1 s_1) with s_t = exp2((m_t - max(m_0, m_1)) alpha log2 e).
@@ -488,6 +497,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         named_bar_sync(1 + t, 128);
         if (row == 0) mbar_arrive(&bar_q_free[qb]);
       }
+#ifdef GPROJ_TRACE
+      if (row == 0) tile_event(20 + t, lin, T, ev_n0, ev_n0, ev_n2, global_ns(), ev_c0, clock64());
+#endif
     }
   }
 

@@ -164,6 +164,9 @@ __device__ __forceinline__ void store_rows_clipped(const uint8_t *stage, int sla
   }
 }
 
+// Bytes of one 64-row block of the d = 64 row-constant tile (64 rows x 16 BF16 columns).
+constexpr int kExtBlockBytes = 2048;
+
 enum BwdWaitCode {
   kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26, kDqWaitBuf = 0x27, kDqWaitResFree = 0x28, kDqWaitAccFree = 0x29,
   kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36, kDkvWaitBuf = 0x37, kDkvWaitResFree = 0x38, kDkvWaitAccFree = 0x39
@@ -557,9 +560,27 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       // Per 64-row block of a sequence (the last one padded with zeros): 64 x {-LSE log2 e}, then 64 x {-D}.
       const int rel = qrow - tl.seq0;                  // row inside the sequence
       if (wg == 0 && rel < ((tl.seq_end - tl.seq0 + C::kStepRows - 1) / C::kStepRows) * C::kStepRows) {
-        float *blk = stats + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * 128 + (rel & 63);
-        blk[0] = neg_lse2;
-        blk[64] = -Dv;
+        if (D == 64) {
+          // d = 64: the dK/dV side takes both row constants through its score products instead of reading them per
+          // column.  Per 64-row block a K-major operand tile of 16 BF16 columns without swizzle (eight-row groups of 256
+          // bytes: the rows' first eight columns, then their last eight): columns 0..2 hold -LSE / alpha and columns
+          // 8..10 hold -D, each as three BF16 pieces whose sum is the FP32 value, the other columns zero.  A row with an
+          // empty support (LSE = +inf) gets a large finite value: its probabilities are zero either way, and an
+          // infinity would turn the zero entries of the constant operand into NaN.
+          const float c = fmaxf(__fdiv_rn(neg_lse2, scale_log2), -1.0e30f), nd = -Dv;
+          const uint32_t c0 = pack_bf16x2(c, 0.f), n0 = pack_bf16x2(nd, 0.f);
+          const float c_r1 = c - bf16_lo_to_f32(c0), n_r1 = nd - bf16_lo_to_f32(n0);
+          const uint32_t c1 = pack_bf16x2(c_r1, 0.f), n1 = pack_bf16x2(n_r1, 0.f);
+          const uint32_t c2 = pack_bf16x2(c_r1 - bf16_lo_to_f32(c1), 0.f), n2 = pack_bf16x2(n_r1 - bf16_lo_to_f32(n1), 0.f);
+          uint8_t *blk = reinterpret_cast<uint8_t *>(stats) + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * kExtBlockBytes +
+                         ((rel & 63) >> 3) * 256 + (rel & 7) * 16;
+          *reinterpret_cast<uint4 *>(blk) = make_uint4(c0 | (c1 << 16), c2, 0u, 0u);
+          *reinterpret_cast<uint4 *>(blk + 128) = make_uint4(n0 | (n1 << 16), n2, 0u, 0u);
+        } else {
+          float *blk = stats + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * 128 + (rel & 63);
+          blk[0] = neg_lse2;
+          blk[64] = -Dv;
+        }
       }
 
       uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);

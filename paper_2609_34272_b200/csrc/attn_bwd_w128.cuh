@@ -44,8 +44,9 @@ struct BwdW128 {
   static constexpr int kWG = 4, kCompute = 128 * kWG, kThreads = 128 + kCompute;  // warp 0: stage producer (lane 0) and tile loader (lane 1); warps 1, 2, 3: MMA issuers (S^T; second stage; dP^T); 16 compute warps
   static constexpr uint32_t kColX = 0, kColY = 128, kColZ = 256, kColAcc0 = 384, kColAcc1 = 448;
   static constexpr int kTmemCols = 512;
-  // K, V resident, ring of (Q, dO, Z, two 64-row statistic blocks) step tiles, staging (dK, dV)
-  static constexpr int kDkvStageBytes = 3 * kTileBytes + 1024;
+  // K, V resident, ring of (Q, dO, Z, two 64-row blocks of the row-constant tile) step tiles, staging (dK, dV)
+  static constexpr int kExtBytes = 2 * kExtBlockBytes;             // 128 rows x 16 BF16 columns
+  static constexpr int kDkvStageBytes = 3 * kTileBytes + kExtBytes;
   static constexpr int kDkvSmemBytes = 2 * kTileBytes + kStages * kDkvStageBytes + 2 * kTileBytes + 1024;
   static_assert(kDkvSmemBytes <= 227 * 1024, "shared memory budget");
 };
@@ -56,30 +57,31 @@ enum BwdW128WaitCode {
 };
 
 // Arithmetic of one 16-column chunk of the dK/dV side (thread <-> key row, columns = queries), Algorithm 1 lines 5-8:
-//   p = exp2(x * (alpha log2 e) - LSE log2 e),  r = BF16(p),  t = BF16(fl32[p * fl32(dP - D)]).
-// xs: the chunk's S^T words, xp: its dP^T words (loaded at the start of the step), nl / nd: the chunk's per-column
-// -LSE log2 e and -D (shared memory, same address in every lane).  With MASKED, column c is dropped when c < lim (a query
-// before this key) or c > hi (past the sequence's last query); a dropped column gets t = 0 explicitly, because its -D
-// may be arbitrary bits.  The packed operands go over the chunk's own S^T columns: r the first eight, t the last eight.
+//   p = exp2((x - LSE / alpha) * (alpha log2 e)),  r = BF16(p),  t = BF16(fl32[p * (dP - D)]).
+// Both row constants arrive with the products: the score product carries one extra K = 16 slice whose operands are a
+// constant matrix of ones (three columns) and the step's row-constant tile, so xs holds x - LSE / alpha and xp holds
+// dP - D, accumulated in FP32 by the tensor core (the three BF16 pieces of a constant add up to its FP32 value; the
+// subtraction is rounded by the accumulator instead of by an add.rn: a different last bit at most).  Reading the
+// constants per column from shared memory instead cost this kernel 14 % (every lane needs every column's value).
+// With MASKED, column c is dropped when c < lim (a query before this key) or c > hi (past the sequence's last query);
+// a dropped column gets t = 0 explicitly, because its constants may be arbitrary bits.  The packed operands go over the
+// chunk's own S^T columns: r the first eight, t the last eight.
 template <bool MASKED>
-__device__ __forceinline__ void dkv_chunk(uint32_t tS, const uint32_t (&xs)[16], const uint32_t (&xp)[16], const float *nl, const float *nd,
-                                          float scale_log2, int lim, int hi) {
+__device__ __forceinline__ void dkv_chunk(uint32_t tS, const uint32_t (&xs)[16], const uint32_t (&xp)[16], float scale_log2, int lim, int hi) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2);
   uint32_t pr[8], pt[8];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 4 * i);   // four columns per 16-byte read
-    const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 4 * i);
     float a[4], p[4], t[4];
-    f32x2_split(fma2(f32x2_bits(xs[4 * i], xs[4 * i + 1]), scale2, l4.x), a[0], a[1]);
-    f32x2_split(fma2(f32x2_bits(xs[4 * i + 2], xs[4 * i + 3]), scale2, l4.y), a[2], a[3]);
+    f32x2_split(mul2(f32x2_bits(xs[4 * i], xs[4 * i + 1]), scale2), a[0], a[1]);
+    f32x2_split(mul2(f32x2_bits(xs[4 * i + 2], xs[4 * i + 3]), scale2), a[2], a[3]);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       p[e] = fast_exp2(a[e]);
       if (MASKED && (4 * i + e < lim || 4 * i + e > hi)) p[e] = 0.f;
     }
-    f32x2_split(mul2(f32x2(p[0], p[1]), add2(f32x2_bits(xp[4 * i], xp[4 * i + 1]), d4.x)), t[0], t[1]);
-    f32x2_split(mul2(f32x2(p[2], p[3]), add2(f32x2_bits(xp[4 * i + 2], xp[4 * i + 3]), d4.y)), t[2], t[3]);
+    f32x2_split(mul2(f32x2(p[0], p[1]), f32x2_bits(xp[4 * i], xp[4 * i + 1])), t[0], t[1]);
+    f32x2_split(mul2(f32x2(p[2], p[3]), f32x2_bits(xp[4 * i + 2], xp[4 * i + 3])), t[2], t[3]);
     if (MASKED) {
 #pragma unroll
       for (int e = 0; e < 4; ++e)
@@ -118,7 +120,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sK = smem;
   uint8_t *sV = sK + C::kTileBytes;
-  uint8_t *sStage = sV + C::kTileBytes;   // stage s: Q, dO, Z step tiles, then two blocks of {64 x -LSE log2 e, 64 x -D}
+  uint8_t *sStage = sV + C::kTileBytes;   // stage s: Q, dO, Z step tiles, then the step's row-constant tile (two 64-row blocks)
   uint8_t *sOut = sStage + S * C::kDkvStageBytes;   // staging: dK tile, then dV tile
 
   __shared__ uint64_t bar_res_full, bar_res_free, bar_q_full[S], bar_q_empty[S];
@@ -126,6 +128,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   __shared__ uint64_t bar_acc_done, bar_acc_free, bar_drain[3];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
+  // Constant operand of the extra K = 16 slice: three eight-row core matrices (zeros, rows of (1, 1, 1, 0, 0, 0, 0, 0), zeros).
+  // S^T reads (ones, zeros): it adds columns 0..2 of the row-constant tile; dP^T reads (zeros, ones): columns 8..10.
+  __shared__ __align__(128) uint4 s_ones[24];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
@@ -133,7 +138,11 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
   if (cta_skip != 0) return;
 
   const bool use_z = (flags & kFlagNoKCorrection) == 0;
-  const uint32_t stage_tx = (use_z ? 3 : 2) * C::kTileBytes + 1024;
+  const uint32_t stage_tx = (use_z ? 3 : 2) * C::kTileBytes + C::kExtBytes;
+  if (threadIdx.x < 24) {
+    s_ones[threadIdx.x] = (threadIdx.x >= 8 && threadIdx.x < 16) ? make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+  }
 
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
@@ -200,9 +209,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
           tma_load_3d(dst, &tmQ, &bar_q_full[st], 0, qrow, qh);
           tma_load_3d(dst + C::kTileBytes, &tmdO, &bar_q_full[st], 0, qrow, qh);
           if (use_z) tma_load_3d(dst + 2 * C::kTileBytes, &tmZ, &bar_q_full[st], 0, qrow, qh);
-          // two 64-row statistic blocks (the second may lie past the sequence's last block: its columns are masked)
-          bulk_load_1d(dst + 3 * C::kTileBytes, stats + (static_cast<size_t>(qh) * nblk + tl.blk0 + (qrel >> 6)) * 128, 1024,
-                       &bar_q_full[st]);
+          // two 64-row blocks of the row-constant tile (the second may lie past the sequence's last block: its columns are masked)
+          bulk_load_1d(dst + 3 * C::kTileBytes, reinterpret_cast<const uint8_t *>(stats) + (static_cast<size_t>(qh) * nblk + tl.blk0 + (qrel >> 6)) * kExtBlockBytes,
+                       C::kExtBytes, &bar_q_full[st]);
         }
       }
       if (cta_abort) {
@@ -228,6 +237,8 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);   // [128 keys] x [128 queries], contraction over d
     const SmemDesc dscK = make_smem_desc(smem_u32(sK), 16, 1024), dscV = make_smem_desc(smem_u32(sV), 16, 1024);
     const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);
+    const SmemDesc dscOnes = make_smem_desc_noswizzle(smem_u32(s_ones) + 128, 128, 0);                 // (ones, zeros), every row group the same
+    const SmemDesc dscExt0 = make_smem_desc_noswizzle(smem_u32(sStage + 3 * C::kTileBytes), 128, 256);
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const int T = G * steps_of(tile_of(lin));
@@ -242,6 +253,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) umma_ss(tS, dscK.at(k * 32), dscQ.at(k * 32), idesc_s, k > 0);
+          umma_ss(tS, dscOnes.at(0), dscExt0.at(st * C::kDkvStageBytes), idesc_s, 1u);   // - LSE / alpha in every key row
           umma_commit(&bar_s_full[sb]);
         }
         __syncwarp();
@@ -261,6 +273,8 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
     const SmemDesc dscV = make_smem_desc(smem_u32(sV), 16, 1024);
     const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);
+    const SmemDesc dscOnes = make_smem_desc_noswizzle(smem_u32(s_ones), 128, 0);                       // (zeros, ones)
+    const SmemDesc dscExt0 = make_smem_desc_noswizzle(smem_u32(sStage + 3 * C::kTileBytes), 128, 256);
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const int T = G * steps_of(tile_of(lin));
@@ -274,6 +288,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         if (elect_one_sync()) {
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) umma_ss(tmem_base + C::kColY, dscV.at(k * 32), dscdO.at(k * 32), idesc_s, k > 0);
+          umma_ss(tmem_base + C::kColY, dscOnes.at(0), dscExt0.at(st * C::kDkvStageBytes), idesc_s, 1u);   // - D in every key row
           umma_commit(&bar_dp_full);
           if (n == T - 1) umma_commit(&bar_res_free);   // second of two arrivals: no product reads this V tile any more
         }
@@ -345,10 +360,6 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         const int cb = 16 * wg;
         const uint32_t tS0 = tmem_base + lane_addr + (sb ? C::kColZ : C::kColX) + 16 * wg, tS1 = tS0 + 64;
         const uint32_t tdP0 = tmem_base + lane_addr + C::kColY + 16 * wg, tdP1 = tdP0 + 64;
-        // The scores of this step were issued after its stage (and with it the row statistics) had landed in shared
-        // memory, so their completion covers both.  The first 64 columns lie in statistic block 0, the last 64 in block 1:
-        // {64 x -LSE log2 e, 64 x -D} each.
-        const float *st0 = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kTileBytes) + 16 * wg, *st1 = st0 + 128;
         constexpr int kChunk1 = 64;
         const int nh = n % Th;                                              // step within the current query head
         const int Lq = tl.oseq_end - tl.oseq0, off = (tl.seq_end - tl.seq0) - Lq, krel0 = tl.row0 - tl.seq0;
@@ -368,15 +379,15 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(&bar_y_free);                   // dP^T is in registers: the tensor core may write the next step's
-        if (masked) dkv_chunk<true>(tS0, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[0]), st0, st0 + 64, scale_log2, lim, hi);
-        else        dkv_chunk<false>(tS0, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[0]), st0, st0 + 64, scale_log2, 0, 0);
+        if (masked) dkv_chunk<true>(tS0, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[0]), scale_log2, lim, hi);
+        else        dkv_chunk<false>(tS0, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[0]), scale_log2, 0, 0);
         tmem_ld16(tS1, xs);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar_rt_ready[sb][0]);
         tmem_wait_ld();
-        if (masked) dkv_chunk<true>(tS1, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[16]), st1, st1 + 64, scale_log2, lim - kChunk1, hi - kChunk1);
-        else        dkv_chunk<false>(tS1, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[16]), st1, st1 + 64, scale_log2, 0, 0);
+        if (masked) dkv_chunk<true>(tS1, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[16]), scale_log2, lim - kChunk1, hi - kChunk1);
+        else        dkv_chunk<false>(tS1, xs, *reinterpret_cast<const uint32_t (*)[16]>(&xp[16]), scale_log2, 0, 0);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar_rt_ready[sb][1]);

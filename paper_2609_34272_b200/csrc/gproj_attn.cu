@@ -177,8 +177,9 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
 
 // Row statistics {-LSE log2 e, -D}: blocks of 64 rows, 512 B each (per head ceil(N / 64) of them, the last one
 // zero-padded), plus one spare block: the 128-wide steps fetch two blocks at a time and may reach one past the end.
-size_t stats_blocks_bytes(size_t blocks) { return align256((blocks + 1) * 512); }
-size_t stats_bytes(int heads, int N) { return stats_blocks_bytes(static_cast<size_t>(heads) * ((N + 63) / 64)); }
+// At d = 64 a block is the K-major row-constant tile of the dK/dV side's extra product slice instead (64 rows x 16 BF16).
+size_t stats_blocks_bytes(size_t blocks, int d) { return align256((blocks + 1) * (d == 64 ? static_cast<size_t>(gproj::kExtBlockBytes) : 512)); }
+size_t stats_bytes(int heads, int N, int d) { return stats_blocks_bytes(static_cast<size_t>(heads) * ((N + 63) / 64), d); }
 
 }  // namespace
 
@@ -384,7 +385,7 @@ extern "C" {
 
 size_t gproj_attn_bwd_workspace_bytes(int B, int H, int N, int d) {
   if (check_shape(B, H, N, d) != GPROJ_OK) return 0;
-  return stats_bytes(B * H, N) + align256(static_cast<size_t>(B) * H * N * static_cast<size_t>(d) * 2);
+  return stats_bytes(B * H, N, d) + align256(static_cast<size_t>(B) * H * N * static_cast<size_t>(d) * 2);
 }
 
 int gproj_attn_bwd(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,
@@ -424,7 +425,7 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
   const bool run_dq = !(flags & GPROJ_FLAG_ONLY_DKV_PASS);
   bool run_dkv = !(flags & GPROJ_FLAG_ONLY_DQ_PASS);
   if (!run_dq && !run_dkv) return GPROJ_ERR_FLAGS;
-  const size_t stats_sz = stats_blocks_bytes(static_cast<size_t>(B) * H * nblk);
+  const size_t stats_sz = stats_blocks_bytes(static_cast<size_t>(B) * H * nblk, d);
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
       workspace_bytes < stats_sz + align256(static_cast<size_t>(B) * H * N * static_cast<size_t>(d) * 2))
     return GPROJ_ERR_WORKSPACE;
@@ -637,7 +638,7 @@ int gproj_attn_fwd_varlen(const void *Q, const void *K, const void *V, void *O, 
 size_t gproj_attn_bwd_varlen_workspace_bytes(const int *cu_seqlens, int num_seqs, int H, int d) {
   PackedShape ps;
   if (!packed_shape(cu_seqlens, cu_seqlens, num_seqs, &ps) || check_shape(1, H, ps.total_q, d) != GPROJ_OK) return 0;
-  return stats_blocks_bytes(static_cast<size_t>(H) * ps.nblk) + align256(static_cast<size_t>(H) * ps.total_q * static_cast<size_t>(d) * 2);
+  return stats_blocks_bytes(static_cast<size_t>(H) * ps.nblk, d) + align256(static_cast<size_t>(H) * ps.total_q * static_cast<size_t>(d) * 2);
 }
 
 int gproj_attn_bwd_varlen(const void *Q, const void *K, const void *V, const void *O, const float *LSE, const void *dO,

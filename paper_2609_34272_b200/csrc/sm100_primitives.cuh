@@ -242,6 +242,13 @@ __device__ __forceinline__ SmemDesc make_smem_desc(uint32_t saddr, uint32_t lbo_
   const uint64_t d = smem_desc_sw128(saddr, lbo_bytes, sbo_bytes);
   return SmemDesc{static_cast<uint32_t>(d), static_cast<uint32_t>(d >> 32)};
 }
+// K-major operand without swizzle: 8-row x 16-byte core matrices of 128 contiguous bytes; LBO = byte stride between the
+// two core matrices of a K = 16 slice, SBO = byte stride between groups of eight rows (0: every group reads the same eight
+// rows, a matrix whose rows are all equal).
+__device__ __forceinline__ SmemDesc make_smem_desc_noswizzle(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  const uint64_t d = smem_desc_sw128(saddr, lbo_bytes, sbo_bytes) & ~(static_cast<uint64_t>(7) << 61);
+  return SmemDesc{static_cast<uint32_t>(d), static_cast<uint32_t>(d >> 32)};
+}
 
 // Instruction descriptor for kind::f16 with BF16 A/B and FP32 accumulation.
 //   bits [4,6) D format (1 = F32)  [7,10) A format (1 = BF16)  [10,13) B format (1 = BF16)

@@ -39,13 +39,16 @@ def test_status_strings(lib):
 
 
 def test_workspace_bytes(lib):
-    # one BF16 query-shaped array + two FP32 row arrays (the paper's "Cost" paragraph allows more)
-    B, H, N, d = 2, 3, 256, 64
+    # one BF16 query-shaped array + the row constants (LSE, D) in 64-row blocks plus one spare block (the paper's "Cost"
+    # paragraph allows more).  d = 128: two FP32 values per row, 512 B per block.  d = 64: the constants travel as a
+    # 16-column BF16 operand tile of the dK/dV side's score products, 32 B per row, 2048 B per block.
+    B, H, N = 2, 3, 256
     rows = B * H * N
-    # row statistics: 8 bytes per row in 64-row blocks plus one spare block (256-byte aligned), then the BF16 array
-    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, d) == rows * 8 + 512 + rows * d * 2
-    # ragged length: statistics are padded to whole 64-row blocks per head (2 blocks x 512 B), the query-shaped array is not
-    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 3 * 512 + 100 * 64 * 2
+    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, 128) == rows * 8 + 512 + rows * 128 * 2
+    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, 64) == rows * 32 + 2048 + rows * 64 * 2
+    # ragged length: the blocks are padded to whole 64-row blocks per head (2 blocks + the spare), the query-shaped array is not
+    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 128) == 3 * 512 + 100 * 128 * 2
+    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 3 * 2048 + 100 * 64 * 2
     assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 0, 64) == 0
     assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 128, 96) == 0
 

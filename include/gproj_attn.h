@@ -75,9 +75,9 @@ int gproj_attn_fwd(const void *Q, const void *K, const void *V, void *O, float *
  * Bytes of device scratch gproj_attn_bwd needs for this shape (0 if the shape is unsupported).
  * The paper's resource statement (Appendix "Implemented Arithmetic", "Cost") allows a query-shaped
  * workspace and two row-statistic arrays; this implementation uses one BF16 query-shaped array
- * (the operand BF16(lambda_i q_i) of Algorithm 1 line 17) and the two row constants (LSE, D) in blocks of 64 rows:
- * two FP32 values per row at d = 128; at d = 64 thirty-two bytes per row, because there the constants reach the
- * dK/dV side as a 16-column BF16 operand of its score products (each constant as three BF16 pieces).
+ * (the operand BF16(lambda_i q_i) of Algorithm 1 line 17) and the two row constants (LSE, D) in blocks of 64 rows,
+ * thirty-two bytes per row: they reach the dK/dV side as a 16-column BF16 operand of its score products (each
+ * constant as three BF16 pieces that add up to the FP32 value).
  */
 size_t gproj_attn_bwd_workspace_bytes(int B, int H, int N, int d);
 

@@ -46,6 +46,9 @@ namespace gproj {
 constexpr unsigned kFlagNoQCorrection = 1u;
 constexpr unsigned kFlagNoKCorrection = 2u;
 
+// Bytes of one 64-row block of the row-constant tile (64 rows x 16 BF16 columns).
+constexpr int kExtBlockBytes = 2048;
+
 template <int D>
 struct BwdCfg {
   static constexpr int kSlabs = D / 64;
@@ -81,7 +84,7 @@ struct BwdCfg {
                                       (kPrefetchO ? kBigTileBytes : 0) + 1024;
   // dK/dV-side kernel: K, V resident; ring of (Q, dO, Z, stats) step tiles
   static constexpr int kDkvStages = (D == 64) ? 5 : 3;
-  static constexpr int kDkvStageBytes = 3 * kStepTileBytes + 1024;   // + 2 x 64 floats of row statistics (512 B used)
+  static constexpr int kDkvStageBytes = 3 * kStepTileBytes + kExtBlockBytes;   // + the step's 64-row block of the row-constant tile
   static constexpr int kDkvSmemBytes = 2 * kBigTileBytes + kDkvStages * kDkvStageBytes + (kSepStaging ? 2 * kBigTileBytes : 0) + 1024;
   static_assert(kDqStages >= kNB + 1 && kDkvStages >= kNB + 1, "a stage stays busy until its second-stage MMAs finish");
 };
@@ -164,9 +167,6 @@ __device__ __forceinline__ void store_rows_clipped(const uint8_t *stage, int sla
   }
 }
 
-// Bytes of one 64-row block of the d = 64 row-constant tile (64 rows x 16 BF16 columns).
-constexpr int kExtBlockBytes = 2048;
-
 enum BwdWaitCode {
   kDqWaitQ = 0x21, kDqWaitKV = 0x22, kDqWaitKVEmpty = 0x23, kDqWaitSdP = 0x24, kDqWaitTR = 0x25, kDqWaitAcc = 0x26, kDqWaitBuf = 0x27, kDqWaitResFree = 0x28, kDqWaitAccFree = 0x29,
   kDkvWaitKV = 0x31, kDkvWaitQ = 0x32, kDkvWaitQEmpty = 0x33, kDkvWaitSdP = 0x34, kDkvWaitTR = 0x35, kDkvWaitAcc = 0x36, kDkvWaitBuf = 0x37, kDkvWaitResFree = 0x38, kDkvWaitAccFree = 0x39
@@ -236,10 +236,12 @@ __device__ __forceinline__ void dq_slice(uint32_t tS, uint32_t tdP, float scale_
 
 // Phase 1 of the dK/dV side (thread <-> key row, columns = queries).  `lim` = (key row) - (query index of the slice's
 // column 0): with MASKED, column c is a query before this key when c < lim; `hi` = (last query of the sequence) - (query
-// index of column 0): a column c > hi belongs to the next packed sequence (or is zero fill).  nl: the slice's per-column
-// -LSE log2 e (shared memory, same address for every lane: broadcast reads).
+// index of column 0): a column c > hi belongs to the next packed sequence (or is zero fill).  The scores arrive as
+// x - LSE / alpha: the score product carries one extra K = 16 slice (a constant matrix of ones times the step's
+// row-constant tile), so no per-column constant has to be read here (every lane would need every column's value:
+// broadcast reads from shared memory cost the 64-query kernel at d = 64 14 % when it still had them).
 template <bool MASKED>
-__device__ __forceinline__ void dkv_phase1(uint32_t tS, const float *nl, float scale_log2, int lim, int hi, float (&p)[32]) {
+__device__ __forceinline__ void dkv_phase1(uint32_t tS, float scale_log2, int lim, int hi, float (&p)[32]) {
   const uint64_t scale2 = f32x2(scale_log2, scale_log2);
   uint32_t xs[2][16];
   tmem_ld16(tS, xs[0]);
@@ -250,11 +252,10 @@ __device__ __forceinline__ void dkv_phase1(uint32_t tS, const float *nl, float s
     uint32_t pr[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(nl + 16 * c + 4 * i);   // four columns per 16-byte read
       const int col = 16 * c + 4 * i;
       float a[4];
-      f32x2_split(fma2(f32x2_bits(xs[c][4 * i], xs[c][4 * i + 1]), scale2, l4.x), a[0], a[1]);
-      f32x2_split(fma2(f32x2_bits(xs[c][4 * i + 2], xs[c][4 * i + 3]), scale2, l4.y), a[2], a[3]);
+      f32x2_split(mul2(f32x2_bits(xs[c][4 * i], xs[c][4 * i + 1]), scale2), a[0], a[1]);
+      f32x2_split(mul2(f32x2_bits(xs[c][4 * i + 2], xs[c][4 * i + 3]), scale2), a[2], a[3]);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         float pe = fast_exp2(a[e]);
@@ -268,8 +269,8 @@ __device__ __forceinline__ void dkv_phase1(uint32_t tS, const float *nl, float s
   }
 }
 
-// Phase 2 of the dK/dV side.  nd: the slice's per-column -D.
-__device__ __forceinline__ void dkv_phase2(uint32_t tS, uint32_t tdP, const float *nd, const float (&p)[32]) {
+// Phase 2 of the dK/dV side.  The products arrive as dP - D (same extra slice as for the scores).
+__device__ __forceinline__ void dkv_phase2(uint32_t tS, uint32_t tdP, const float (&p)[32]) {
   uint32_t xp[2][16];
   tmem_ld16(tdP, xp[0]);
 #pragma unroll
@@ -279,11 +280,10 @@ __device__ __forceinline__ void dkv_phase2(uint32_t tS, uint32_t tdP, const floa
     uint32_t pt[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(nd + 16 * c + 4 * i);
       const int col = 16 * c + 4 * i;
       float t0, t1, t2, t3;
-      f32x2_split(mul2(f32x2(p[col], p[col + 1]), add2(f32x2_bits(xp[c][4 * i], xp[c][4 * i + 1]), d4.x)), t0, t1);
-      f32x2_split(mul2(f32x2(p[col + 2], p[col + 3]), add2(f32x2_bits(xp[c][4 * i + 2], xp[c][4 * i + 3]), d4.y)), t2, t3);
+      f32x2_split(mul2(f32x2(p[col], p[col + 1]), f32x2_bits(xp[c][4 * i], xp[c][4 * i + 1])), t0, t1);
+      f32x2_split(mul2(f32x2(p[col + 2], p[col + 3]), f32x2_bits(xp[c][4 * i + 2], xp[c][4 * i + 3])), t2, t3);
       pt[2 * i] = pack_bf16x2(t0, t1);
       pt[2 * i + 1] = pack_bf16x2(t2, t3);
     }
@@ -557,30 +557,24 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       const float Dv = s_D[row];
       const float lse_row = (qrow < tl.seq_end) ? (C::kPrefetchO ? lse_pre : LSE[head_row0 + qrow]) : 0.f;
       const float neg_lse2 = -lse_row * 1.4426950408889634f;
-      // Per 64-row block of a sequence (the last one padded with zeros): 64 x {-LSE log2 e}, then 64 x {-D}.
+      // Row constants for the dK/dV side, per 64-row block of a sequence (the last one padded with zeros).
       const int rel = qrow - tl.seq0;                  // row inside the sequence
       if (wg == 0 && rel < ((tl.seq_end - tl.seq0 + C::kStepRows - 1) / C::kStepRows) * C::kStepRows) {
-        if (D == 64) {
-          // d = 64: the dK/dV side takes both row constants through its score products instead of reading them per
-          // column.  Per 64-row block a K-major operand tile of 16 BF16 columns without swizzle (eight-row groups of 256
-          // bytes: the rows' first eight columns, then their last eight): columns 0..2 hold -LSE / alpha and columns
-          // 8..10 hold -D, each as three BF16 pieces whose sum is the FP32 value, the other columns zero.  A row with an
-          // empty support (LSE = +inf) gets a large finite value: its probabilities are zero either way, and an
-          // infinity would turn the zero entries of the constant operand into NaN.
-          const float c = fmaxf(__fdiv_rn(neg_lse2, scale_log2), -1.0e30f), nd = -Dv;
-          const uint32_t c0 = pack_bf16x2(c, 0.f), n0 = pack_bf16x2(nd, 0.f);
-          const float c_r1 = c - bf16_lo_to_f32(c0), n_r1 = nd - bf16_lo_to_f32(n0);
-          const uint32_t c1 = pack_bf16x2(c_r1, 0.f), n1 = pack_bf16x2(n_r1, 0.f);
-          const uint32_t c2 = pack_bf16x2(c_r1 - bf16_lo_to_f32(c1), 0.f), n2 = pack_bf16x2(n_r1 - bf16_lo_to_f32(n1), 0.f);
-          uint8_t *blk = reinterpret_cast<uint8_t *>(stats) + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * kExtBlockBytes +
-                         ((rel & 63) >> 3) * 256 + (rel & 7) * 16;
-          *reinterpret_cast<uint4 *>(blk) = make_uint4(c0 | (c1 << 16), c2, 0u, 0u);
-          *reinterpret_cast<uint4 *>(blk + 128) = make_uint4(n0 | (n1 << 16), n2, 0u, 0u);
-        } else {
-          float *blk = stats + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * 128 + (rel & 63);
-          blk[0] = neg_lse2;
-          blk[64] = -Dv;
-        }
+        // The dK/dV side takes both row constants through its score products instead of reading them per column.  Per
+        // 64-row block a K-major operand tile of 16 BF16 columns without swizzle (eight-row groups of 256 bytes: the
+        // rows' first eight columns, then their last eight): columns 0..2 hold -LSE / alpha and columns 8..10 hold -D,
+        // each as three BF16 pieces whose sum is the FP32 value, the other columns zero.  A row with an empty support
+        // (LSE = +inf) gets a large finite value: its probabilities are zero either way, and an infinity would turn the
+        // zero entries of the constant operand into NaN.
+        const float c = fmaxf(__fdiv_rn(neg_lse2, scale_log2), -1.0e30f), nd = -Dv;
+        const uint32_t c0 = pack_bf16x2(c, 0.f), n0 = pack_bf16x2(nd, 0.f);
+        const float c_r1 = c - bf16_lo_to_f32(c0), n_r1 = nd - bf16_lo_to_f32(n0);
+        const uint32_t c1 = pack_bf16x2(c_r1, 0.f), n1 = pack_bf16x2(n_r1, 0.f);
+        const uint32_t c2 = pack_bf16x2(c_r1 - bf16_lo_to_f32(c1), 0.f), n2 = pack_bf16x2(n_r1 - bf16_lo_to_f32(n1), 0.f);
+        uint8_t *blk = reinterpret_cast<uint8_t *>(stats) + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * kExtBlockBytes +
+                       ((rel & 63) >> 3) * 256 + (rel & 7) * 16;
+        *reinterpret_cast<uint4 *>(blk) = make_uint4(c0 | (c1 << 16), c2, 0u, 0u);
+        *reinterpret_cast<uint4 *>(blk + 128) = make_uint4(n0 | (n1 << 16), n2, 0u, 0u);
       }
 
       uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);
@@ -746,7 +740,15 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
   if (cta_skip != 0) return;
 
   const bool use_z = (flags & kFlagNoKCorrection) == 0;
-  const uint32_t stage_tx = (use_z ? 3 : 2) * C::kStepTileBytes + 512;
+  const uint32_t stage_tx = (use_z ? 3 : 2) * C::kStepTileBytes + kExtBlockBytes;
+  // Constant operand of the extra K = 16 slice of the score products: three eight-row core matrices (zeros, rows of
+  // (1, 1, 1, 0, 0, 0, 0, 0), zeros).  S^T reads (ones, zeros): it adds columns 0..2 of the row-constant tile, the three
+  // BF16 pieces of -LSE / alpha; dP^T reads (zeros, ones): columns 8..10, the pieces of -D.
+  __shared__ __align__(128) uint4 s_ones[24];
+  if (threadIdx.x < 24) {
+    s_ones[threadIdx.x] = (threadIdx.x >= 8 && threadIdx.x < 16) ? make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+  }
 
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
@@ -814,7 +816,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
             tma_load_3d(dst + C::kStepTileBytes + s * C::kStepSlabBytes, &tmdO, &bar_q_full[st], s * 64, qrow, qh);
             if (use_z) tma_load_3d(dst + 2 * C::kStepTileBytes + s * C::kStepSlabBytes, &tmZ, &bar_q_full[st], s * 64, qrow, qh);
           }
-          bulk_load_1d(dst + 3 * C::kStepTileBytes, stats + (static_cast<size_t>(qh) * nblk + tl.blk0 + (qrel >> 6)) * 128, 512, &bar_q_full[st]);
+          bulk_load_1d(dst + 3 * C::kStepTileBytes, reinterpret_cast<const uint8_t *>(stats) + (static_cast<size_t>(qh) * nblk + tl.blk0 + (qrel >> 6)) * kExtBlockBytes,
+                       kExtBlockBytes, &bar_q_full[st]);
         }
       }
       if (cta_abort) {
@@ -843,6 +846,9 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, 64, 0, 0);    // [128 keys] x [64 queries], contraction over d
     const SmemDesc dscK = make_smem_desc(smem_u32(sK), 16, 1024), dscV = make_smem_desc(smem_u32(sV), 16, 1024);
     const SmemDesc dscQ0 = make_smem_desc(smem_u32(sStage), 16, 1024);                       // K-major view of stage 0
+    const SmemDesc dscOnesS = make_smem_desc_noswizzle(smem_u32(s_ones) + 128, 128, 0);      // (ones, zeros), every row group the same
+    const SmemDesc dscOnesP = make_smem_desc_noswizzle(smem_u32(s_ones), 128, 0);            // (zeros, ones)
+    const SmemDesc dscExt0 = make_smem_desc_noswizzle(smem_u32(sStage + 3 * C::kStepTileBytes), 128, 256);
     int g = 0, ti = 0;
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const int T = G * steps_of(tile_of(lin));
@@ -860,12 +866,14 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
             umma_ss(tS, dscK.at(oa), dscQ.at(ob), idesc_s, k > 0);
           }
+          umma_ss(tS, dscOnesS.at(0), dscExt0.at(st * C::kDkvStageBytes), idesc_s, 1u);     // - LSE / alpha in every key row
           umma_commit(&bar_s_full[b]);                      // phase 1 of the ALUs needs only S^T
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint32_t oa = (k / 4) * C::kBigSlabBytes + (k % 4) * 32, ob = (k / 4) * C::kStepSlabBytes + (k % 4) * 32;
             umma_ss(tdP, dscV.at(oa), dscdO.at(ob), idesc_s, k > 0);
           }
+          umma_ss(tdP, dscOnesP.at(0), dscExt0.at(st * C::kDkvStageBytes), idesc_s, 1u);    // - D in every key row
           umma_commit(&bar_dp_full[b]);
           if (n == T - 1) umma_commit(&bar_res_free);   // no MMA reads this K / V tile any more
         }
@@ -940,27 +948,24 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
 #endif
       for (int n = (grp - g0 % C::kGroups + C::kGroups) % C::kGroups; n < T; n += C::kGroups) {
         const int g = g0 + n, st = g % S, b = g % NB;
-        // The scores of this step were issued after its stage (and with it the row statistics) had landed in shared
-        // memory, so their completion covers both.
         mbar_wait(&bar_s_full[b], (g / NB) & 1, ab, kDkvWaitSdP);
         tc_fence_after();
         const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;
-        const float *nl = reinterpret_cast<const float *>(sStage + st * C::kDkvStageBytes + 3 * C::kStepTileBytes) + C::kSliceCols * slice;
         const int nh = n % Th;                                      // step within the current query head
         const int Lq = tl.oseq_end - tl.oseq0, off = (tl.seq_end - tl.seq0) - Lq, krel0 = tl.row0 - tl.seq0;
         const int qs = q_start + nh * C::kStepRows;                           // first query (inside its sequence) of the step
         const int q0 = qs + C::kSliceCols * slice;                            // ... of the slice's column 0
         float pkeep[32];
         if ((CAUSAL && qs < krel0 + 128 - off) || qs + C::kStepRows > Lq)
-          dkv_phase1<true>(tS16, nl, scale_log2, CAUSAL ? krel0 + row - off - q0 : 0, Lq - 1 - q0, pkeep);
+          dkv_phase1<true>(tS16, scale_log2, CAUSAL ? krel0 + row - off - q0 : 0, Lq - 1 - q0, pkeep);
         else
-          dkv_phase1<false>(tS16, nl, scale_log2, 0, 0, pkeep);
+          dkv_phase1<false>(tS16, scale_log2, 0, 0, pkeep);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar_r_ready[b]);
         mbar_wait(&bar_dp_full[b], (g / NB) & 1, ab, kDkvWaitSdP);
         tc_fence_after();
-        dkv_phase2(tS16, tdP16, nl + 64, pkeep);
+        dkv_phase2(tS16, tdP16, pkeep);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar_t_ready[b]);

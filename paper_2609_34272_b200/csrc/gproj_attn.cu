@@ -175,10 +175,10 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
                void *workspace, size_t workspace_bytes, unsigned flags, const int4 *plan_q, const int4 *plan_kv,
                int n_plan_q_tiles, int n_plan_kv_tiles, int nblk, void *stream);
 
-// Row statistics {-LSE log2 e, -D}: blocks of 64 rows, 512 B each (per head ceil(N / 64) of them, the last one
-// zero-padded), plus one spare block: the 128-wide steps fetch two blocks at a time and may reach one past the end.
-// At d = 64 a block is the K-major row-constant tile of the dK/dV side's extra product slice instead (64 rows x 16 BF16).
-size_t stats_blocks_bytes(size_t blocks, int d) { return align256((blocks + 1) * (d == 64 ? static_cast<size_t>(gproj::kExtBlockBytes) : 512)); }
+// Row constants (-LSE / alpha, -D) for the dK/dV side: per 64 rows one K-major operand tile of 16 BF16 columns (2048 B;
+// per head ceil(N / 64) of them, the last one zero-padded), plus one spare block: the 128-wide steps fetch two blocks at
+// a time and may reach one past the end.
+size_t stats_blocks_bytes(size_t blocks, int) { return align256((blocks + 1) * static_cast<size_t>(gproj::kExtBlockBytes)); }
 size_t stats_bytes(int heads, int N, int d) { return stats_blocks_bytes(static_cast<size_t>(heads) * ((N + 63) / 64), d); }
 
 }  // namespace
@@ -433,7 +433,7 @@ int launch_bwd(const void *Q, const void *K, const void *V, const void *O, const
   if (int rc = device_state(&st)) return rc;
 
   const int BH = B * H, BHkv = B * Hkv;
-  float *stats = static_cast<float *>(workspace);   // per 64-row block: 64 x {-LSE log2 e}, 64 x {-D}
+  float *stats = static_cast<float *>(workspace);   // per 64-row block: the row-constant tile (see stats_blocks_bytes)
   __nv_bfloat16 *Zneg = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + stats_sz);
 
   CUtensorMap mQ128, mdO128, mK64, mV64, mK128, mV128, mQ64, mdO64, mZ64, mdQst, mZst, mdKst, mdVst;

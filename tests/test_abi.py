@@ -40,15 +40,14 @@ def test_status_strings(lib):
 
 def test_workspace_bytes(lib):
     # one BF16 query-shaped array + the row constants (LSE, D) in 64-row blocks plus one spare block (the paper's "Cost"
-    # paragraph allows more).  d = 128: two FP32 values per row, 512 B per block.  d = 64: the constants travel as a
-    # 16-column BF16 operand tile of the dK/dV side's score products, 32 B per row, 2048 B per block.
+    # paragraph allows more): the constants travel as a 16-column BF16 operand tile of the dK/dV side's score products,
+    # 32 B per row, 2048 B per block.
     B, H, N = 2, 3, 256
     rows = B * H * N
-    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, 128) == rows * 8 + 512 + rows * 128 * 2
-    assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, 64) == rows * 32 + 2048 + rows * 64 * 2
-    # ragged length: the blocks are padded to whole 64-row blocks per head (2 blocks + the spare), the query-shaped array is not
-    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 128) == 3 * 512 + 100 * 128 * 2
-    assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, 64) == 3 * 2048 + 100 * 64 * 2
+    for d in (64, 128):
+        assert binding.gproj_attn_bwd_workspace_bytes(B, H, N, d) == rows * 32 + 2048 + rows * d * 2
+        # ragged length: the blocks are padded to whole 64-row blocks per head (2 blocks + the spare), the query-shaped array is not
+        assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 100, d) == 3 * 2048 + 100 * d * 2
     assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 0, 64) == 0
     assert binding.gproj_attn_bwd_workspace_bytes(1, 1, 128, 96) == 0
 

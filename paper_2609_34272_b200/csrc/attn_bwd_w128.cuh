@@ -41,7 +41,7 @@ struct BwdW128 {
   static constexpr int kTileBytes = 128 * 128;                     // 128 rows x 64 BF16: one 128-byte-row slab
   static constexpr int kStepRows = 128;
   static constexpr int kStages = 3;
-  static constexpr int kWG = 4, kCompute = 128 * kWG, kThreads = 128 + kCompute;  // warp 0: stage producer (lane 0) and tile loader (lane 1); warps 1, 2, 3: MMA issuers (S^T; second stage; dP^T); 16 compute warps
+  static constexpr int kWG = 4, kCompute = 128 * kWG, kLoaderWarp = 4 + 4 * kWG, kThreads = 128 + kCompute + 32;  // warp 0: stage producer; warps 1, 2, 3: MMA issuers (S^T; second stage; dP^T); 16 compute warps; last warp: K / V tile loader
   static constexpr uint32_t kColX = 0, kColY = 128, kColZ = 256, kColAcc0 = 384, kColAcc1 = 448;
   static constexpr int kTmemCols = 512;
   // K, V resident, ring of (Q, dO, Z, two 64-row blocks of the row-constant tile) step tiles, staging (dK, dV)
@@ -218,19 +218,6 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         for (int q = (g > S ? g - S : 0); q < g; ++q)
           for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_q_full[q % S], (q / S) & 1); ++spin) {}
       }
-    } else if (lane == 1) {
-      // -------------------------------------------------------------- TMA loader of the stationary (K, V) tiles (second lane of
-      // the producer's warp: the two single-thread roles share a warp, which leaves 608 threads and 104 registers each)
-      int ti = 0;
-      for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int bh = hix(lin), krow0 = tile_of(lin).row0;
-        if (ti >= 1) mbar_wait(&bar_res_free, (ti - 1) & 1, ab, kWkResFree);
-        mbar_expect_tx(&bar_res_full, 2 * C::kTileBytes);
-        tma_load_3d(sK, &tmK, &bar_res_full, 0, krow0, bh);
-        tma_load_3d(sV, &tmV, &bar_res_full, 0, krow0, bh);
-      }
-      if (cta_abort && ti > 0)
-        for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_res_full, (ti - 1) & 1); ++spin) {}
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- tensor-core issuer 1: S^T = K Q^T, dP^T = V dO^T
@@ -344,6 +331,21 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       }
     }
     drain_mmas_if_aborted(&bar_drain[1], ab);
+  } else if (warp == C::kLoaderWarp) {
+    // ---------------------------------------------------------------- TMA loader of the stationary (K, V) tiles.  A warp of its
+    // own: as a second lane of the stage producer's warp its loads at a tile boundary waited for the producer's polling loop.
+    if (lane == 0) {
+      int ti = 0;
+      for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+        const int bh = hix(lin), krow0 = tile_of(lin).row0;
+        if (ti >= 1) mbar_wait(&bar_res_free, (ti - 1) & 1, ab, kWkResFree);
+        mbar_expect_tx(&bar_res_full, 2 * C::kTileBytes);
+        tma_load_3d(sK, &tmK, &bar_res_full, 0, krow0, bh);
+        tma_load_3d(sV, &tmV, &bar_res_full, 0, krow0, bh);
+      }
+      if (cta_abort && ti > 0)
+        for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_res_full, (ti - 1) & 1); ++spin) {}
+    }
   } else {
     // ---------------------------------------------------------------- compute: thread <-> (key row, 32-query slice of every step)
     const int wg = (warp - 4) >> 2;
@@ -353,6 +355,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const TileInfo tl = tile_of(lin);
       const int bh = hix(lin), Th = steps_of(tl), T = G * Th, q_start = q_start_of(tl);
+#ifdef GPROJ_TRACE
+      const unsigned long long ev_n0 = global_ns(); const long long ev_c0 = clock64(); unsigned long long ev_n1 = 0;
+#endif
       for (int n = 0; n < T; ++n) {
         const int g = g0 + n, st = g % S, sb = g & 1;
         // This thread's two 16-column chunks: columns 16 w .. 16 w + 15 of the step's first 64 queries, then of its last 64
@@ -372,6 +377,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         mbar_wait(&bar_s_full[sb], (g >> 1) & 1, ab, kWkS);
         mbar_wait(&bar_dp_full, g & 1, ab, kWkDP);
         tc_fence_after();
+#ifdef GPROJ_TRACE
+        if (n == 0) ev_n1 = global_ns();
+#endif
         uint32_t xp[32], xs[16];
         tmem_ld16(tdP0, *reinterpret_cast<uint32_t (*)[16]>(&xp[0]));
         tmem_ld16(tdP1, *reinterpret_cast<uint32_t (*)[16]>(&xp[16]));
@@ -393,6 +401,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
         mbar_arrive(&bar_rt_ready[sb][1]);
       }
 
+#ifdef GPROJ_TRACE
+      const unsigned long long ev_n2 = global_ns();
+#endif
       mbar_wait(&bar_acc_done, ti & 1, ab, kWkAcc);
       tc_fence_after();
       uint8_t *stage_dk = sOut, *stage_dv = sOut + C::kTileBytes;
@@ -431,6 +442,9 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
                                          (wg == 0 ? dKg : dVg) + (static_cast<size_t>(bh) * N + tl.row0) * D, row, tl.seq_end - tl.row0);
         named_bar_sync(1, C::kCompute);
       }
+#ifdef GPROJ_TRACE
+      if ((threadIdx.x & 127) == 0 && wg == 0) tile_event(8, lin, T, ev_n0, ev_n1, ev_n2, global_ns(), ev_c0, clock64());
+#endif
       g0 += T;
     }
     if (threadIdx.x == 128) bulk_wait_group_read0();

@@ -947,7 +947,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 rows
       const unsigned long long tile_t0 = global_ns();
 #endif
       for (int n = (grp - g0 % C::kGroups + C::kGroups) % C::kGroups; n < T; n += C::kGroups) {
-        const int g = g0 + n, st = g % S, b = g % NB;
+        const int g = g0 + n, b = g % NB;
         mbar_wait(&bar_s_full[b], (g / NB) & 1, ab, kDkvWaitSdP);
         tc_fence_after();
         const uint32_t tS16 = slice_addr + 128 * b, tdP16 = tS16 + 64;

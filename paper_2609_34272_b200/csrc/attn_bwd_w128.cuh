@@ -359,7 +359,7 @@ bwd_dkv_w128_kernel(const __grid_constant__ CUtensorMap tmK,    // box 64 x 128 
       const unsigned long long ev_n0 = global_ns(); const long long ev_c0 = clock64(); unsigned long long ev_n1 = 0;
 #endif
       for (int n = 0; n < T; ++n) {
-        const int g = g0 + n, st = g % S, sb = g & 1;
+        const int g = g0 + n, sb = g & 1;
         // This thread's two 16-column chunks: columns 16 w .. 16 w + 15 of the step's first 64 queries, then of its last 64
         // (operand slices k = w and k = 4 + w).
         const int cb = 16 * wg;

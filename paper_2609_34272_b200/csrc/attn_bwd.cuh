@@ -77,11 +77,13 @@ struct BwdCfg {
   static constexpr int kDqStages = (D == 64) ? 6 : 4;
   static constexpr int kDqStageBytes = 2 * kStepTileBytes;
   static constexpr int kDqResBufs = (D == 64) ? 2 : 1;             // stationary (Q, dO) buffers
-  // d = 64: the saved-output rows of the NEXT tile (for D = rowsum(dO o O)) are copied into shared memory asynchronously
-  // during the current tile's epilogue; at d = 128 there is no room and the rows are loaded at the tile's start.
-  static constexpr bool kPrefetchO = (D == 64);
+  // d = 64 (two stationary buffers): D = rowsum(dO o O), LSE and the row-constant tile of a tile are prepared by the
+  // stationary-tile loader's warp as soon as the tile's dO has landed, i.e. while the tile before it still runs; the
+  // compute warps only pick the two values up.  At d = 128 there is one stationary buffer and the compute warps do it at
+  // the tile's start.
+  static constexpr bool kLoaderStats = (D == 64);
   static constexpr int kDqSmemBytes = kDqResBufs * 2 * kBigTileBytes + kDqStages * kDqStageBytes + (kSepStaging ? 2 * kBigTileBytes : 0) +
-                                      (kPrefetchO ? kBigTileBytes : 0) + 1024;
+                                      1024;
   // dK/dV-side kernel: K, V resident; ring of (Q, dO, Z, stats) step tiles
   static constexpr int kDkvStages = (D == 64) ? 5 : 3;
   static constexpr int kDkvStageBytes = 3 * kStepTileBytes + kExtBlockBytes;   // + the step's 64-row block of the row-constant tile
@@ -291,6 +293,23 @@ __device__ __forceinline__ void dkv_phase2(uint32_t tS, uint32_t tdP, const floa
   }
 }
 
+// Row constants of one query row for the dK/dV side, which takes them through its score products instead of reading
+// them per column.  Per 64-row block a K-major operand tile of 16 BF16 columns without swizzle (eight-row groups of 256
+// bytes: the rows' first eight columns, then their last eight): columns 0..2 hold -LSE / alpha and columns 8..10 hold -D,
+// each as three BF16 pieces whose sum is the FP32 value, the other columns zero.  A row with an empty support
+// (LSE = +inf) gets a large finite value: its probabilities are zero either way, and an infinity would turn the zero
+// entries of the constant operand into NaN.
+__device__ __forceinline__ void write_row_constants(float *stats, size_t block, int row_in_block, float neg_lse2, float Dv, float scale_log2) {
+  const float c = fmaxf(__fdiv_rn(neg_lse2, scale_log2), -1.0e30f), nd = -Dv;
+  const uint32_t c0 = pack_bf16x2(c, 0.f), n0 = pack_bf16x2(nd, 0.f);
+  const float c_r1 = c - bf16_lo_to_f32(c0), n_r1 = nd - bf16_lo_to_f32(n0);
+  const uint32_t c1 = pack_bf16x2(c_r1, 0.f), n1 = pack_bf16x2(n_r1, 0.f);
+  const uint32_t c2 = pack_bf16x2(c_r1 - bf16_lo_to_f32(c1), 0.f), n2 = pack_bf16x2(n_r1 - bf16_lo_to_f32(n1), 0.f);
+  uint8_t *blk = reinterpret_cast<uint8_t *>(stats) + block * kExtBlockBytes + (row_in_block >> 3) * 256 + (row_in_block & 7) * 16;
+  *reinterpret_cast<uint4 *>(blk) = make_uint4(c0 | (c1 << 16), c2, 0u, 0u);
+  *reinterpret_cast<uint4 *>(blk + 128) = make_uint4(n0 | (n1 << 16), n2, 0u, 0u);
+}
+
 // ============================================================================================
 // dQ side
 // ============================================================================================
@@ -315,13 +334,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   uint8_t *sRes = smem;                                        // buffer rb: Q tile, then dO tile
   uint8_t *sKV = sRes + R * 2 * C::kBigTileBytes;              // stage s: K step tile, then V step tile
   uint8_t *sOut = sKV + S * C::kDqStageBytes;                  // staging (dQ tile, then Z tile) when separate
-  uint8_t *sO = sOut + (C::kSepStaging ? 2 * C::kBigTileBytes : 0);   // saved-output rows of the next tile (kPrefetchO), row-major
 
   __shared__ uint64_t bar_res_full[R], bar_res_free[R], bar_kv_full[S], bar_kv_empty[S];
-  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_acc_done, bar_acc_free, bar_drain[2];
+  __shared__ uint64_t bar_sdp_full[NB], bar_tr_ready[NB], bar_acc_done, bar_acc_free, bar_drain[2], bar_stats_ready[R];
   __shared__ uint32_t tmem_base_smem;
   __shared__ int cta_abort, cta_skip;
-  __shared__ float s_rho[C::kWG - 1][128], s_m[C::kWG - 1][128], s_lam[128], s_D[128], s_lse[128];
+  __shared__ float s_rho[C::kWG - 1][128], s_m[C::kWG - 1][128], s_lam[128], s_D[R][128], s_lse[R][128];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) cta_skip = *reinterpret_cast<volatile int *>(status);
@@ -333,7 +351,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
   AbortState ab{status, &cta_abort};
   if (threadIdx.x == 0) {
     cta_abort = 0;
-    for (int r = 0; r < R; ++r) { mbar_init(&bar_res_full[r], 1); mbar_init(&bar_res_free[r], 2); }
+    for (int r = 0; r < R; ++r) { mbar_init(&bar_res_full[r], 1); mbar_init(&bar_res_free[r], 2); mbar_init(&bar_stats_ready[r], 32); }
     for (int s = 0; s < S; ++s) { mbar_init(&bar_kv_full[s], 1); mbar_init(&bar_kv_empty[s], 1); }
     for (int b = 0; b < NB; ++b) { mbar_init(&bar_sdp_full[b], 1); mbar_init(&bar_tr_ready[b], 128 * C::kSlices); }
     mbar_init(&bar_acc_done, 1);
@@ -396,23 +414,68 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       }
     }
   } else if (warp == 3) {
-    // ---------------------------------------------------------------- TMA loader of the stationary (Q, dO) tiles
-    if (lane == 0) {
-      int ti = 0;
-      for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
-        const int rb = ti % R, bh = hix(lin), qrow0 = tile_of(lin).row0;
+    // ---------------------------------------------------------------- TMA loader of the stationary (Q, dO) tiles; with
+    // kLoaderStats the whole warp then prepares the tile's row constants (see below)
+    int ti = 0;
+    for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
+      const int rb = ti % R, bh = hix(lin);
+      const TileInfo tl = tile_of(lin);
+      if (lane == 0) {
         if (ti >= R) mbar_wait(&bar_res_free[rb], ((ti / R) - 1) & 1, ab, kDqWaitResFree);
         mbar_expect_tx(&bar_res_full[rb], 2 * C::kBigTileBytes);
         uint8_t *dst = sRes + rb * 2 * C::kBigTileBytes;
         for (int s = 0; s < C::kSlabs; ++s) {
-          tma_load_3d(dst + s * C::kBigSlabBytes, &tmQ, &bar_res_full[rb], s * 64, qrow0, bh);
-          tma_load_3d(dst + C::kBigTileBytes + s * C::kBigSlabBytes, &tmdO, &bar_res_full[rb], s * 64, qrow0, bh);
+          tma_load_3d(dst + s * C::kBigSlabBytes, &tmQ, &bar_res_full[rb], s * 64, tl.row0, bh);
+          tma_load_3d(dst + C::kBigTileBytes + s * C::kBigSlabBytes, &tmdO, &bar_res_full[rb], s * 64, tl.row0, bh);
         }
       }
-      if (cta_abort) {
-        for (int q = (ti > R ? ti - R : 0); q < ti; ++q)
-          for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_res_full[q % R], (q / R) & 1); ++spin) {}
+      __syncwarp();
+      if (C::kLoaderStats && ti > 0) {       // the first tile's are computed by the (then idle) compute warps: sixteen warps are faster
+        // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1), LSE, and the row-constant tile
+        // for the dK/dV side, for the four rows lane, lane + 32, ... of the tile: dO from the stationary tile in shared
+        // memory, O from global memory.  The sum keeps the order of the d = 128 path (eight elements by sequential FMAs,
+        // the eight partial sums by a butterfly).  The buffer pair rb is free: lane 0 has seen its release above.
+        mbar_wait(&bar_res_full[rb], (ti / R) & 1, ab, kDqWaitQ);
+        const size_t head_row0 = static_cast<size_t>(bh) * N;
+        const uint8_t *sdO = sRes + rb * 2 * C::kBigTileBytes + C::kBigTileBytes;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+          const int r = lane + 32 * it, qrow = tl.row0 + r;
+          float part[D / 8];
+#pragma unroll
+          for (int c = 0; c < D / 8; ++c) {
+            uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+            if (qrow < tl.seq_end) {
+              a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + qrow) * D) + c);
+              b = *reinterpret_cast<const uint4 *>(sdO + (c >> 3) * C::kBigSlabBytes + swz128_offset(r, c & 7));
+            }
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+            float acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+              acc = fmaf(bf16_lo_to_f32(aw[w]), bf16_lo_to_f32(bw[w]), acc);
+              acc = fmaf(bf16_hi_to_f32(aw[w]), bf16_hi_to_f32(bw[w]), acc);
+            }
+            part[c] = acc;
+          }
+#pragma unroll
+          for (int off = D / 16; off >= 1; off >>= 1)
+#pragma unroll
+            for (int c = 0; c < off; ++c) part[c] += part[c + off];
+          const float Dv = part[0];
+          const float lse_row = (qrow < tl.seq_end) ? LSE[head_row0 + qrow] : 0.f;
+          s_D[rb][r] = Dv;
+          s_lse[rb][r] = lse_row;
+          const int rel = qrow - tl.seq0;                  // row inside the sequence
+          if (rel < ((tl.seq_end - tl.seq0 + 63) / 64) * 64)
+            write_row_constants(stats, (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)), rel & 63, -lse_row * 1.4426950408889634f, Dv, scale_log2);
+        }
+        mbar_arrive(&bar_stats_ready[rb]);
       }
+    }
+    if (lane == 0 && cta_abort) {
+      for (int q = (ti > R ? ti - R : 0); q < ti; ++q)
+        for (int spin = 0; spin < 100000 && !mbar_try_wait(&bar_res_full[q % R], (q / R) & 1); ++spin) {}
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- tensor-core issuer 1: scores
@@ -492,22 +555,6 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
     int g0 = 0, ti = 0;
     constexpr int L = D / 8, RPI = 32 / L;               // D computation: lanes per row, rows per warp-wide load
     const int sub = lane / L, part = lane % L;
-    // kPrefetchO: the O rows and the LSE of tile lin_n travel to shared memory while the tile before it finishes
-    auto prefetch_tile = [&](int lin_n) {
-      const TileInfo tn = tile_of(lin_n);
-      const size_t hr0 = static_cast<size_t>(hix(lin_n)) * N;
-#pragma unroll
-      for (int it = 0; it < 8 / RPI; ++it) {
-        const int r = 8 * (warp - 4) + it * RPI + sub;
-        if (tn.row0 + r < tn.seq_end) cp_async16(sO + r * (D * 2) + part * 16, Og + (hr0 + tn.row0 + r) * D + part * 8);
-      }
-      if (wg == 0 && tn.row0 + row < tn.seq_end) cp_async4(&s_lse[row], LSE + hr0 + tn.row0 + row);
-      cp_async_commit();
-    };
-    if (C::kPrefetchO) {
-      const int lin0 = sched.peek();
-      if (lin0 >= 0) prefetch_tile(lin0);
-    }
     for (int lin = sched.next(); lin >= 0; lin = sched.next(), ++ti) {
       const TileInfo tl = tile_of(lin);
       const int bh = hix(lin), T = steps_of(tl), rb = ti % R;
@@ -517,29 +564,24 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
       const unsigned long long ev_n0 = global_ns(); const long long ev_c0 = clock64(); unsigned long long ev_n1 = 0, ev_n2 = 0;
 #endif
 
-      // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1): each of the 16 compute warps
-      // takes eight rows, 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
-      if (C::kPrefetchO) {
-        cp_async_wait_all();                                      // this thread's share of the O rows and LSE
-        mbar_wait(&bar_res_full[rb], (ti / R) & 1, ab, kDqWaitQ);   // dO is read from the stationary tile
-        named_bar_sync(2, C::kCompute);                           // everybody's share
-      }
-      // read before the barrier below: the next tile's prefetch, which overwrites it, is issued behind that barrier
-      const float lse_pre = C::kPrefetchO ? s_lse[row] : 0.f;
-      {
+      float Dv, lse_row;
+      if (C::kLoaderStats && ti > 0) {
+        // prepared by the loader's warp while the previous tile ran
+        mbar_wait(&bar_res_full[rb], (ti / R) & 1, ab, kDqWaitQ);       // the tile's Q is read in the epilogue
+        mbar_wait(&bar_stats_ready[rb], ((ti - 1) / R) & 1, ab, kDqWaitQ);
+        Dv = s_D[rb][row];
+        lse_row = s_lse[rb][row];
+      } else {
+        if (C::kLoaderStats) mbar_wait(&bar_res_full[rb], (ti / R) & 1, ab, kDqWaitQ);
+        // D_i = sum_c dO_ic O_ic from the saved BF16 output, FP32 (Algorithm 1 line 1): each of the 16 compute warps
+        // takes eight rows, 16-byte loads (D/8 lanes share a row) and a shuffle reduction.
 #pragma unroll
         for (int it = 0; it < 8 / RPI; ++it) {
           const int r = 8 * (warp - 4) + it * RPI + sub;
           uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
           if (tl.row0 + r < tl.seq_end) {
-            if (C::kPrefetchO) {
-              a = *reinterpret_cast<const uint4 *>(sO + r * (D * 2) + part * 16);
-              b = *reinterpret_cast<const uint4 *>(sRes + rb * 2 * C::kBigTileBytes + C::kBigTileBytes + (part >> 3) * C::kBigSlabBytes +
-                                                   swz128_offset(r, part & 7));
-            } else {
-              a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + tl.row0 + r) * D) + part);
-              b = __ldg(reinterpret_cast<const uint4 *>(dOg + (head_row0 + tl.row0 + r) * D) + part);
-            }
+            a = __ldg(reinterpret_cast<const uint4 *>(Og + (head_row0 + tl.row0 + r) * D) + part);
+            b = __ldg(reinterpret_cast<const uint4 *>(dOg + (head_row0 + tl.row0 + r) * D) + part);
           }
           const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
           float acc = 0.f;
@@ -550,32 +592,17 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
           }
 #pragma unroll
           for (int off = L / 2; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-          if (part == 0) s_D[r] = acc;
+          if (part == 0) s_D[rb][r] = acc;
         }
+        named_bar_sync(2, C::kCompute);
+        Dv = s_D[rb][row];
+        lse_row = (qrow < tl.seq_end) ? LSE[head_row0 + qrow] : 0.f;
+        // Row constants for the dK/dV side, per 64-row block of a sequence (the last one padded with zeros).
+        const int rel = qrow - tl.seq0;                  // row inside the sequence
+        if (wg == 0 && rel < ((tl.seq_end - tl.seq0 + 63) / 64) * 64)
+          write_row_constants(stats, static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6), rel & 63, -lse_row * 1.4426950408889634f, Dv, scale_log2);
       }
-      named_bar_sync(2, C::kCompute);
-      const float Dv = s_D[row];
-      const float lse_row = (qrow < tl.seq_end) ? (C::kPrefetchO ? lse_pre : LSE[head_row0 + qrow]) : 0.f;
       const float neg_lse2 = -lse_row * 1.4426950408889634f;
-      // Row constants for the dK/dV side, per 64-row block of a sequence (the last one padded with zeros).
-      const int rel = qrow - tl.seq0;                  // row inside the sequence
-      if (wg == 0 && rel < ((tl.seq_end - tl.seq0 + C::kStepRows - 1) / C::kStepRows) * C::kStepRows) {
-        // The dK/dV side takes both row constants through its score products instead of reading them per column.  Per
-        // 64-row block a K-major operand tile of 16 BF16 columns without swizzle (eight-row groups of 256 bytes: the
-        // rows' first eight columns, then their last eight): columns 0..2 hold -LSE / alpha and columns 8..10 hold -D,
-        // each as three BF16 pieces whose sum is the FP32 value, the other columns zero.  A row with an empty support
-        // (LSE = +inf) gets a large finite value: its probabilities are zero either way, and an infinity would turn the
-        // zero entries of the constant operand into NaN.
-        const float c = fmaxf(__fdiv_rn(neg_lse2, scale_log2), -1.0e30f), nd = -Dv;
-        const uint32_t c0 = pack_bf16x2(c, 0.f), n0 = pack_bf16x2(nd, 0.f);
-        const float c_r1 = c - bf16_lo_to_f32(c0), n_r1 = nd - bf16_lo_to_f32(n0);
-        const uint32_t c1 = pack_bf16x2(c_r1, 0.f), n1 = pack_bf16x2(n_r1, 0.f);
-        const uint32_t c2 = pack_bf16x2(c_r1 - bf16_lo_to_f32(c1), 0.f), n2 = pack_bf16x2(n_r1 - bf16_lo_to_f32(n1), 0.f);
-        uint8_t *blk = reinterpret_cast<uint8_t *>(stats) + (static_cast<size_t>(bh) * nblk + tl.blk0 + (rel >> 6)) * kExtBlockBytes +
-                       ((rel & 63) >> 3) * 256 + (rel & 7) * 16;
-        *reinterpret_cast<uint4 *>(blk) = make_uint4(c0 | (c1 << 16), c2, 0u, 0u);
-        *reinterpret_cast<uint4 *>(blk + 128) = make_uint4(n0 | (n1 << 16), n2, 0u, 0u);
-      }
 
       uint64_t rho2 = f32x2(0.f, 0.f), msum2 = f32x2(0.f, 0.f);
 #ifdef GPROJ_TRACE
@@ -605,12 +632,6 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ,    // box 64 x 128 rows
 #ifdef GPROJ_TRACE
       ev_n2 = global_ns();
 #endif
-      if (C::kPrefetchO) {
-        // every thread took its D and LSE out of shared memory before its first step (behind the barrier above), and dO of
-        // the next tile sits in the other stationary buffer: the next tile's rows may travel during this tile's epilogue
-        const int lin_n = sched.peek();
-        if (lin_n >= 0) prefetch_tile(lin_n);
-      }
       // ---- row statistics of all warpgroups (fixed order), lambda = rho / m with the zero-mass rule (Algorithm 1 line 14)
       float rho_lo, rho_hi, m_lo, m_hi;
       f32x2_split(rho2, rho_lo, rho_hi);

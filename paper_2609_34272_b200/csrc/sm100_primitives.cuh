@@ -173,17 +173,6 @@ __device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async
 
 // Byte offset of 16-byte chunk `chunk16` (0..7) of row `row` inside a 128-byte-row slab laid out with the
 // 128-byte swizzle TMA uses (chunk index XOR row mod 8).  Slab bases are 1024-byte aligned.
-// Per-thread asynchronous copies global -> shared memory (no register staging): issued early, waited for where the data
-// is needed; other threads see the bytes after the issuing thread's wait and a barrier.
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async4(void *smem_dst, const void *gmem_src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-
 __device__ __forceinline__ uint32_t swz128_offset(int row, int chunk16) {
   return static_cast<uint32_t>(row) * 128u + (static_cast<uint32_t>(chunk16 ^ (row & 7)) << 4);
 }

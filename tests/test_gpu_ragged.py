@@ -189,3 +189,25 @@ def test_head_shards_give_the_bits_of_the_whole_call(d, causal):
             assert torch.equal(dq2, fl(dQ)[:, sl]) and torch.equal(dk2, fl(dK)[:, sl]) and torch.equal(dv2, fl(dV)[:, sl]), (world, r)
     rc, detail = g.gproj_last_device_status()
     assert rc == 0, hex(detail)
+
+
+@pytest.mark.parametrize("B,H,N,d,causal", [(2, 24, 1000, 64, True), (1, 160, 300, 64, False), (2, 80, 257, 128, True), (1, 300, 65, 64, True)])
+def test_ragged_lengths_with_several_tiles_per_cta(B, H, N, d, causal):
+    # More tiles than twice the SM count, with a ragged last tile in every head: a CTA walks three or more tiles, so the
+    # per-tile hand-overs that only start at a CTA's second and third tile (row constants prepared one tile ahead in the
+    # other stationary buffer, buffers reused across tiles) are exercised on ragged data.  The oracle runs on eight heads.
+    w = Workload("ragged_many", B, H, N, d, causal, k_offset=8.0, seed=900 + N + H)
+    inp = make_inputs(w)
+    dev = {k: v.cuda() for k, v in inp.items()}
+    O, LSE = g.gproj_attn_fwd(dev["Q"], dev["K"], dev["V"], w.softmax_scale, causal)
+    dQ, dK, dV = g.gproj_attn_bwd(dev["Q"], dev["K"], dev["V"], O, LSE, dev["dO"], w.softmax_scale, causal)
+    rc, detail = g.gproj_last_device_status()
+    assert rc == 0, (g.status_string(rc), hex(detail))
+    rng = np.random.default_rng(N + H)
+    for hh in sorted(set(rng.integers(0, B * H, size=6).tolist()) | {0, B * H - 1}):
+        b, h = divmod(hh, H)
+        one = lambda t: t[b:b + 1, h:h + 1]
+        ex = oracle.attn_fwd_bwd_f64(*(bits(one(inp[k])) for k in ("Q", "K", "V", "dO")), w.softmax_scale, causal)
+        got = {"O": to_np(one(O)), "LSE": LSE[b:b + 1, h:h + 1].cpu().numpy().astype(np.float64),
+               "dQ": to_np(one(dQ)), "dK": to_np(one(dK)), "dV": to_np(one(dV))}
+        check(got, ex)
